@@ -1,0 +1,403 @@
+#!/usr/bin/env python
+"""Benchmark of the W4A4 linear hot path (rotate -> INT4 quantise -> INT4 GEMM -> dequant).
+
+One step = one pass of the whole path (sq_linear) over one batch of synthetic activations of
+the named workload.  Prints ONE JSON line.
+
+  python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+
+N > 1: launched under torchrun, one process per GPU; the path shards over tokens with no
+collective (each rank owns its own batch and a replica of the packed weights), so scaling is
+"weak" and the only communication is the barrier / max-over-ranks of the timing.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+from paper_2511_22316_b200 import workloads as wl  # noqa: E402
+
+METRIC = "w4a4_linear_tops"
+UNIT = "TOPS"
+DEFAULT_WORKLOAD = wl.L7B_QKVO.name
+FALLBACK_PEAKS = {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0}
+INT8_OVER_BF16 = 2.0      # nominal dense ratio (4.5 POPS int8 : 2.25 PFLOP/s bf16)
+
+# dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
+# profiles/ (bytes; None until a capture exists for that kernel and workload).
+NCU_TRAFFIC = {}
+
+
+def peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    try:
+        with open(path) as f:
+            p = json.load(f)
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "source": "measured"}
+    except Exception:
+        d = dict(FALLBACK_PEAKS)
+        d["source"] = "fallback"
+        return d
+
+
+def ops_per_step(w):
+    return 2.0 * w.M * w.N * w.K
+
+
+def rotate_quant_bytes(w):
+    """Algorithmic HBM bytes of steps 1+2 per launch: read fp16 row, write packed row + step."""
+    return w.M * (2.0 * w.n + w.n / 2.0 + 2.0)
+
+
+def gemm_bytes(w):
+    return (w.M + w.N) * w.K / 2.0 + 2.0 * w.M * w.N + 2.0 * (w.M + w.N)
+
+
+# ----------------------------------------------------------------------------------------------
+# clock sampling during the timed region
+# ----------------------------------------------------------------------------------------------
+class ClockSampler:
+    QUERY = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,"
+             "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
+             "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu = gpu_index
+        self.proc = None
+        self.lines = []
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu}", f"--query-gpu={self.QUERY}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except Exception:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=5)
+        except Exception:
+            self.proc.kill()
+        sm, smax, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [x.strip() for x in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                smax.append(float(f[2]))
+            except ValueError:
+                continue
+            for name, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None,
+                "sm_max_mhz": max(smax) if smax else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+# ----------------------------------------------------------------------------------------------
+# CPU oracle arm (also `--impl reference`)
+# ----------------------------------------------------------------------------------------------
+class OracleArm:
+    """The oracle, as it stands, on the first `rows` token rows of the workload against the full
+    weight matrix.  The weights are rotated+quantised once, untimed: that is offline setup on the
+    GPU side too.  One pass = rotate, quantise, pack, integer GEMM, dequantise."""
+
+    def __init__(self, w, rows: int, X=None, W=None):
+        from oracle import singlequant_oracle as ora
+        self.ora = ora
+        self.w = w
+        X = wl.make_activations(w) if X is None else X
+        W = wl.make_weights(w) if W is None else W
+        self.R1, self.R2 = ora.build_rotation(X.astype(np.float32), w.n1, w.n2)
+        Wq, self.sw, _ = ora.pack_weight(W, self.R1, self.R2)
+        self.Wc = ora.unpack_int4(Wq)
+        self.rows = min(rows, w.M)
+        self.Xs = X[:self.rows]
+        self.sample = (f"first {self.rows} of {w.M} token rows per pass against the full "
+                       f"{w.N}x{w.K} weight matrix")
+
+    def one_pass(self):
+        ora = self.ora
+        Xq, sx, _ = ora.rotate_quant(self.Xs, self.R1, self.R2)
+        acc = ora.gemm_i32(ora.unpack_int4(Xq), self.Wc)
+        return ora.dequant(acc, sx, self.sw)
+
+    def timed_pass(self) -> float:
+        t0 = time.perf_counter()
+        self.one_pass()
+        return time.perf_counter() - t0
+
+    def tops(self, seconds: float) -> float:
+        return 2.0 * self.rows * self.w.N * self.w.K / seconds / 1e12
+
+    @staticmethod
+    def threads() -> int:
+        try:
+            from threadpoolctl import threadpool_info
+            return max([p.get("num_threads", 1) for p in threadpool_info()] + [1])
+        except Exception:
+            return len(os.sched_getaffinity(0))
+
+
+def run_reference(args, w):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return 0
+    arm = OracleArm(w, rows=256)
+    for _ in range(args.warmup):
+        arm.one_pass()
+    times = [arm.timed_pass() for _ in range(args.steps)]
+    dt = statistics.mean(times)
+    value = arm.tops(dt)
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": 1e3 * dt,
+        "higher_is_better": True, "scaling": "weak", "vs_baseline": None, "dtype": "f64",
+        "data": "synthetic",
+        "config": {"workload": w.name, "M": w.M, "N": w.N, "K": w.K, "sample": arm.sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": arm.threads(), "kind": "oracle",
+                         "sample": arm.sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+    return 0
+
+
+# ----------------------------------------------------------------------------------------------
+# CUDA arm
+# ----------------------------------------------------------------------------------------------
+def run_ours(args, w):
+    import torch
+    from paper_2511_22316_b200 import binding as sq
+    from paper_2511_22316_b200 import build as sqbuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if rank == 0 or world == 1:
+        sqbuild.build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    sq.load()
+
+    M, N, K = w.M, w.N, w.K
+    # every rank draws its own batch (weak scaling over tokens); the weights are replicated
+    import dataclasses
+    w_rank = dataclasses.replace(w, seed=w.seed + 7919 * rank) if rank else w
+    X = wl.make_activations(w_rank)
+    W = wl.make_weights(w)
+    rot = sq.sq_build_rotation(X.astype(np.float32), w.n1, w.n2, seed=0)
+
+    dW = torch.from_numpy(W).cuda()
+    Wq = torch.empty((N, K // 2), dtype=torch.uint8, device="cuda")
+    sw = torch.empty((N,), dtype=torch.float16, device="cuda")
+    sq.sq_pack_weight(rot, dW, N, K, Wq, sw)
+    torch.cuda.synchronize()
+    del dW
+
+    # ring of buffer sets larger than L2 so that no step finds its inputs cached
+    l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
+    per_set = M * K * 2 + M * K // 2 + M * N * 2 + N * K // 2
+    nsets = max(2, int(np.ceil(1.5 * l2 / per_set)) + 1)
+    ws_bytes = sq.sq_linear_workspace_bytes(M, N, K)
+    Xh = torch.from_numpy(X).pin_memory()
+    sets = []
+    for i in range(nsets):
+        ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
+        off = (-ws.data_ptr()) % 256
+        sets.append({
+            "X": Xh.cuda(non_blocking=False).clone(),
+            "Wq": Wq.clone(), "sw": sw.clone(),
+            "Y": torch.empty((M, N), dtype=torch.float16, device="cuda"),
+            "ws": ws, "ws_ptr": ws.data_ptr() + off,
+            "Xq": torch.empty((M, K // 2), dtype=torch.uint8, device="cuda"),
+            "sx": torch.empty((M,), dtype=torch.float16, device="cuda"),
+        })
+    gws_bytes = sq.sq_w4a4_gemm_workspace_bytes(M, N, K)
+    gws = torch.empty(max(gws_bytes, 256), dtype=torch.uint8, device="cuda")
+
+    def step(i):
+        s = sets[i % nsets]
+        sq.sq_linear(rot, s["X"], M, s["Wq"], s["sw"], N, K, s["ws_ptr"], ws_bytes, s["Y"])
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    for i in range(max(args.warmup, 3)):
+        step(i)
+    sync_all()
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+
+    # ---- timed region: exactly K steps of sq_linear ------------------------------------------
+    launches0 = sq.sq_kernel_launch_count()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    sync_all()
+    e0.record()
+    for i in range(args.steps):
+        step(i)
+    e1.record()
+    sync_all()
+    ms_total = e0.elapsed_time(e1)
+    launches = sq.sq_kernel_launch_count() - launches0
+
+    # ---- attribution: the same two kernels, launched through their own entry points, each
+    # bracketed by events on the launching stream (same ring, same stream, right after) -------
+    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(args.steps)]
+    for i in range(args.steps):
+        s = sets[i % nsets]
+        ev[i][0].record()
+        sq.sq_rotate_quant_act(rot, s["X"], M, s["Xq"], s["sx"])
+        ev[i][1].record()
+        sq.sq_w4a4_gemm(s["Xq"], s["sx"], s["Wq"], s["sw"], M, N, K, s["Y"], None,
+                        gws if gws_bytes else None, gws_bytes)
+        ev[i][2].record()
+    torch.cuda.synchronize()
+    rq_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+    gemm_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+
+    # ---- end to end: host activations in, host outputs out, through sq_linear_host ------------
+    hws_bytes = sq.sq_linear_host_workspace_bytes(M, N, K)
+    hws = torch.empty(hws_bytes + 256, dtype=torch.uint8, device="cuda")
+    hoff = (-hws.data_ptr()) % 256
+    Yh = torch.empty((M, N), dtype=torch.float16).pin_memory()
+    e2e_steps = max(3, min(args.steps, 20))
+    for _ in range(2):
+        sq.sq_linear_host(rot, Xh, M, sets[0]["Wq"], sets[0]["sw"], N, K, hws.data_ptr() + hoff, hws_bytes, Yh)
+    sync_all()
+    h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    h0.record()
+    for i in range(e2e_steps):
+        s = sets[i % nsets]
+        sq.sq_linear_host(rot, Xh, M, s["Wq"], s["sw"], N, K, hws.data_ptr() + hoff, hws_bytes, Yh)
+    h1.record()
+    sync_all()
+    e2e_ms = h0.elapsed_time(h1) / e2e_steps
+    status = sq.sq_last_device_status()
+
+    clocks = sampler.stop() if rank == 0 else None
+
+    # ---- max over ranks ---------------------------------------------------------------------
+    t = torch.tensor([ms_total, e2e_ms, rq_ms, gemm_ms], dtype=torch.float64, device="cuda")
+    if dist is not None:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    ms_total, e2e_ms, rq_ms, gemm_ms = (float(x) for x in t.tolist())
+    ms_per_step = ms_total / args.steps
+
+    if rank == 0:
+        pk = peaks()
+        value = world * ops_per_step(w) / (ms_per_step * 1e-3) / 1e12
+        e2e_value = world * ops_per_step(w) / (e2e_ms * 1e-3) / 1e12
+        gemm_tops = ops_per_step(w) / (gemm_ms * 1e-3) / 1e12
+        rq_gbs = rotate_quant_bytes(w) / (rq_ms * 1e-3) / 1e9
+        int8_peak = pk["bf16_tflops"] * INT8_OVER_BF16
+        roof_gemm = {"kernel": "w4a4_gemm_tc_kernel", "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak,
+                     "unit": "TOP/s", "frac": gemm_tops / int8_peak,
+                     "traffic": NCU_TRAFFIC.get(("gemm", w.name)),
+                     "peak_source": f"{pk['source']} bf16 burst x{INT8_OVER_BF16:g} (nominal int8:bf16 ratio)",
+                     "ms_per_launch": gemm_ms, "algorithmic_ops": ops_per_step(w),
+                     "frac_of_spec_4500": gemm_tops / 4500.0}
+        roof_rq = {"kernel": "rotate_quant_kernel", "bound": "hbm", "achieved": rq_gbs, "peak": pk["hbm_gbs"],
+                   "unit": "GB/s", "frac": rq_gbs / pk["hbm_gbs"],
+                   "traffic": NCU_TRAFFIC.get(("rotate_quant", w.name)),
+                   "peak_source": f"{pk['source']} copy bandwidth", "ms_per_launch": rq_ms,
+                   "algorithmic_bytes": rotate_quant_bytes(w), "frac_of_spec_8000": rq_gbs / 8000.0}
+        dominant, other = (roof_gemm, roof_rq) if gemm_ms >= rq_ms else (roof_rq, roof_gemm)
+
+        cpu = None
+        if world == 1:
+            arm = OracleArm(w, rows=256, X=X, W=W)
+            arm.one_pass()
+            times, t_start = [], time.perf_counter()
+            while time.perf_counter() - t_start < 10.0 or not times:
+                times.append(arm.timed_pass())
+            cpu = {"value": arm.tops(statistics.mean(times)), "unit": UNIT, "cores": arm.threads(),
+                   "kind": "oracle", "sample": f"{arm.sample}; {len(times)} passes, "
+                                               f"{statistics.mean(times):.3f} s per pass"}
+        line = {
+            "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "int8",
+            "data": "synthetic",
+            "config": {"workload": w.name, "M_per_gpu": M, "N": N, "K": K, "n1": w.n1, "n2": w.n2,
+                       "parallelism": f"token-sharded x{world}, no collective",
+                       "l2": f"ring of {nsets} buffer sets ({nsets * per_set / 1e6:.0f} MB > L2 "
+                             f"{l2 / 1e6:.0f} MB)"},
+            "roofline": dominant,
+            "roofline_other": other,
+            "kernel_ms": {"rotate_quant": rq_ms, "w4a4_gemm": gemm_ms, "sum": rq_ms + gemm_ms,
+                          "step": ms_per_step},
+            "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": M * K * 2,
+                    "d2h_bytes_per_step": M * N * 2, "api": "sq_linear_host (pinned host X -> host Y)"},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "device_status": status,
+        }
+        if cpu is not None:
+            line["cpu_baseline"] = cpu
+        print(json.dumps(line))
+    if dist is not None:
+        dist.barrier()
+        dist.destroy_process_group()
+    return 0
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=50)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    args = ap.parse_args()
+    w = wl.by_name(args.workload)
+    if args.impl == "reference":
+        return run_reference(args, w)
+    return run_ours(args, w)
+
+
+if __name__ == "__main__":
+    sys.exit(main())

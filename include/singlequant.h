@@ -1,0 +1,154 @@
+/*
+ * singlequant.h - C ABI of the B200 (sm_100a) W4A4 linear hot path of SingleQuant.
+ *
+ * The path (paper, Section "SingleQuant"):
+ *   step 1  Kronecker rotation of every activation token: the length-n row is viewed as an
+ *           n1 x n2 row-major matrix X~_t and Z_t = R1^T X~_t R2       (Eq. "eq18", and the
+ *           per-slice form of the mode products that follows it);
+ *   step 2  per-token symmetric INT4 quantisation Q_Delta(z) = Delta*floor(z/Delta + 1/2)
+ *           (Section 3.2) with Delta_t = fp16(max|Z_t| / 7), two codes per byte;
+ *   step 3  INT4 x INT4 GEMM against weights rotated offline by the same operator
+ *           (Flat(W~_R) = W^T R), int32 accumulation, dequantisation by token step x channel
+ *           step to fp16                                  (X W = Flat(X~_R) Flat(W~_R)^T).
+ *
+ * General conventions
+ *   - Pointers marked HOST are ordinary host memory; pointers marked DEVICE are CUDA device
+ *     memory of the device that was current when the rotation handle was created.  The
+ *     caller owns every buffer; the library allocates only the sq_rotation_t handle (and the
+ *     device copies of R1, R2 inside it), freed by sq_rotation_destroy.
+ *   - All matrices are dense row-major.  X is [M x n] (one token per row, ld = n), W is
+ *     [N x K] with K = n (one OUTPUT channel per row), Y is [M x N].
+ *   - Packed INT4 layout (public, canonical): row r, byte j holds channel 2j in its low nibble
+ *     and channel 2j+1 in its high nibble, two's complement, row stride K/2 bytes.
+ *   - Steps (scales) are IEEE fp16.  The step used to quantise is the ROUNDED fp16 value.
+ *   - DEVICE pointers must be 16-byte aligned; K (= n) must be even.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream).  Device
+ *     calls only enqueue work and never synchronise, except where stated.
+ *   - Every call validates its arguments on the host before any launch and reports problems
+ *     through the return code; nothing throws, aborts or traps.  M = 0 or N = 0 is SQ_OK and
+ *     a no-op.
+ *   - Kernels wait on hardware barriers with bounded spins; a wait that runs out sets a
+ *     device status word that sq_last_device_status returns as SQ_ERR_TIMEOUT.
+ */
+#ifndef SINGLEQUANT_H_
+#define SINGLEQUANT_H_
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+  SQ_OK = 0,
+  SQ_ERR_INVALID_ARG = 1,   /* NULL pointer, negative size, bad flag                         */
+  SQ_ERR_SHAPE = 2,         /* n1*n2 != n, odd K, K mismatch with the rotation, ...          */
+  SQ_ERR_ALIGN = 3,         /* a DEVICE pointer is not 16-byte aligned                       */
+  SQ_ERR_UNSUPPORTED = 4,   /* a size beyond what the kernels handle (stated per call)       */
+  SQ_ERR_NOMEM = 5,         /* allocation of the handle failed / workspace too small         */
+  SQ_ERR_CUDA = 6,          /* a CUDA runtime or driver call failed                          */
+  SQ_ERR_TIMEOUT = 7        /* a bounded device-side wait ran out (see sq_last_device_status) */
+} sq_status_t;
+
+typedef struct sq_rotation sq_rotation_t;   /* opaque: host + device copies of R1 and R2 */
+
+/* Components of R = (R1^U R^A)^T (x) (H R2^U); a cleared bit replaces that component by the
+ * identity (the paper's ablation of ART and URT). */
+enum { SQ_ROT_ART = 1, SQ_ROT_URT = 2, SQ_ROT_HADAMARD = 4, SQ_ROT_DEFAULT = 7 };
+
+/* Algorithm 1 (Kronecker Dimension Factorization).  Host only.  n2 = the power of two dividing
+ * n closest to sqrt(n), the first found winning ties; n1 = n / n2.  n >= 1. */
+sq_status_t sq_factorize(int64_t n, int32_t* n1, int32_t* n2);
+
+/* Builds R1 = (R1^U R^A)^T [n1 x n1] and R2 = H R2^U [n2 x n2] (paragraphs "Alignment Rotation
+ * Transformation", "Uniformity Rotation Transformation", "The Overall SingleQuant Method") in
+ * float64 on the host from one calibration batch, stores them as fp32, copies them to the
+ * current device and returns a handle.  Host-synchronous.
+ *   calib      HOST fp32 [T x n] row-major, T >= 1
+ *   n1, n2     n1*n2 == n; n2 must be a power of two when SQ_ROT_HADAMARD is set
+ *   flags      SQ_ROT_* bits
+ *   seed       seeds the library's own generator for the random orthogonal block O of ART when
+ *              O_or_null is NULL
+ *   O_or_null  HOST fp64 [(n1-2) x (n1-2)] orthogonal block for ART, or NULL
+ *   out        receives the handle
+ * The vectors ART/URT are built from: the calibration token with the largest |entry| is
+ * reshaped to n1 x n2; ART and URT_1 use the column holding that entry; URT_2 uses the row of
+ * the left-rotated token with the largest |entry|, after the Hadamard mix. */
+sq_status_t sq_build_rotation(const float* calib, int64_t T, int64_t n, int32_t n1, int32_t n2,
+                              uint32_t flags, uint64_t seed, const double* O_or_null,
+                              sq_rotation_t** out);
+
+/* Wraps caller-made factors (HOST fp32, row-major, R1 [n1 x n1], R2 [n2 x n2]) in a handle.
+ * No orthogonality check is made. */
+sq_status_t sq_rotation_from_factors(const float* R1, const float* R2, int32_t n1, int32_t n2,
+                                     sq_rotation_t** out);
+
+/* Copies the fp32 factors back to HOST buffers of n1*n1 and n2*n2 floats. */
+sq_status_t sq_rotation_get_factors(const sq_rotation_t* rot, float* R1, float* R2);
+sq_status_t sq_rotation_dims(const sq_rotation_t* rot, int32_t* n1, int32_t* n2);
+void sq_rotation_destroy(sq_rotation_t* rot);
+
+/* Steps 1+2, fused: Z_t = R1^T X~_t R2 in fp32 on chip, Delta_t = fp16(max|Z_t|/7),
+ * code = clamp(floor(fl(fl(z * fl(1/Delta)) + 0.5)), -8, 7) in fp32 arithmetic, packed.
+ *   rot           handle; n = n1*n2 of the handle.  Supported: n even, n <= 32768.
+ *   X             DEVICE fp16 [M x n]
+ *   Xq            DEVICE uint8 [M x n/2]   (out)
+ *   sx            DEVICE fp16 [M]          (out; Delta_t; 0 for an all-zero row)
+ *   Zdbg_or_null  DEVICE fp32 [M x n]      (out, optional: the rotated rows, for parity tests) */
+sq_status_t sq_rotate_quant_act(const sq_rotation_t* rot, const void* X, int64_t M,
+                                void* Xq, void* sx, void* Zdbg_or_null, void* stream);
+
+/* Offline weight path: the same operator on the rows of W (Flat(W~_R) = W^T R), then
+ * round-to-nearest INT4 with one step per output channel.
+ *   rot_or_null   NULL = identity rotation (plain per-channel INT4)
+ *   W             DEVICE fp16 [N x K], K == n of the handle
+ *   Wq            DEVICE uint8 [N x K/2]   (out)
+ *   sw            DEVICE fp16 [N]          (out) */
+sq_status_t sq_pack_weight(const sq_rotation_t* rot_or_null, const void* W, int64_t N, int64_t K,
+                           void* Wq, void* sw, void* stream);
+
+/* Step 3: acc[t,c] = sum_k Xq[t,k] * Wq[c,k] (int32, exact), Y[t,c] = fp16(acc * sx[t] * sw[c]).
+ *   Xq  DEVICE uint8 [M x K/2]     sx  DEVICE fp16 [M]
+ *   Wq  DEVICE uint8 [N x K/2]     sw  DEVICE fp16 [N]
+ *   Y   DEVICE fp16  [M x N] (out)
+ *   accdbg_or_null  DEVICE int32 [M x N] (out, optional: the raw accumulators)
+ *   workspace       DEVICE scratch of at least sq_w4a4_gemm_workspace_bytes(M,N,K) bytes, or
+ *                   NULL (then small-M problems run without split-K, slower but identical)
+ * Supported: K even, K <= 65536 (so that the 256x-scaled int32 accumulator cannot overflow).
+ * The tensor-core path needs K % 128 == 0 and N % 8 == 0; other shapes run a plain integer
+ * kernel with the same results. */
+size_t sq_w4a4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+sq_status_t sq_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw,
+                         int64_t M, int64_t N, int64_t K, void* Y, void* accdbg_or_null,
+                         void* workspace, size_t workspace_bytes, void* stream);
+
+/* The whole layer on one stream: steps 1+2 into the workspace (Xq, sx), then step 3.
+ *   workspace  DEVICE, at least sq_linear_workspace_bytes(M, N, K) bytes, 256-byte aligned */
+size_t sq_linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
+sq_status_t sq_linear(const sq_rotation_t* rot, const void* X, int64_t M,
+                      const void* Wq, const void* sw, int64_t N, int64_t K,
+                      void* workspace, size_t workspace_bytes, void* Y, void* stream);
+
+/* The whole layer from HOST activations to HOST outputs: copies X (HOST fp16 [M x n], pinned
+ * memory recommended) to the device, runs sq_linear, copies Y back (HOST fp16 [M x N]) and
+ * waits for the stream.  Weights stay on the device.
+ *   workspace  DEVICE, at least sq_linear_host_workspace_bytes(M, N, K) bytes */
+size_t sq_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K);
+sq_status_t sq_linear_host(const sq_rotation_t* rot, const void* X_host, int64_t M,
+                           const void* Wq, const void* sw, int64_t N, int64_t K,
+                           void* workspace, size_t workspace_bytes, void* Y_host, void* stream);
+
+/* Synchronises `stream`, then returns and clears the device status word: SQ_OK, or
+ * SQ_ERR_TIMEOUT if any kernel since the last call gave up a bounded wait, or SQ_ERR_CUDA. */
+sq_status_t sq_last_device_status(void* stream);
+
+/* Number of kernels this library has launched in the calling process (monotonic counter). */
+uint64_t sq_kernel_launch_count(void);
+
+const char* sq_status_string(sq_status_t s);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SINGLEQUANT_H_ */

@@ -1,0 +1,262 @@
+// C ABI entry points: argument validation on the host, then the kernel launchers.
+#include <cmath>
+#include <cstring>
+#include <new>
+
+#include "sq_internal.h"
+#include "sq_ptx.cuh"
+
+namespace sq {
+std::atomic<uint64_t> g_launches{0};
+
+sq_status_t read_and_clear_device_status(cudaStream_t s) {
+  if (cudaStreamSynchronize(s) != cudaSuccess) return SQ_ERR_CUDA;
+  unsigned int v = 0;
+  if (cudaMemcpyFromSymbol(&v, g_device_status, sizeof(v)) != cudaSuccess) return SQ_ERR_CUDA;
+  if (v != 0) {
+    const unsigned int zero = 0;
+    if (cudaMemcpyToSymbol(g_device_status, &zero, sizeof(zero)) != cudaSuccess) return SQ_ERR_CUDA;
+    return SQ_ERR_TIMEOUT;
+  }
+  return SQ_OK;
+}
+}  // namespace sq
+
+namespace {
+
+constexpr int64_t kMaxN = 32768;       // rotate+quant: the row and its fp32 image stay in shared memory
+constexpr int64_t kMaxK = 65536;       // GEMM: 256 * 64 * K must fit in int32
+constexpr int64_t kMaxRows = (1ll << 31) - 1;
+
+inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
+
+sq_status_t make_handle(std::vector<float>&& R1, std::vector<float>&& R2, int32_t n1, int32_t n2,
+                        sq_rotation_t** out) {
+  sq_rotation* h = new (std::nothrow) sq_rotation();
+  if (!h) return SQ_ERR_NOMEM;
+  h->n1 = n1;
+  h->n2 = n2;
+  h->R1 = std::move(R1);
+  h->R2 = std::move(R2);
+  if (cudaGetDevice(&h->device) != cudaSuccess) {
+    delete h;
+    return SQ_ERR_CUDA;
+  }
+  const size_t b1 = sizeof(float) * h->R1.size(), b2 = sizeof(float) * h->R2.size();
+  if (cudaMalloc(&h->dR1, b1) != cudaSuccess || cudaMalloc(&h->dR2, b2) != cudaSuccess ||
+      cudaMemcpy(h->dR1, h->R1.data(), b1, cudaMemcpyHostToDevice) != cudaSuccess ||
+      cudaMemcpy(h->dR2, h->R2.data(), b2, cudaMemcpyHostToDevice) != cudaSuccess) {
+    cudaGetLastError();
+    if (h->dR1) cudaFree(h->dR1);
+    if (h->dR2) cudaFree(h->dR2);
+    delete h;
+    return SQ_ERR_CUDA;
+  }
+  *out = h;
+  return SQ_OK;
+}
+
+sq_status_t check_rows_args(const void* in, const void* q, const void* sc, const void* dbg, int64_t rows,
+                            int64_t n) {
+  if (rows < 0 || rows > kMaxRows) return SQ_ERR_INVALID_ARG;
+  if (n < 2 || (n & 1)) return SQ_ERR_SHAPE;
+  if (n > kMaxN) return SQ_ERR_UNSUPPORTED;
+  if (rows == 0) return SQ_OK;
+  if (!in || !q || !sc) return SQ_ERR_INVALID_ARG;
+  if (!sq::aligned16(in) || !sq::aligned16(q) || !sq::aligned16(sc) || !sq::aligned16(dbg)) return SQ_ERR_ALIGN;
+  return SQ_OK;
+}
+
+sq_status_t check_gemm_args(const void* Xq, const void* sx, const void* Wq, const void* sw, int64_t M, int64_t N,
+                            int64_t K, const void* Y, const void* acc) {
+  if (M < 0 || N < 0 || M > kMaxRows || N > kMaxRows) return SQ_ERR_INVALID_ARG;
+  if (K < 2 || (K & 1)) return SQ_ERR_SHAPE;
+  if (K > kMaxK) return SQ_ERR_UNSUPPORTED;
+  if (M == 0 || N == 0) return SQ_OK;
+  if (!Xq || !sx || !Wq || !sw || !Y) return SQ_ERR_INVALID_ARG;
+  if (!sq::aligned16(Xq) || !sq::aligned16(sx) || !sq::aligned16(Wq) || !sq::aligned16(sw) || !sq::aligned16(Y) ||
+      !sq::aligned16(acc))
+    return SQ_ERR_ALIGN;
+  return SQ_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+sq_status_t sq_factorize(int64_t n, int32_t* n1, int32_t* n2) {
+  if (!n1 || !n2 || n < 1 || n > (1ll << 40)) return SQ_ERR_INVALID_ARG;
+  const double root = std::sqrt(static_cast<double>(n));
+  int64_t best = 1;
+  for (int64_t a = 1; a <= n; a *= 2) {
+    if (n % a != 0) continue;
+    if (std::fabs(static_cast<double>(a) - root) < std::fabs(static_cast<double>(best) - root)) best = a;
+  }
+  if (n / best > INT32_MAX) return SQ_ERR_UNSUPPORTED;
+  *n1 = static_cast<int32_t>(n / best);
+  *n2 = static_cast<int32_t>(best);
+  return SQ_OK;
+}
+
+sq_status_t sq_build_rotation(const float* calib, int64_t T, int64_t n, int32_t n1, int32_t n2, uint32_t flags,
+                              uint64_t seed, const double* O_or_null, sq_rotation_t** out) {
+  if (!out) return SQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!calib || T < 1 || n1 < 1 || n2 < 1 || (flags & ~7u)) return SQ_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(n1) * n2 != n) return SQ_ERR_SHAPE;
+  if ((flags & SQ_ROT_HADAMARD) && (n2 & (n2 - 1)) != 0) return SQ_ERR_SHAPE;
+  if (n1 > 4096 || n2 > 4096) return SQ_ERR_UNSUPPORTED;
+  std::vector<float> R1, R2;
+  sq_status_t st = sq::build_factors_host(calib, T, n, n1, n2, flags, seed, O_or_null, R1, R2);
+  if (st != SQ_OK) return st;
+  return make_handle(std::move(R1), std::move(R2), n1, n2, out);
+}
+
+sq_status_t sq_rotation_from_factors(const float* R1, const float* R2, int32_t n1, int32_t n2,
+                                     sq_rotation_t** out) {
+  if (!out) return SQ_ERR_INVALID_ARG;
+  *out = nullptr;
+  if (!R1 || !R2 || n1 < 1 || n2 < 1) return SQ_ERR_INVALID_ARG;
+  if (n1 > 4096 || n2 > 4096) return SQ_ERR_UNSUPPORTED;
+  std::vector<float> a(R1, R1 + static_cast<size_t>(n1) * n1), b(R2, R2 + static_cast<size_t>(n2) * n2);
+  return make_handle(std::move(a), std::move(b), n1, n2, out);
+}
+
+sq_status_t sq_rotation_get_factors(const sq_rotation_t* rot, float* R1, float* R2) {
+  if (!rot || !R1 || !R2) return SQ_ERR_INVALID_ARG;
+  std::memcpy(R1, rot->R1.data(), sizeof(float) * rot->R1.size());
+  std::memcpy(R2, rot->R2.data(), sizeof(float) * rot->R2.size());
+  return SQ_OK;
+}
+
+sq_status_t sq_rotation_dims(const sq_rotation_t* rot, int32_t* n1, int32_t* n2) {
+  if (!rot || !n1 || !n2) return SQ_ERR_INVALID_ARG;
+  *n1 = rot->n1;
+  *n2 = rot->n2;
+  return SQ_OK;
+}
+
+void sq_rotation_destroy(sq_rotation_t* rot) {
+  if (!rot) return;
+  if (rot->dR1) cudaFree(rot->dR1);
+  if (rot->dR2) cudaFree(rot->dR2);
+  delete rot;
+}
+
+sq_status_t sq_rotate_quant_act(const sq_rotation_t* rot, const void* X, int64_t M, void* Xq, void* sx,
+                                void* Zdbg_or_null, void* stream) {
+  if (!rot) return SQ_ERR_INVALID_ARG;
+  const int64_t n = static_cast<int64_t>(rot->n1) * rot->n2;
+  if (rot->n2 & 1) return SQ_ERR_SHAPE;
+  sq_status_t st = check_rows_args(X, Xq, sx, Zdbg_or_null, M, n);
+  if (st != SQ_OK || M == 0) return st;
+  return sq::launch_rotate_quant(rot->dR1, rot->dR2, rot->n1, rot->n2, X, M, Xq, sx,
+                                 static_cast<float*>(Zdbg_or_null), static_cast<cudaStream_t>(stream));
+}
+
+sq_status_t sq_pack_weight(const sq_rotation_t* rot_or_null, const void* W, int64_t N, int64_t K, void* Wq,
+                           void* sw, void* stream) {
+  if (rot_or_null) {
+    if (static_cast<int64_t>(rot_or_null->n1) * rot_or_null->n2 != K) return SQ_ERR_SHAPE;
+    if (rot_or_null->n2 & 1) return SQ_ERR_SHAPE;
+  }
+  sq_status_t st = check_rows_args(W, Wq, sw, nullptr, N, K);
+  if (st != SQ_OK || N == 0) return st;
+  if (rot_or_null)
+    return sq::launch_rotate_quant(rot_or_null->dR1, rot_or_null->dR2, rot_or_null->n1, rot_or_null->n2, W, N, Wq,
+                                   sw, nullptr, static_cast<cudaStream_t>(stream));
+  return sq::launch_rotate_quant(nullptr, nullptr, 1, static_cast<int>(K), W, N, Wq, sw, nullptr,
+                                 static_cast<cudaStream_t>(stream));
+}
+
+size_t sq_w4a4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M <= 0 || N <= 0 || K <= 0) return 0;
+  return sq::gemm_workspace_bytes(M, N, K);
+}
+
+sq_status_t sq_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw, int64_t M, int64_t N,
+                         int64_t K, void* Y, void* accdbg_or_null, void* workspace, size_t workspace_bytes,
+                         void* stream) {
+  sq_status_t st = check_gemm_args(Xq, sx, Wq, sw, M, N, K, Y, accdbg_or_null);
+  if (st != SQ_OK || M == 0 || N == 0) return st;
+  if (workspace && !sq::aligned16(workspace)) return SQ_ERR_ALIGN;
+  return sq::launch_w4a4_gemm(Xq, sx, Wq, sw, M, N, K, Y, static_cast<int32_t*>(accdbg_or_null), workspace,
+                              workspace ? workspace_bytes : 0, static_cast<cudaStream_t>(stream));
+}
+
+// Workspace layout of sq_linear: [Xq: M*K/2][sx: 2*M][GEMM scratch], each 256-byte aligned.
+size_t sq_linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M <= 0 || N <= 0 || K <= 0) return 0;
+  return align_up(static_cast<size_t>(M) * (K / 2), 256) + align_up(static_cast<size_t>(M) * 2, 256) +
+         align_up(sq::gemm_workspace_bytes(M, N, K), 256);
+}
+
+sq_status_t sq_linear(const sq_rotation_t* rot, const void* X, int64_t M, const void* Wq, const void* sw,
+                      int64_t N, int64_t K, void* workspace, size_t workspace_bytes, void* Y, void* stream) {
+  if (!rot) return SQ_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(rot->n1) * rot->n2 != K) return SQ_ERR_SHAPE;
+  if (M < 0 || N < 0) return SQ_ERR_INVALID_ARG;
+  if (M == 0 || N == 0) return SQ_OK;
+  if (!workspace) return SQ_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQ_ERR_ALIGN;
+  if (workspace_bytes < sq_linear_workspace_bytes(M, N, K)) return SQ_ERR_NOMEM;
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  void* Xq = ws;
+  void* sx = ws + align_up(static_cast<size_t>(M) * (K / 2), 256);
+  void* gws = static_cast<unsigned char*>(sx) + align_up(static_cast<size_t>(M) * 2, 256);
+  const size_t gws_bytes = sq::gemm_workspace_bytes(M, N, K);
+  sq_status_t st = sq_rotate_quant_act(rot, X, M, Xq, sx, nullptr, stream);
+  if (st != SQ_OK) return st;
+  return sq_w4a4_gemm(Xq, sx, Wq, sw, M, N, K, Y, nullptr, gws_bytes ? gws : nullptr, gws_bytes, stream);
+}
+
+// Workspace layout of sq_linear_host: [X: 2*M*K][Y: 2*M*N][sq_linear workspace].
+size_t sq_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K) {
+  if (M <= 0 || N <= 0 || K <= 0) return 0;
+  return align_up(static_cast<size_t>(M) * K * 2, 256) + align_up(static_cast<size_t>(M) * N * 2, 256) +
+         sq_linear_workspace_bytes(M, N, K);
+}
+
+sq_status_t sq_linear_host(const sq_rotation_t* rot, const void* X_host, int64_t M, const void* Wq, const void* sw,
+                           int64_t N, int64_t K, void* workspace, size_t workspace_bytes, void* Y_host,
+                           void* stream) {
+  if (!rot || M < 0 || N < 0 || K < 2) return SQ_ERR_INVALID_ARG;
+  if (M == 0 || N == 0) return SQ_OK;
+  if (!X_host || !Y_host || !workspace) return SQ_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQ_ERR_ALIGN;
+  if (workspace_bytes < sq_linear_host_workspace_bytes(M, N, K)) return SQ_ERR_NOMEM;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  const size_t xb = static_cast<size_t>(M) * K * 2, yb = static_cast<size_t>(M) * N * 2;
+  void* dX = ws;
+  void* dY = ws + align_up(xb, 256);
+  void* lws = static_cast<unsigned char*>(dY) + align_up(yb, 256);
+  if (cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return SQ_ERR_CUDA;
+  sq_status_t st = sq_linear(rot, dX, M, Wq, sw, N, K, lws, sq_linear_workspace_bytes(M, N, K), dY, stream);
+  if (st != SQ_OK) return st;
+  if (cudaMemcpyAsync(Y_host, dY, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SQ_ERR_CUDA;
+  if (cudaStreamSynchronize(s) != cudaSuccess) return SQ_ERR_CUDA;
+  return SQ_OK;
+}
+
+sq_status_t sq_last_device_status(void* stream) {
+  return sq::read_and_clear_device_status(static_cast<cudaStream_t>(stream));
+}
+
+uint64_t sq_kernel_launch_count(void) { return sq::g_launches.load(std::memory_order_relaxed); }
+
+const char* sq_status_string(sq_status_t s) {
+  switch (s) {
+    case SQ_OK: return "ok";
+    case SQ_ERR_INVALID_ARG: return "invalid argument";
+    case SQ_ERR_SHAPE: return "shape mismatch";
+    case SQ_ERR_ALIGN: return "pointer not 16-byte aligned";
+    case SQ_ERR_UNSUPPORTED: return "size not supported";
+    case SQ_ERR_NOMEM: return "out of memory or workspace too small";
+    case SQ_ERR_CUDA: return "CUDA call failed";
+    case SQ_ERR_TIMEOUT: return "device-side wait timed out";
+  }
+  return "unknown status";
+}
+
+}  // extern "C"

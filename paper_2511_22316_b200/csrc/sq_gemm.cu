@@ -1,0 +1,314 @@
+// Step 3 of the hot path: INT4 x INT4 GEMM with int32 accumulation and the dequantisation
+// (token step x channel step -> fp16) fused into the epilogue:
+//   acc[t, c] = sum_k Xq[t, k] Wq[c, k],   Y[t, c] = fp16(acc * sx[t] * sw[c])
+// i.e. the "NT" product Flat(X~_R) Flat(W~_R)^T on the integer codes.
+//
+// Tensor-core kernel (sm_100a): packed nibbles arrive by TMA into a staging ring; four unpack
+// warps widen them to int8 in shared memory, written directly in the 128-byte-swizzled K-major
+// layout the UMMA descriptors expect; one thread issues tcgen05.mma kind::i8 into a TMEM int32
+// accumulator; the same four warps then read TMEM, dequantise and store fp16.
+//
+// Widening without arithmetic: a nibble moved to the top of a byte is the int8 value 16*code
+// (two's complement keeps the sign), so  lo = (w << 4) & 0xF0F0F0F0  and  hi = w & 0xF0F0F0F0
+// turn one packed word into eight int8 operands.  Both operands carry the factor 16, so the
+// accumulator holds 256 * acc; the epilogue shifts it out exactly.  Within a k-block the even
+// and odd channels land in different 16-byte chunks; A and B use the same permutation, which
+// leaves every dot product unchanged.
+#include <cuda.h>
+#include <cuda_fp16.h>
+
+#include <mutex>
+
+#include "sq_internal.h"
+#include "sq_ptx.cuh"
+
+namespace sq {
+
+namespace {
+
+constexpr int BM = 128;          // tokens per tile (UMMA M)
+constexpr int BK = 128;          // int4 channels per k-block: 64 packed bytes -> one 128-byte int8 row
+constexpr int PACKED_ROW = BK / 2;
+constexpr int UNPACK_WARPS = 4;
+constexpr int GEMM_THREADS = (2 + UNPACK_WARPS) * 32;
+
+enum WaitSite : uint32_t { SITE_STAGE_EMPTY = 1, SITE_STAGE_FULL, SITE_OP_EMPTY, SITE_OP_FULL, SITE_TMEM_FULL };
+
+template <int BN, int STAGES>
+struct GemmSmem {
+  static constexpr int A_OP = BM * 128;               // int8 operand tile
+  static constexpr int B_OP = BN * 128;
+  static constexpr int A_ST = BM * PACKED_ROW;        // packed staging tile
+  static constexpr int B_ST = BN * PACKED_ROW;
+  static constexpr int OFF_A_OP = 0;
+  static constexpr int OFF_B_OP = OFF_A_OP + STAGES * A_OP;
+  static constexpr int OFF_A_ST = OFF_B_OP + STAGES * B_OP;
+  static constexpr int OFF_B_ST = OFF_A_ST + STAGES * A_ST;
+  static constexpr int OFF_BAR = OFF_B_ST + STAGES * B_ST;
+  static constexpr int NUM_BARS = 4 * STAGES + 1;
+  static constexpr int OFF_TMEM = OFF_BAR + NUM_BARS * 8;
+  static constexpr int TOTAL = OFF_TMEM + 16;
+  static constexpr int DYN_BYTES = TOTAL + 1024;      // slack for the 1024-byte alignment
+};
+
+// Widens `rows` x 64 packed bytes (row stride 64) into `rows` x 128 int8 (128-byte swizzle).
+template <int ROWS>
+__device__ __forceinline__ void unpack_tile(const unsigned char* __restrict__ st, unsigned char* __restrict__ op,
+                                            int t) {
+  constexpr int ITEMS = ROWS * 4;                      // 16-byte packed chunks
+  const uint4* src = reinterpret_cast<const uint4*>(st);
+#pragma unroll 4
+  for (int idx = t; idx < ITEMS; idx += UNPACK_WARPS * 32) {
+    const uint4 w = src[idx];
+    const int r = idx >> 2, j = idx & 3;
+    uint4 lo, hi;
+    lo.x = (w.x << 4) & 0xF0F0F0F0u; hi.x = w.x & 0xF0F0F0F0u;
+    lo.y = (w.y << 4) & 0xF0F0F0F0u; hi.y = w.y & 0xF0F0F0F0u;
+    lo.z = (w.z << 4) & 0xF0F0F0F0u; hi.z = w.z & 0xF0F0F0F0u;
+    lo.w = (w.w << 4) & 0xF0F0F0F0u; hi.w = w.w & 0xF0F0F0F0u;
+    unsigned char* rowp = op + r * 128;
+    const int sw = r & 7;
+    *reinterpret_cast<uint4*>(rowp + (((2 * j) ^ sw) << 4)) = lo;
+    *reinterpret_cast<uint4*>(rowp + (((2 * j + 1) ^ sw) << 4)) = hi;
+  }
+}
+
+template <int BN, int STAGES>
+__global__ void __launch_bounds__(GEMM_THREADS, 1)
+w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                    const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
+                    __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
+  using L = GemmSmem<BN, STAGES>;
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+  uint64_t* stage_full = bars;
+  uint64_t* stage_empty = bars + STAGES;
+  uint64_t* op_full = bars + 2 * STAGES;
+  uint64_t* op_empty = bars + 3 * STAGES;
+  uint64_t* tmem_full = bars + 4 * STAGES;
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_TMEM);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM;
+  const int num_kb = K / BK;
+
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmap_x);
+    tma_prefetch_desc(&tmap_w);
+    for (int s = 0; s < STAGES; ++s) {
+      mbar_init(&stage_full[s], 1);
+      mbar_init(&stage_empty[s], UNPACK_WARPS);
+      mbar_init(&op_full[s], UNPACK_WARPS);
+      mbar_init(&op_empty[s], 1);
+    }
+    mbar_init(tmem_full, 1);
+    mbar_fence_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(tmem_slot, BN);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_d = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------------------
+    if (elect_one()) {
+      for (int kb = 0; kb < num_kb; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        if (!mbar_wait(&stage_empty[s], ph ^ 1, SITE_STAGE_EMPTY)) break;
+        mbar_arrive_expect_tx(&stage_full[s], L::A_ST + L::B_ST);
+        tma_load_2d(smem + L::OFF_A_ST + s * L::A_ST, &tmap_x, &stage_full[s], kb * PACKED_ROW, m0);
+        tma_load_2d(smem + L::OFF_B_ST + s * L::B_ST, &tmap_w, &stage_full[s], kb * PACKED_ROW, n0);
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer --------------------------------------------
+    if (elect_one()) {
+      constexpr uint32_t idesc = umma_idesc(/*c=s32*/ 2, /*a=s8*/ 1, /*b=s8*/ 1, BM, BN);
+      bool ok = true;
+      for (int kb = 0; kb < num_kb && ok; ++kb) {
+        const int s = kb % STAGES;
+        const uint32_t ph = (kb / STAGES) & 1;
+        ok = mbar_wait(&op_full[s], ph, SITE_OP_FULL);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t a_base = smem_u32(smem + L::OFF_A_OP + s * L::A_OP);
+        const uint32_t b_base = smem_u32(smem + L::OFF_B_OP + s * L::B_OP);
+#pragma unroll
+        for (int k = 0; k < 4; ++k) {                  // 4 x (K = 32 int8) per 128-byte row
+          umma_i8(tmem_d, umma_desc_sw128(a_base + k * 32), umma_desc_sw128(b_base + k * 32), idesc,
+                  (kb | k) != 0 ? 1u : 0u);
+        }
+        umma_commit(&op_empty[s]);                      // frees the operand stage when the MMAs retire
+      }
+      umma_commit(tmem_full);                           // accumulator complete (or abandoned)
+    }
+  } else {
+    // ------------------------------ unpack warps, then epilogue -----------------------------
+    const int t = threadIdx.x - 64;                    // 0 .. 127
+    bool ok = true;
+    for (int kb = 0; kb < num_kb; ++kb) {
+      const int s = kb % STAGES;
+      const uint32_t ph = (kb / STAGES) & 1;
+      ok = mbar_wait(&stage_full[s], ph, SITE_STAGE_FULL) && mbar_wait(&op_empty[s], ph ^ 1, SITE_OP_EMPTY);
+      if (!ok) break;
+      unpack_tile<BM>(smem + L::OFF_A_ST + s * L::A_ST, smem + L::OFF_A_OP + s * L::A_OP, t);
+      unpack_tile<BN>(smem + L::OFF_B_ST + s * L::B_ST, smem + L::OFF_B_OP + s * L::B_OP, t);
+      fence_proxy_async_smem();                         // generic-proxy stores -> visible to the MMA
+      __syncwarp();
+      if (lane == 0) {
+        mbar_arrive(&stage_empty[s]);
+        mbar_arrive(&op_full[s]);
+      }
+    }
+    if (ok) ok = mbar_wait(tmem_full, 0, SITE_TMEM_FULL);
+    tc_fence_after_sync();
+    if (ok) {
+      const int quarter = warp & 3;                     // TMEM lanes this warp may read
+      const int row = m0 + quarter * 32 + lane;
+      const float sxv = (row < M) ? __half2float(sx[row]) : 0.0f;
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(tmem_d + (static_cast<uint32_t>(quarter * 32) << 16) + c * 32, r);
+        tmem_wait_ld();
+        const int col0 = n0 + c * 32;
+        if (row < M && col0 < N) {
+          __half* yrow = Y + static_cast<size_t>(row) * N + col0;
+          int32_t* arow = accdbg ? accdbg + static_cast<size_t>(row) * N + col0 : nullptr;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {                 // groups of 8 columns (N % 8 == 0)
+            if (col0 + g * 8 < N) {
+              __align__(16) __half h[8];
+              int32_t a[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                a[e] = static_cast<int32_t>(r[g * 8 + e]) >> 8;          // exact: acc256 = 256 * acc
+                const float swv = __half2float(__ldg(sw + col0 + g * 8 + e));
+                h[e] = __float2half_rn(static_cast<float>(a[e]) * (sxv * swv));
+              }
+              *reinterpret_cast<uint4*>(yrow + g * 8) = *reinterpret_cast<const uint4*>(h);
+              if (arow) {
+                *reinterpret_cast<int4*>(arow + g * 8) = make_int4(a[0], a[1], a[2], a[3]);
+                *reinterpret_cast<int4*>(arow + g * 8 + 4) = make_int4(a[4], a[5], a[6], a[7]);
+              }
+            }
+          }
+        }
+      }
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_d, BN);
+  }
+}
+
+// Plain integer kernel for shapes the tensor-core path does not take (K % 128 != 0, N % 8 != 0):
+// one thread per output, byte-wise.  Same results, bit for bit.
+__global__ void w4a4_gemm_simple_kernel(const uint8_t* __restrict__ Xq, const __half* __restrict__ sx,
+                                        const uint8_t* __restrict__ Wq, const __half* __restrict__ sw,
+                                        int M, int N, int K, __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  const int t = blockIdx.y;
+  if (c >= N || t >= M) return;
+  const uint8_t* a = Xq + static_cast<size_t>(t) * (K / 2);
+  const uint8_t* b = Wq + static_cast<size_t>(c) * (K / 2);
+  int32_t acc = 0;
+  for (int j = 0; j < K / 2; ++j) {
+    const int av = a[j], bv = b[j];
+    const int a0 = (av << 28) >> 28, a1 = (av << 24) >> 28;      // sign-extended nibbles
+    const int b0 = (bv << 28) >> 28, b1 = (bv << 24) >> 28;
+    acc += a0 * b0 + a1 * b1;
+  }
+  const float s = __half2float(sx[t]) * __half2float(sw[c]);
+  Y[static_cast<size_t>(t) * N + c] = __float2half_rn(static_cast<float>(acc) * s);
+  if (accdbg) accdbg[static_cast<size_t>(t) * N + c] = acc;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Tensor maps (driver entry point fetched at run time, so the library has no link-time
+// dependency on libcuda and still loads on a machine without a driver).
+// ---------------------------------------------------------------------------------------------
+using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+EncodeTiledFn get_encode_fn() {
+  static EncodeTiledFn fn = nullptr;
+  static std::once_flag once;
+  std::call_once(once, [] {
+    void* p = nullptr;
+    cudaDriverEntryPointQueryResult q;
+    if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+        q == cudaDriverEntryPointSuccess)
+      fn = reinterpret_cast<EncodeTiledFn>(p);
+  });
+  return fn;
+}
+
+// 2-D uint8 map over a packed [rows x row_bytes] matrix; box = box_rows x 64 bytes, no swizzle,
+// out-of-range rows read as zero.
+bool make_packed_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_rows) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return false;
+  const cuuint64_t dims[2] = {row_bytes, rows};
+  const cuuint64_t strides[1] = {row_bytes};
+  const cuuint32_t box[2] = {static_cast<cuuint32_t>(PACKED_ROW), box_rows};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN, int STAGES>
+sq_status_t launch_tc(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N, int K, void* Y,
+                      int32_t* accdbg, cudaStream_t s) {
+  using L = GemmSmem<BN, STAGES>;
+  CUtensorMap mx, mw;
+  if (!make_packed_map(&mx, Xq, M, K / 2, BM) || !make_packed_map(&mw, Wq, N, K / 2, BN)) return SQ_ERR_CUDA;
+  auto kern = w4a4_gemm_tc_kernel<BN, STAGES>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
+      return SQ_ERR_CUDA;
+    attr_set = true;
+  }
+  dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
+  kern<<<grid, GEMM_THREADS, L::DYN_BYTES, s>>>(mx, mw, static_cast<const __half*>(sx),
+                                                static_cast<const __half*>(sw), M, N, K, static_cast<__half*>(Y),
+                                                accdbg);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+}
+
+}  // namespace
+
+size_t gemm_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
+
+sq_status_t launch_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw, int64_t M, int64_t N,
+                             int64_t K, void* Y, int32_t* accdbg, void*, size_t, cudaStream_t s) {
+  if (M == 0 || N == 0) return SQ_OK;
+  const bool tc_ok = (K % BK == 0) && (N % 8 == 0) && K >= BK;
+  if (tc_ok) {
+    if (N >= 256 && M > 64)
+      return launch_tc<256, 3>(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
+    return launch_tc<128, 4>(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
+  }
+  dim3 block(128), grid((unsigned)((N + 127) / 128), (unsigned)M);
+  w4a4_gemm_simple_kernel<<<grid, block, 0, s>>>(static_cast<const uint8_t*>(Xq), static_cast<const __half*>(sx),
+                                                 static_cast<const uint8_t*>(Wq), static_cast<const __half*>(sw),
+                                                 (int)M, (int)N, (int)K, static_cast<__half*>(Y), accdbg);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+}
+
+}  // namespace sq

@@ -1,0 +1,45 @@
+// Internal declarations shared by the translation units of libsinglequant.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <atomic>
+#include <vector>
+
+#include "../../include/singlequant.h"
+
+struct sq_rotation {
+  int32_t n1 = 0, n2 = 0;
+  int device = -1;
+  std::vector<float> R1;   // host fp32 [n1 x n1]
+  std::vector<float> R2;   // host fp32 [n2 x n2]
+  float* dR1 = nullptr;    // device fp32 [n1 x n1]
+  float* dR2 = nullptr;    // device fp32 [n2 x n2]
+};
+
+namespace sq {
+
+extern std::atomic<uint64_t> g_launches;
+inline void count_launch(uint64_t k = 1) { g_launches.fetch_add(k, std::memory_order_relaxed); }
+
+inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+// Host-side construction of the factors in float64 (sq_rotation_host.cu).
+sq_status_t build_factors_host(const float* calib, int64_t T, int64_t n, int32_t n1, int32_t n2,
+                               uint32_t flags, uint64_t seed, const double* O,
+                               std::vector<float>& R1, std::vector<float>& R2);
+
+// Steps 1+2 (sq_rotate_quant.cu).  R1/R2 device fp32 or both nullptr for the identity.
+sq_status_t launch_rotate_quant(const float* dR1, const float* dR2, int n1, int n2, const void* X,
+                                int64_t rows, void* Xq, void* scales, float* Zdbg, cudaStream_t s);
+
+// Step 3 (sq_gemm.cu).
+size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
+sq_status_t launch_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw,
+                             int64_t M, int64_t N, int64_t K, void* Y, int32_t* accdbg,
+                             void* workspace, size_t workspace_bytes, cudaStream_t s);
+
+// Device status word helpers (sq_api.cu).
+sq_status_t read_and_clear_device_status(cudaStream_t s);
+
+}  // namespace sq
