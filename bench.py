@@ -348,7 +348,7 @@ def run_ours(args, w):
         dominant, other = (roof_gemm, roof_rq) if gemm_ms >= rq_ms else (roof_rq, roof_gemm)
 
         cpu = None
-        if world == 1:
+        if world == 1 and not args.no_cpu_baseline:
             arm = OracleArm(w, rows=256, X=X, W=W)
             arm.one_pass()
             times, t_start = [], time.perf_counter()
@@ -392,6 +392,8 @@ def main():
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true",
+                    help="skip the timed CPU oracle leg (for profiler runs)")
     args = ap.parse_args()
     w = wl.by_name(args.workload)
     if args.impl == "reference":
