@@ -2,5 +2,6 @@
 // file-scope device symbols, so everything is compiled together (no relocatable device code).
 #include "sq_gemm.cu"
 #include "sq_rotate_quant.cu"
+#include "sq_rotate_quant_tc.cu"
 #include "sq_rotation_host.cu"
 #include "sq_api.cu"

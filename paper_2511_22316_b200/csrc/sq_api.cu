@@ -22,6 +22,17 @@ sq_status_t read_and_clear_device_status(cudaStream_t s) {
 }
 }  // namespace sq
 
+extern "C" void sq_rotation_destroy(sq_rotation_t* rot);
+
+namespace sq {
+sq_status_t rotate_quant_dispatch(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
+                                  float* Zdbg, cudaStream_t s) {
+  static const bool force_generic = getenv("SQ_ROTATE_GENERIC") != nullptr;
+  if (h->tc_ready && !force_generic) return launch_rotate_quant_tc(h, X, rows, Xq, scales, Zdbg, s);
+  return launch_rotate_quant(h->dR1, h->dR2, h->n1, h->n2, X, rows, Xq, scales, Zdbg, s);
+}
+}  // namespace sq
+
 namespace {
 
 constexpr int64_t kMaxN = 32768;       // rotate+quant: the row and its fp32 image stay in shared memory
@@ -50,6 +61,10 @@ sq_status_t make_handle(std::vector<float>&& R1, std::vector<float>&& R2, int32_
     if (h->dR1) cudaFree(h->dR1);
     if (h->dR2) cudaFree(h->dR2);
     delete h;
+    return SQ_ERR_CUDA;
+  }
+  if (sq::rotate_quant_tc_supported(n1, n2) && !sq::rotate_quant_tc_prepare(h)) {
+    sq_rotation_destroy(h);
     return SQ_ERR_CUDA;
   }
   *out = h;
@@ -140,6 +155,8 @@ void sq_rotation_destroy(sq_rotation_t* rot) {
   if (!rot) return;
   if (rot->dR1) cudaFree(rot->dR1);
   if (rot->dR2) cudaFree(rot->dR2);
+  if (rot->dA1img) cudaFree(rot->dA1img);
+  if (rot->dB2img) cudaFree(rot->dB2img);
   delete rot;
 }
 
@@ -150,8 +167,8 @@ sq_status_t sq_rotate_quant_act(const sq_rotation_t* rot, const void* X, int64_t
   if (rot->n2 & 1) return SQ_ERR_SHAPE;
   sq_status_t st = check_rows_args(X, Xq, sx, Zdbg_or_null, M, n);
   if (st != SQ_OK || M == 0) return st;
-  return sq::launch_rotate_quant(rot->dR1, rot->dR2, rot->n1, rot->n2, X, M, Xq, sx,
-                                 static_cast<float*>(Zdbg_or_null), static_cast<cudaStream_t>(stream));
+  return sq::rotate_quant_dispatch(rot, X, M, Xq, sx, static_cast<float*>(Zdbg_or_null),
+                                   static_cast<cudaStream_t>(stream));
 }
 
 sq_status_t sq_pack_weight(const sq_rotation_t* rot_or_null, const void* W, int64_t N, int64_t K, void* Wq,
@@ -163,8 +180,7 @@ sq_status_t sq_pack_weight(const sq_rotation_t* rot_or_null, const void* W, int6
   sq_status_t st = check_rows_args(W, Wq, sw, nullptr, N, K);
   if (st != SQ_OK || N == 0) return st;
   if (rot_or_null)
-    return sq::launch_rotate_quant(rot_or_null->dR1, rot_or_null->dR2, rot_or_null->n1, rot_or_null->n2, W, N, Wq,
-                                   sw, nullptr, static_cast<cudaStream_t>(stream));
+    return sq::rotate_quant_dispatch(rot_or_null, W, N, Wq, sw, nullptr, static_cast<cudaStream_t>(stream));
   return sq::launch_rotate_quant(nullptr, nullptr, 1, static_cast<int>(K), W, N, Wq, sw, nullptr,
                                  static_cast<cudaStream_t>(stream));
 }

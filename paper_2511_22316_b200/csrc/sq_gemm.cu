@@ -3,10 +3,11 @@
 //   acc[t, c] = sum_k Xq[t, k] Wq[c, k],   Y[t, c] = fp16(acc * sx[t] * sw[c])
 // i.e. the "NT" product Flat(X~_R) Flat(W~_R)^T on the integer codes.
 //
-// Tensor-core kernel (sm_100a): packed nibbles arrive by TMA into a staging ring; four unpack
+// Tensor-core kernel (sm_100a): packed nibbles arrive by TMA into a staging ring; eight unpack
 // warps widen them to int8 in shared memory, written directly in the 128-byte-swizzled K-major
 // layout the UMMA descriptors expect; one thread issues tcgen05.mma kind::i8 into a TMEM int32
-// accumulator; the same four warps then read TMEM, dequantise and store fp16.
+// accumulator; four epilogue warps read TMEM, dequantise and store fp16 while the next tile's main
+// loop runs into the other accumulator buffer.
 //
 // Widening without arithmetic: a nibble moved to the top of a byte is the int8 value 16*code
 // (two's complement keeps the sign), so  lo = (w << 4) & 0xF0F0F0F0  and  hi = w & 0xF0F0F0F0
@@ -29,168 +30,233 @@ namespace {
 constexpr int BM = 128;          // tokens per tile (UMMA M)
 constexpr int BK = 128;          // int4 channels per k-block: 64 packed bytes -> one 128-byte int8 row
 constexpr int PACKED_ROW = BK / 2;
-constexpr int UNPACK_WARPS = 4;
-constexpr int GEMM_THREADS = (2 + UNPACK_WARPS) * 32;
+constexpr int UNPACK_WARPS = 8;
+constexpr int EPI_WARPS = 4;
+constexpr int UNPACK_THREADS = UNPACK_WARPS * 32;
+constexpr int GEMM_THREADS = (2 + UNPACK_WARPS + EPI_WARPS) * 32;
 
-enum WaitSite : uint32_t { SITE_STAGE_EMPTY = 1, SITE_STAGE_FULL, SITE_OP_EMPTY, SITE_OP_FULL, SITE_TMEM_FULL };
+enum WaitSite : uint32_t {
+  SITE_STAGE_EMPTY = 1, SITE_STAGE_FULL, SITE_OP_EMPTY, SITE_OP_FULL, SITE_TMEM_FULL, SITE_TMEM_EMPTY
+};
 
-template <int BN, int STAGES>
+// Shared-memory plan.  The staging ring holds TMA blocks of 256 channels (128 packed bytes per
+// row, 128-byte swizzle); the operand ring holds int8 k-blocks of 128 channels (one 128-byte
+// swizzled row per matrix row), two per staging block.
+template <int BN, int S_OP, int S_ST>
 struct GemmSmem {
-  static constexpr int A_OP = BM * 128;               // int8 operand tile
+  static constexpr int A_OP = BM * 128;               // int8 operand tile (one k-block)
   static constexpr int B_OP = BN * 128;
-  static constexpr int A_ST = BM * PACKED_ROW;        // packed staging tile
-  static constexpr int B_ST = BN * PACKED_ROW;
+  static constexpr int A_ST = BM * 128;               // packed staging tile (two k-blocks)
+  static constexpr int B_ST = BN * 128;
   static constexpr int OFF_A_OP = 0;
-  static constexpr int OFF_B_OP = OFF_A_OP + STAGES * A_OP;
-  static constexpr int OFF_A_ST = OFF_B_OP + STAGES * B_OP;
-  static constexpr int OFF_B_ST = OFF_A_ST + STAGES * A_ST;
-  static constexpr int OFF_BAR = OFF_B_ST + STAGES * B_ST;
-  static constexpr int NUM_BARS = 4 * STAGES + 1;
+  static constexpr int OFF_B_OP = OFF_A_OP + S_OP * A_OP;
+  static constexpr int OFF_A_ST = OFF_B_OP + S_OP * B_OP;
+  static constexpr int OFF_B_ST = OFF_A_ST + S_ST * A_ST;
+  static constexpr int OFF_BAR = OFF_B_ST + S_ST * B_ST;
+  static constexpr int NUM_BARS = 2 * S_OP + 2 * S_ST + 4;
   static constexpr int OFF_TMEM = OFF_BAR + NUM_BARS * 8;
   static constexpr int TOTAL = OFF_TMEM + 16;
   static constexpr int DYN_BYTES = TOTAL + 1024;      // slack for the 1024-byte alignment
 };
 
-// Widens `rows` x 64 packed bytes (row stride 64) into `rows` x 128 int8 (128-byte swizzle).
+// Widens half h (64 packed bytes = 128 channels) of ROWS staged rows into ROWS x 128 int8.
+// Staging rows are 128 bytes with the 128-byte swizzle (16-byte chunk c of row r sits at chunk
+// c ^ (r & 7)); operand rows use the same swizzle.  Even channels of the k-block go to operand
+// chunks 0..3 and odd channels to chunks 4..7, for A and B alike.
+// Thread t works on chunk j = t & 3 of rows r0 + 64*i, r0 = 8*(t >> 5) + ((t >> 3) & 3) + 4*((t >> 2) & 1):
+// a quarter-warp covers rows {a, a+4} of one 8-row group, which makes its eight 16-byte loads
+// and each of its two rounds of eight 16-byte stores fall into eight different bank groups.
 template <int ROWS>
 __device__ __forceinline__ void unpack_tile(const unsigned char* __restrict__ st, unsigned char* __restrict__ op,
-                                            int t) {
-  constexpr int ITEMS = ROWS * 4;                      // 16-byte packed chunks
-  const uint4* src = reinterpret_cast<const uint4*>(st);
-#pragma unroll 4
-  for (int idx = t; idx < ITEMS; idx += UNPACK_WARPS * 32) {
-    const uint4 w = src[idx];
-    const int r = idx >> 2, j = idx & 3;
+                                            int t, int h) {
+  static_assert(ROWS % 64 == 0, "tile rows must be a multiple of 64");
+  constexpr int PER_THREAD = ROWS / 64;
+  const int j = t & 3;
+  const int r0 = ((t >> 5) << 3) + ((t >> 3) & 3) + (((t >> 2) & 1) << 2);
+  const int sw = r0 & 7;
+  const unsigned char* src = st + r0 * 128 + ((((h << 2) + j) ^ sw) << 4);
+  unsigned char* dst_lo = op + r0 * 128 + ((j ^ sw) << 4);
+  unsigned char* dst_hi = op + r0 * 128 + (((4 + j) ^ sw) << 4);
+  uint4 w[PER_THREAD];
+#pragma unroll
+  for (int i = 0; i < PER_THREAD; ++i) w[i] = *reinterpret_cast<const uint4*>(src + i * (64 * 128));
+#pragma unroll
+  for (int i = 0; i < PER_THREAD; ++i) {
     uint4 lo, hi;
-    lo.x = (w.x << 4) & 0xF0F0F0F0u; hi.x = w.x & 0xF0F0F0F0u;
-    lo.y = (w.y << 4) & 0xF0F0F0F0u; hi.y = w.y & 0xF0F0F0F0u;
-    lo.z = (w.z << 4) & 0xF0F0F0F0u; hi.z = w.z & 0xF0F0F0F0u;
-    lo.w = (w.w << 4) & 0xF0F0F0F0u; hi.w = w.w & 0xF0F0F0F0u;
-    unsigned char* rowp = op + r * 128;
-    const int sw = r & 7;
-    *reinterpret_cast<uint4*>(rowp + (((2 * j) ^ sw) << 4)) = lo;
-    *reinterpret_cast<uint4*>(rowp + (((2 * j + 1) ^ sw) << 4)) = hi;
+    lo.x = (w[i].x << 4) & 0xF0F0F0F0u; hi.x = w[i].x & 0xF0F0F0F0u;
+    lo.y = (w[i].y << 4) & 0xF0F0F0F0u; hi.y = w[i].y & 0xF0F0F0F0u;
+    lo.z = (w[i].z << 4) & 0xF0F0F0F0u; hi.z = w[i].z & 0xF0F0F0F0u;
+    lo.w = (w[i].w << 4) & 0xF0F0F0F0u; hi.w = w[i].w & 0xF0F0F0F0u;
+    *reinterpret_cast<uint4*>(dst_lo + i * (64 * 128)) = lo;
+    *reinterpret_cast<uint4*>(dst_hi + i * (64 * 128)) = hi;
   }
 }
 
-template <int BN, int STAGES>
+// Persistent kernel: CTA b works on tiles b, b + gridDim.x, ...; tile index = m_tile * tiles_n +
+// n_tile.  Warp 0 lane 0: TMA producer.  Warp 1 lane 0: MMA issuer.  Warps 2..9: unpack.
+// Warps 10..13: epilogue (TMEM -> dequant -> fp16 stores), overlapped with the next tile's main
+// loop through two TMEM accumulator buffers.
+template <int BN, int S_OP, int S_ST>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
-                    __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
-  using L = GemmSmem<BN, STAGES>;
+                    __half* __restrict__ Y, int32_t* __restrict__ accdbg, int probe) {
+  using L = GemmSmem<BN, S_OP, S_ST>;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
   uint64_t* stage_full = bars;
-  uint64_t* stage_empty = bars + STAGES;
-  uint64_t* op_full = bars + 2 * STAGES;
-  uint64_t* op_empty = bars + 3 * STAGES;
-  uint64_t* tmem_full = bars + 4 * STAGES;
+  uint64_t* stage_empty = bars + S_ST;
+  uint64_t* op_full = bars + 2 * S_ST;
+  uint64_t* op_empty = bars + 2 * S_ST + S_OP;
+  uint64_t* tmem_full = bars + 2 * S_ST + 2 * S_OP;        // [2]
+  uint64_t* tmem_empty = tmem_full + 2;                     // [2]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_TMEM);
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const int n0 = blockIdx.x * BN, m0 = blockIdx.y * BM;
-  const int num_kb = K / BK;
+  const int num_kb = K / BK;                  // int8 k-blocks of 128 channels
+  const int num_sb = (num_kb + 1) / 2;        // staging blocks of 256 channels (the last may be half used)
+  const int tiles_n = (N + BN - 1) / BN, tiles_m = (M + BM - 1) / BM;
+  const int num_tiles = tiles_n * tiles_m;
+  const uint32_t limit = wait_limit();
 
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmap_x);
     tma_prefetch_desc(&tmap_w);
-    for (int s = 0; s < STAGES; ++s) {
+    for (int s = 0; s < S_ST; ++s) {
       mbar_init(&stage_full[s], 1);
       mbar_init(&stage_empty[s], UNPACK_WARPS);
+    }
+    for (int s = 0; s < S_OP; ++s) {
       mbar_init(&op_full[s], UNPACK_WARPS);
       mbar_init(&op_empty[s], 1);
     }
-    mbar_init(tmem_full, 1);
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&tmem_full[b], 1);
+      mbar_init(&tmem_empty[b], EPI_WARPS);
+    }
     mbar_fence_init();
   }
   if (warp == 0) {
-    tmem_alloc(tmem_slot, BN);
+    tmem_alloc(tmem_slot, 2 * BN);
     tmem_relinquish();
   }
   tc_fence_before_sync();
   __syncthreads();
   tc_fence_after_sync();
-  const uint32_t tmem_d = *tmem_slot;
+  const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------------------
     if (elect_one()) {
-      for (int kb = 0; kb < num_kb; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        if (!mbar_wait(&stage_empty[s], ph ^ 1, SITE_STAGE_EMPTY)) break;
-        mbar_arrive_expect_tx(&stage_full[s], L::A_ST + L::B_ST);
-        tma_load_2d(smem + L::OFF_A_ST + s * L::A_ST, &tmap_x, &stage_full[s], kb * PACKED_ROW, m0);
-        tma_load_2d(smem + L::OFF_B_ST + s * L::B_ST, &tmap_w, &stage_full[s], kb * PACKED_ROW, n0);
+      uint32_t sit = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+        for (int sb = 0; sb < num_sb; ++sb, ++sit) {
+          const int s = sit % S_ST;
+          const uint32_t ph = (sit / S_ST) & 1;
+          ok = mbar_wait(&stage_empty[s], ph ^ 1, SITE_STAGE_EMPTY, limit);
+          if (!ok) break;
+          if (probe & 8) { mbar_arrive(&stage_full[s]); continue; }
+          mbar_arrive_expect_tx(&stage_full[s], L::A_ST + L::B_ST);
+          tma_load_2d(smem + L::OFF_A_ST + s * L::A_ST, &tmap_x, &stage_full[s], sb * 128, m0);
+          tma_load_2d(smem + L::OFF_B_ST + s * L::B_ST, &tmap_w, &stage_full[s], sb * 128, n0);
+        }
       }
     }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------------------
     if (elect_one()) {
       constexpr uint32_t idesc = umma_idesc(/*c=s32*/ 2, /*a=s8*/ 1, /*b=s8*/ 1, BM, BN);
+      uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int kb = 0; kb < num_kb && ok; ++kb) {
-        const int s = kb % STAGES;
-        const uint32_t ph = (kb / STAGES) & 1;
-        ok = mbar_wait(&op_full[s], ph, SITE_OP_FULL);
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+        const uint32_t b = tcount & 1;
+        ok = mbar_wait(&tmem_empty[b], ((tcount >> 1) & 1) ^ 1, SITE_TMEM_EMPTY, limit);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t a_base = smem_u32(smem + L::OFF_A_OP + s * L::A_OP);
-        const uint32_t b_base = smem_u32(smem + L::OFF_B_OP + s * L::B_OP);
+        const uint32_t tmem_d = tmem_base + b * BN;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int s = it % S_OP;
+          const uint32_t ph = (it / S_OP) & 1;
+          ok = mbar_wait(&op_full[s], ph, SITE_OP_FULL, limit);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t a_base = smem_u32(smem + L::OFF_A_OP + s * L::A_OP);
+          const uint32_t b_base = smem_u32(smem + L::OFF_B_OP + s * L::B_OP);
 #pragma unroll
-        for (int k = 0; k < 4; ++k) {                  // 4 x (K = 32 int8) per 128-byte row
-          umma_i8(tmem_d, umma_desc_sw128(a_base + k * 32), umma_desc_sw128(b_base + k * 32), idesc,
-                  (kb | k) != 0 ? 1u : 0u);
+          for (int k = 0; k < 4; ++k) {                // 4 x (K = 32 int8) per 128-byte row
+            if (!(probe & 2))
+            umma_i8(tmem_d, umma_desc_sw128(a_base + k * 32), umma_desc_sw128(b_base + k * 32), idesc,
+                    (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(&op_empty[s]);                    // frees the operand stage when the MMAs retire
         }
-        umma_commit(&op_empty[s]);                      // frees the operand stage when the MMAs retire
+        umma_commit(&tmem_full[b]);                     // accumulator complete (or abandoned)
       }
-      umma_commit(tmem_full);                           // accumulator complete (or abandoned)
+    }
+  } else if (warp < 2 + UNPACK_WARPS) {
+    // ------------------------------ unpack warps --------------------------------------------
+    const int t = threadIdx.x - 64;                    // 0 .. UNPACK_THREADS-1
+    uint32_t it = 0, sit = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int sb = 0; sb < num_sb && ok; ++sb, ++sit) {
+        const int ss = sit % S_ST;
+        ok = mbar_wait(&stage_full[ss], (sit / S_ST) & 1, SITE_STAGE_FULL, limit);
+        if (!ok) break;
+        for (int h = 0; h < 2 && 2 * sb + h < num_kb; ++h, ++it) {
+          const int s = it % S_OP;
+          ok = mbar_wait(&op_empty[s], ((it / S_OP) & 1) ^ 1, SITE_OP_EMPTY, limit);
+          if (!ok) break;
+          if (!(probe & 1)) {
+          unpack_tile<BM>(smem + L::OFF_A_ST + ss * L::A_ST, smem + L::OFF_A_OP + s * L::A_OP, t, h);
+          unpack_tile<BN>(smem + L::OFF_B_ST + ss * L::B_ST, smem + L::OFF_B_OP + s * L::B_OP, t, h);
+          }
+          fence_proxy_async_smem();                     // generic-proxy stores -> visible to the MMA
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&op_full[s]);
+        }
+        if (!ok) break;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&stage_empty[ss]);
+      }
     }
   } else {
-    // ------------------------------ unpack warps, then epilogue -----------------------------
-    const int t = threadIdx.x - 64;                    // 0 .. 127
+    // ------------------------------ epilogue warps ------------------------------------------
+    const int quarter = warp & 3;                       // TMEM lanes this warp may read
+    uint32_t tcount = 0;
     bool ok = true;
-    for (int kb = 0; kb < num_kb; ++kb) {
-      const int s = kb % STAGES;
-      const uint32_t ph = (kb / STAGES) & 1;
-      ok = mbar_wait(&stage_full[s], ph, SITE_STAGE_FULL) && mbar_wait(&op_empty[s], ph ^ 1, SITE_OP_EMPTY);
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+      const int m0 = (tile / tiles_n) * BM, n0 = (tile % tiles_n) * BN;
+      const uint32_t b = tcount & 1;
+      ok = mbar_wait(&tmem_full[b], (tcount >> 1) & 1, SITE_TMEM_FULL, limit);
       if (!ok) break;
-      unpack_tile<BM>(smem + L::OFF_A_ST + s * L::A_ST, smem + L::OFF_A_OP + s * L::A_OP, t);
-      unpack_tile<BN>(smem + L::OFF_B_ST + s * L::B_ST, smem + L::OFF_B_OP + s * L::B_OP, t);
-      fence_proxy_async_smem();                         // generic-proxy stores -> visible to the MMA
-      __syncwarp();
-      if (lane == 0) {
-        mbar_arrive(&stage_empty[s]);
-        mbar_arrive(&op_full[s]);
-      }
-    }
-    if (ok) ok = mbar_wait(tmem_full, 0, SITE_TMEM_FULL);
-    tc_fence_after_sync();
-    if (ok) {
-      const int quarter = warp & 3;                     // TMEM lanes this warp may read
+      tc_fence_after_sync();
       const int row = m0 + quarter * 32 + lane;
       const float sxv = (row < M) ? __half2float(sx[row]) : 0.0f;
+      const uint32_t tmem_d = tmem_base + b * BN + (static_cast<uint32_t>(quarter * 32) << 16);
 #pragma unroll 1
       for (int c = 0; c < BN / 32; ++c) {
         uint32_t r[32];
-        tmem_ld_32x32b_x32(tmem_d + (static_cast<uint32_t>(quarter * 32) << 16) + c * 32, r);
+        tmem_ld_32x32b_x32(tmem_d + c * 32, r);
         tmem_wait_ld();
         const int col0 = n0 + c * 32;
-        if (row < M && col0 < N) {
+        if (row < M && col0 < N && !(probe & 4)) {
           __half* yrow = Y + static_cast<size_t>(row) * N + col0;
           int32_t* arow = accdbg ? accdbg + static_cast<size_t>(row) * N + col0 : nullptr;
 #pragma unroll
           for (int g = 0; g < 4; ++g) {                 // groups of 8 columns (N % 8 == 0)
             if (col0 + g * 8 < N) {
+              const uint4 swraw = __ldg(reinterpret_cast<const uint4*>(sw + col0 + g * 8));
+              const __half* swh = reinterpret_cast<const __half*>(&swraw);
               __align__(16) __half h[8];
               int32_t a[8];
 #pragma unroll
               for (int e = 0; e < 8; ++e) {
-                a[e] = static_cast<int32_t>(r[g * 8 + e]) >> 8;          // exact: acc256 = 256 * acc
-                const float swv = __half2float(__ldg(sw + col0 + g * 8 + e));
-                h[e] = __float2half_rn(static_cast<float>(a[e]) * (sxv * swv));
+                a[e] = static_cast<int32_t>(r[g * 8 + e]) >> 8;          // exact: the accumulator is 256 * acc
+                h[e] = __float2half_rn(static_cast<float>(a[e]) * (sxv * __half2float(swh[e])));
               }
               *reinterpret_cast<uint4*>(yrow + g * 8) = *reinterpret_cast<const uint4*>(h);
               if (arow) {
@@ -201,6 +267,9 @@ w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           }
         }
       }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tmem_empty[b]);       // this warp's quarter of the buffer is drained
     }
   }
 
@@ -208,7 +277,7 @@ w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
   __syncthreads();
   if (warp == 0) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_d, BN);
+    tmem_dealloc(tmem_base, 2 * BN);
   }
 }
 
@@ -255,37 +324,42 @@ EncodeTiledFn get_encode_fn() {
   return fn;
 }
 
-// 2-D uint8 map over a packed [rows x row_bytes] matrix; box = box_rows x 64 bytes, no swizzle,
-// out-of-range rows read as zero.
+// 2-D uint8 map over a packed [rows x row_bytes] matrix; box = box_rows x 128 bytes with the
+// 128-byte swizzle; out-of-range rows and bytes read as zero.
 bool make_packed_map(CUtensorMap* map, const void* base, uint64_t rows, uint64_t row_bytes, uint32_t box_rows) {
   EncodeTiledFn enc = get_encode_fn();
   if (!enc) return false;
   const cuuint64_t dims[2] = {row_bytes, rows};
   const cuuint64_t strides[1] = {row_bytes};
-  const cuuint32_t box[2] = {static_cast<cuuint32_t>(PACKED_ROW), box_rows};
+  const cuuint32_t box[2] = {128, box_rows};
   const cuuint32_t estr[2] = {1, 1};
   return enc(map, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(base), dims, strides, box, estr,
-             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_NONE, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+             CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int BN, int STAGES>
+template <int BN, int S_OP, int S_ST>
 sq_status_t launch_tc(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N, int K, void* Y,
                       int32_t* accdbg, cudaStream_t s) {
-  using L = GemmSmem<BN, STAGES>;
+  using L = GemmSmem<BN, S_OP, S_ST>;
   CUtensorMap mx, mw;
   if (!make_packed_map(&mx, Xq, M, K / 2, BM) || !make_packed_map(&mw, Wq, N, K / 2, BN)) return SQ_ERR_CUDA;
-  auto kern = w4a4_gemm_tc_kernel<BN, STAGES>;
+  auto kern = w4a4_gemm_tc_kernel<BN, S_OP, S_ST>;
   static bool attr_set = false;
   if (!attr_set) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
       return SQ_ERR_CUDA;
     attr_set = true;
   }
-  dim3 grid((N + BN - 1) / BN, (M + BM - 1) / BM);
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return SQ_ERR_CUDA;
+  const int tiles = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
+  const int grid = tiles < sms ? tiles : sms;
   kern<<<grid, GEMM_THREADS, L::DYN_BYTES, s>>>(mx, mw, static_cast<const __half*>(sx),
                                                 static_cast<const __half*>(sw), M, N, K, static_cast<__half*>(Y),
-                                                accdbg);
+                                                accdbg, getenv("SQ_GEMM_PROBE") ? atoi(getenv("SQ_GEMM_PROBE")) : 0);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
 }
@@ -300,8 +374,8 @@ sq_status_t launch_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, con
   const bool tc_ok = (K % BK == 0) && (N % 8 == 0) && K >= BK;
   if (tc_ok) {
     if (N >= 256 && M > 64)
-      return launch_tc<256, 3>(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
-    return launch_tc<128, 4>(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
+      return launch_tc<256, 2, 2>(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
+    return launch_tc<128, 3, 3>(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
   }
   dim3 block(128), grid((unsigned)((N + 127) / 128), (unsigned)M);
   w4a4_gemm_simple_kernel<<<grid, block, 0, s>>>(static_cast<const uint8_t*>(Xq), static_cast<const __half*>(sx),

@@ -15,6 +15,10 @@ struct sq_rotation {
   std::vector<float> R2;   // host fp32 [n2 x n2]
   float* dR1 = nullptr;    // device fp32 [n1 x n1]
   float* dR2 = nullptr;    // device fp32 [n2 x n2]
+  // tensor-core rotate+quant: shared-memory images of the split factors (device), if supported
+  void* dA1img = nullptr;
+  void* dB2img = nullptr;
+  bool tc_ready = false;
 };
 
 namespace sq {
@@ -32,6 +36,15 @@ sq_status_t build_factors_host(const float* calib, int64_t T, int64_t n, int32_t
 // Steps 1+2 (sq_rotate_quant.cu).  R1/R2 device fp32 or both nullptr for the identity.
 sq_status_t launch_rotate_quant(const float* dR1, const float* dR2, int n1, int n2, const void* X,
                                 int64_t rows, void* Xq, void* scales, float* Zdbg, cudaStream_t s);
+
+// Tensor-core variant of steps 1+2 (sq_rotate_quant_tc.cu).
+bool rotate_quant_tc_supported(int n1, int n2);
+bool rotate_quant_tc_prepare(sq_rotation* h);
+sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
+                                   float* Zdbg, cudaStream_t s);
+// Picks the tensor-core kernel when the handle has its images, else the generic fp32 kernel.
+sq_status_t rotate_quant_dispatch(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
+                                  float* Zdbg, cudaStream_t s);
 
 // Step 3 (sq_gemm.cu).
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
