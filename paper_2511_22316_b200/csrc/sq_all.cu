@@ -1,6 +1,7 @@
 // Single translation unit of libsinglequant: the device status word and the kernels share
 // file-scope device symbols, so everything is compiled together (no relocatable device code).
 #include "sq_gemm.cu"
+#include "sq_gemm_pair.cu"
 #include "sq_rotate_quant.cu"
 #include "sq_rotate_quant_tc.cu"
 #include "sq_rotation_host.cu"

@@ -100,7 +100,7 @@ template <int BN, int S_OP, int S_ST>
 __global__ void __launch_bounds__(GEMM_THREADS, 1)
 w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
                     const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
-                    __half* __restrict__ Y, int32_t* __restrict__ accdbg, int probe) {
+                    __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
   using L = GemmSmem<BN, S_OP, S_ST>;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
@@ -158,7 +158,6 @@ w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           const uint32_t ph = (sit / S_ST) & 1;
           ok = mbar_wait(&stage_empty[s], ph ^ 1, SITE_STAGE_EMPTY, limit);
           if (!ok) break;
-          if (probe & 8) { mbar_arrive(&stage_full[s]); continue; }
           mbar_arrive_expect_tx(&stage_full[s], L::A_ST + L::B_ST);
           tma_load_2d(smem + L::OFF_A_ST + s * L::A_ST, &tmap_x, &stage_full[s], sb * 128, m0);
           tma_load_2d(smem + L::OFF_B_ST + s * L::B_ST, &tmap_w, &stage_full[s], sb * 128, n0);
@@ -187,7 +186,6 @@ w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           const uint32_t b_base = smem_u32(smem + L::OFF_B_OP + s * L::B_OP);
 #pragma unroll
           for (int k = 0; k < 4; ++k) {                // 4 x (K = 32 int8) per 128-byte row
-            if (!(probe & 2))
             umma_i8(tmem_d, umma_desc_sw128(a_base + k * 32), umma_desc_sw128(b_base + k * 32), idesc,
                     (kb | k) != 0 ? 1u : 0u);
           }
@@ -210,10 +208,8 @@ w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           const int s = it % S_OP;
           ok = mbar_wait(&op_empty[s], ((it / S_OP) & 1) ^ 1, SITE_OP_EMPTY, limit);
           if (!ok) break;
-          if (!(probe & 1)) {
           unpack_tile<BM>(smem + L::OFF_A_ST + ss * L::A_ST, smem + L::OFF_A_OP + s * L::A_OP, t, h);
           unpack_tile<BN>(smem + L::OFF_B_ST + ss * L::B_ST, smem + L::OFF_B_OP + s * L::B_OP, t, h);
-          }
           fence_proxy_async_smem();                     // generic-proxy stores -> visible to the MMA
           __syncwarp();
           if (lane == 0) mbar_arrive(&op_full[s]);
@@ -243,7 +239,7 @@ w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
         tmem_ld_32x32b_x32(tmem_d + c * 32, r);
         tmem_wait_ld();
         const int col0 = n0 + c * 32;
-        if (row < M && col0 < N && !(probe & 4)) {
+        if (row < M && col0 < N) {
           __half* yrow = Y + static_cast<size_t>(row) * N + col0;
           int32_t* arow = accdbg ? accdbg + static_cast<size_t>(row) * N + col0 : nullptr;
 #pragma unroll
@@ -359,7 +355,7 @@ sq_status_t launch_tc(const void* Xq, const void* sx, const void* Wq, const void
   const int grid = tiles < sms ? tiles : sms;
   kern<<<grid, GEMM_THREADS, L::DYN_BYTES, s>>>(mx, mw, static_cast<const __half*>(sx),
                                                 static_cast<const __half*>(sw), M, N, K, static_cast<__half*>(Y),
-                                                accdbg, getenv("SQ_GEMM_PROBE") ? atoi(getenv("SQ_GEMM_PROBE")) : 0);
+                                                accdbg);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
 }
@@ -372,6 +368,8 @@ sq_status_t launch_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, con
                              int64_t K, void* Y, int32_t* accdbg, void*, size_t, cudaStream_t s) {
   if (M == 0 || N == 0) return SQ_OK;
   const bool tc_ok = (K % BK == 0) && (N % 8 == 0) && K >= BK;
+  if (gemm_pair_supported(M, N, K))
+    return launch_w4a4_gemm_pair(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
   if (tc_ok) {
     if (N >= 256 && M > 64)
       return launch_tc<256, 2, 2>(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);

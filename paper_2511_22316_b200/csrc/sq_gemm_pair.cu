@@ -1,0 +1,315 @@
+// Step 3 for prefill-sized problems: the INT4 x INT4 GEMM on CTA pairs (tcgen05 cta_group::2).
+//
+// Two CTAs of a cluster share one 256 x 256 output tile: CTA r owns token rows [128 r, 128 r + 128)
+// of the tile (its TMEM lanes) and stages weight rows [128 r, 128 r + 128) of the tile (its half
+// of the B operand), so every widened weight byte is written to shared memory once per pair and
+// feeds both SMs' tensor cores.  The activation codes never pass through shared memory as int8:
+// four warps read the packed bytes of "their" token row, widen them in registers and store the
+// int8 operand straight into tensor memory (tcgen05.st), from where the MMA takes its A operand.
+//
+// Pipeline per CTA (block = 256 channels = 128 packed bytes per row = two k-blocks of 128):
+//   warp 0        TMA: packed A rows and packed B rows, one block per staging stage
+//   warps 2..5    A: staging -> registers -> widen -> TMEM ring stage        } arrive on the
+//   warps 6..13   B: staging -> registers -> widen -> swizzled operand ring  } leader's full[s]
+//   warp 1        (leader CTA only) 8 MMAs of K = 32 per block; commit frees the ring stage in
+//                 both CTAs; the last commit of a tile publishes the accumulator to both CTAs
+//   warps 14..17  epilogue: TMEM -> dequantise -> fp16 stores, then hand the accumulator back
+// Every hand-over costs each warp a few hundred cycles of barrier and fence latency whatever the
+// amount of data, which is why a ring stage holds two k-blocks.
+// The widening and the operand byte order are those of the single-CTA kernel (sq_gemm.cu).
+#include <cuda.h>
+#include <cuda_fp16.h>
+
+#include "sq_internal.h"
+#include "sq_ptx.cuh"
+
+namespace sq {
+namespace {
+
+constexpr int P_A_WARPS = 4;
+constexpr int P_B_WARPS = 8;
+constexpr int P_EPI_WARPS = 4;
+constexpr int P_THREADS = (2 + P_A_WARPS + P_B_WARPS + P_EPI_WARPS) * 32;
+constexpr int P_TILE_M = 256;            // tokens per pair tile (128 per CTA)
+constexpr int P_TILE_N = 256;            // output channels per pair tile (128 staged per CTA)
+constexpr int P_A_COL0 = 256;            // first TMEM column of the A operand ring (0..255: accumulator)
+constexpr int P_A_COLS_PER_STAGE = 64;   // 256 int8 per lane = 64 columns
+
+enum PairSite : uint32_t {
+  PSITE_ST_EMPTY = 32, PSITE_ST_FULL_A, PSITE_ST_FULL_B, PSITE_EMPTY_A, PSITE_EMPTY_B, PSITE_FULL,
+  PSITE_TMEM_FULL, PSITE_TMEM_EMPTY
+};
+
+template <int S_OP, int S_ST>
+struct PairSmem {
+  static_assert(S_OP >= 2 && S_OP <= 4, "the A ring has room for at most 4 blocks in TMEM");
+  static constexpr int B_OP = 2 * 128 * 128;         // int8 B half, two k-blocks
+  static constexpr int A_ST = 128 * 128;             // packed A rows, two k-blocks
+  static constexpr int B_ST = 128 * 128;             // packed B rows, two k-blocks
+  static constexpr int OFF_B_OP = 0;
+  static constexpr int OFF_A_ST = OFF_B_OP + S_OP * B_OP;
+  static constexpr int OFF_B_ST = OFF_A_ST + S_ST * A_ST;
+  static constexpr int OFF_BAR = OFF_B_ST + S_ST * B_ST;
+  static constexpr int NUM_BARS = 2 * S_OP + 2 * S_ST + 2;
+  static constexpr int OFF_TMEM = OFF_BAR + NUM_BARS * 8;
+  static constexpr int TOTAL = OFF_TMEM + 16;
+  static constexpr int DYN_BYTES = TOTAL + 1024;
+};
+
+template <int S_OP, int S_ST>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1)
+w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                      const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
+                      __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
+  using L = PairSmem<S_OP, S_ST>;
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+  uint64_t* st_full = bars;                           // [S_ST]  TMA landed (local)
+  uint64_t* st_empty = bars + S_ST;                   // [S_ST]  12 converter warps done (local)
+  uint64_t* full = bars + 2 * S_ST;                   // [S_OP]  24 converter warps of the pair (leader's copy is used)
+  uint64_t* empty = bars + 2 * S_ST + S_OP;           // [S_OP]  MMAs retired (each CTA's own copy)
+  uint64_t* tmem_full = bars + 2 * S_ST + 2 * S_OP;   // accumulator complete (each CTA's own copy)
+  uint64_t* tmem_empty = tmem_full + 1;               // epilogue warps of the pair (leader's copy is used)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_TMEM);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();            // 0 = leader (issues the MMAs)
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  const int num_kb = K / 128;
+  const int num_sb = (num_kb + 1) / 2;
+  const int tiles_n = (N + P_TILE_N - 1) / P_TILE_N, tiles_m = (M + P_TILE_M - 1) / P_TILE_M;
+  const int num_tiles = tiles_n * tiles_m;
+  const uint32_t limit = wait_limit();
+
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmap_x);
+    tma_prefetch_desc(&tmap_w);
+    for (int s = 0; s < S_ST; ++s) {
+      mbar_init(&st_full[s], 1);
+      mbar_init(&st_empty[s], P_A_WARPS + P_B_WARPS);
+    }
+    for (int s = 0; s < S_OP; ++s) {
+      mbar_init(&full[s], 2 * (P_A_WARPS + P_B_WARPS));
+      mbar_init(&empty[s], 1);
+    }
+    mbar_init(tmem_full, 1);
+    mbar_init(tmem_empty, 2 * P_EPI_WARPS);
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_slot, 512);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();                                 // both CTAs' barriers exist before any remote arrival
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------------------------
+    if (elect_one()) {
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+        const int m0 = (tile / tiles_n) * P_TILE_M + static_cast<int>(rank) * 128;
+        const int n0 = (tile % tiles_n) * P_TILE_N + static_cast<int>(rank) * 128;
+        for (int sb = 0; sb < num_sb; ++sb, ++it) {
+          const int ss = it % S_ST;
+          ok = mbar_wait(&st_empty[ss], ((it / S_ST) & 1) ^ 1, PSITE_ST_EMPTY, limit);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&st_full[ss], L::A_ST + L::B_ST);
+          tma_load_2d(smem + L::OFF_A_ST + ss * L::A_ST, &tmap_x, &st_full[ss], sb * 128, m0);
+          tma_load_2d(smem + L::OFF_B_ST + ss * L::B_ST, &tmap_w, &st_full[ss], sb * 128, n0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer (leader CTA) -------------------------------------
+    if (rank == 0 && elect_one()) {
+      constexpr uint32_t idesc = umma_idesc(/*c=s32*/ 2, /*a=s8*/ 1, /*b=s8*/ 1, P_TILE_M, P_TILE_N);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += npairs, ++tcount) {
+        ok = mbar_wait(tmem_empty, (tcount & 1) ^ 1, PSITE_TMEM_EMPTY, limit);
+        if (!ok) break;
+        tc_fence_after_sync();
+        for (int sb = 0; sb < num_sb; ++sb, ++it) {
+          const int s = it % S_OP;
+          ok = mbar_wait(&full[s], (it / S_OP) & 1, PSITE_FULL, limit);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t a_tmem = tmem_base + P_A_COL0 + s * P_A_COLS_PER_STAGE;
+          const uint32_t b_base = smem_u32(smem + L::OFF_B_OP + s * L::B_OP);
+          const int nk = (2 * sb + 1 < num_kb) ? 8 : 4;  // K = 32 int8 each: 8 TMEM columns / 32 smem bytes
+#pragma unroll 4
+          for (int k = 0; k < nk; ++k)
+            umma_i8_ts_pair(tmem_base, a_tmem + k * 8,
+                            umma_desc_sw128(b_base + (k >> 2) * (128 * 128) + (k & 3) * 32), idesc,
+                            (sb | k) != 0 ? 1u : 0u);
+          umma_commit_pair_mc(&empty[s], 3);            // frees ring stage s in both CTAs
+        }
+        umma_commit_pair_mc(tmem_full, 3);              // accumulator complete (or abandoned)
+      }
+    }
+  } else if (warp < 2 + P_A_WARPS) {
+    // ------------------------------ A converters: staging -> registers -> TMEM ------------------
+    const int q = warp & 3;                             // TMEM lane quarter this warp may touch
+    const int r = q * 32 + lane;                        // row of the CTA's 128 tokens = TMEM lane
+    const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+      for (int sb = 0; sb < num_sb && ok; ++sb, ++it) {
+        const int ss = it % S_ST, s = it % S_OP;
+        ok = mbar_wait(&st_full[ss], (it / S_ST) & 1, PSITE_ST_FULL_A, limit);
+        if (!ok) break;
+        const unsigned char* row = smem + L::OFF_A_ST + ss * L::A_ST + r * 128;
+        const int nh = (2 * sb + 1 < num_kb) ? 2 : 1;
+        uint4 w[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) w[c] = *reinterpret_cast<const uint4*>(row + ((c ^ (r & 7)) << 4));
+        ok = mbar_wait(&empty[s], ((it / S_OP) & 1) ^ 1, PSITE_EMPTY_A, limit);
+        if (!ok) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int h = 0; h < 2; ++h) {
+          if (h < nh) {
+            uint32_t v[32];
+#pragma unroll
+            for (int j = 0; j < 4; ++j) {
+              const uint4 x = w[4 * h + j];
+              v[4 * j + 0] = (x.x << 4) & 0xF0F0F0F0u; v[16 + 4 * j + 0] = x.x & 0xF0F0F0F0u;
+              v[4 * j + 1] = (x.y << 4) & 0xF0F0F0F0u; v[16 + 4 * j + 1] = x.y & 0xF0F0F0F0u;
+              v[4 * j + 2] = (x.z << 4) & 0xF0F0F0F0u; v[16 + 4 * j + 2] = x.z & 0xF0F0F0F0u;
+              v[4 * j + 3] = (x.w << 4) & 0xF0F0F0F0u; v[16 + 4 * j + 3] = x.w & 0xF0F0F0F0u;
+            }
+            tmem_st_32x32b_x32(tmem_base + lane_addr + P_A_COL0 + s * P_A_COLS_PER_STAGE + h * 32, v);
+          }
+        }
+        tmem_wait_st();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive_cluster(&full[s], 0);
+          mbar_arrive(&st_empty[ss]);
+        }
+      }
+    }
+  } else if (warp < 2 + P_A_WARPS + P_B_WARPS) {
+    // ------------------------------ B unpackers: staging -> registers -> operand ring -----------
+    const int t = threadIdx.x - (2 + P_A_WARPS) * 32;   // 0 .. 255
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+      for (int sb = 0; sb < num_sb && ok; ++sb, ++it) {
+        const int ss = it % S_ST, s = it % S_OP;
+        ok = mbar_wait(&st_full[ss], (it / S_ST) & 1, PSITE_ST_FULL_B, limit) &&
+             mbar_wait(&empty[s], ((it / S_OP) & 1) ^ 1, PSITE_EMPTY_B, limit);
+        if (!ok) break;
+        const unsigned char* st = smem + L::OFF_B_ST + ss * L::B_ST;
+        unsigned char* op = smem + L::OFF_B_OP + s * L::B_OP;
+        unpack_tile<128>(st, op, t, 0);
+        if (2 * sb + 1 < num_kb) unpack_tile<128>(st, op + 128 * 128, t, 1);
+        fence_proxy_async_smem();                       // generic-proxy stores -> visible to the MMA
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive_cluster(&full[s], 0);
+          mbar_arrive(&st_empty[ss]);
+        }
+      }
+    }
+  } else {
+    // ------------------------------ epilogue ----------------------------------------------------
+    const int q = warp & 3;
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = pair; tile < num_tiles && ok; tile += npairs, ++tcount) {
+      const int m0 = (tile / tiles_n) * P_TILE_M + static_cast<int>(rank) * 128;
+      const int n0 = (tile % tiles_n) * P_TILE_N;
+      ok = mbar_wait(tmem_full, tcount & 1, PSITE_TMEM_FULL, limit);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const int row = m0 + q * 32 + lane;
+      const float sxv = (row < M) ? __half2float(sx[row]) : 0.0f;
+      const uint32_t tmem_d = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < P_TILE_N / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(tmem_d + c * 32, r);
+        tmem_wait_ld();
+        const int col0 = n0 + c * 32;
+        if (row < M && col0 < N) {
+          __half* yrow = Y + static_cast<size_t>(row) * N + col0;
+          int32_t* arow = accdbg ? accdbg + static_cast<size_t>(row) * N + col0 : nullptr;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {                 // groups of 8 columns (N % 8 == 0)
+            if (col0 + g * 8 < N) {
+              const uint4 swraw = __ldg(reinterpret_cast<const uint4*>(sw + col0 + g * 8));
+              const __half* swh = reinterpret_cast<const __half*>(&swraw);
+              __align__(16) __half h[8];
+              int32_t a[8];
+#pragma unroll
+              for (int e = 0; e < 8; ++e) {
+                a[e] = static_cast<int32_t>(r[g * 8 + e]) >> 8;          // exact: the accumulator is 256 * acc
+                h[e] = __float2half_rn(static_cast<float>(a[e]) * (sxv * __half2float(swh[e])));
+              }
+              *reinterpret_cast<uint4*>(yrow + g * 8) = *reinterpret_cast<const uint4*>(h);
+              if (arow) {
+                *reinterpret_cast<int4*>(arow + g * 8) = make_int4(a[0], a[1], a[2], a[3]);
+                *reinterpret_cast<int4*>(arow + g * 8 + 4) = make_int4(a[4], a[5], a[6], a[7]);
+              }
+            }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(tmem_empty, 0);
+    }
+  }
+
+  // Neither CTA may leave while its partner can still reach its shared memory, barriers or TMEM.
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, 512);
+  }
+}
+
+}  // namespace
+
+bool gemm_pair_supported(int64_t M, int64_t N, int64_t K) {
+  return M > 128 && N >= 128 && (K % 128 == 0) && K >= 128 && (N % 8 == 0);
+}
+
+sq_status_t launch_w4a4_gemm_pair(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N,
+                                  int K, void* Y, int32_t* accdbg, cudaStream_t s) {
+  constexpr int S_OP = 3, S_ST = 3;
+  using L = PairSmem<S_OP, S_ST>;
+  CUtensorMap mx, mw;
+  if (!make_packed_map(&mx, Xq, M, K / 2, 128) || !make_packed_map(&mw, Wq, N, K / 2, 128)) return SQ_ERR_CUDA;
+  auto kern = w4a4_gemm_pair_kernel<S_OP, S_ST>;
+  static bool attr_set = false;
+  if (!attr_set) {
+    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
+      return SQ_ERR_CUDA;
+    attr_set = true;
+  }
+  int dev = 0, sms = 148;
+  if (cudaGetDevice(&dev) != cudaSuccess ||
+      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
+    return SQ_ERR_CUDA;
+  const int tiles = ((N + P_TILE_N - 1) / P_TILE_N) * ((M + P_TILE_M - 1) / P_TILE_M);
+  const int pairs = tiles < sms / 2 ? tiles : sms / 2;
+  kern<<<2 * pairs, P_THREADS, L::DYN_BYTES, s>>>(mx, mw, static_cast<const __half*>(sx),
+                                                  static_cast<const __half*>(sw), M, N, K,
+                                                  static_cast<__half*>(Y), accdbg);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+}
+
+}  // namespace sq

@@ -235,6 +235,10 @@ GEMM_SHAPES = [
     # tensor-core kernel: single tile, ragged M and N, several k-blocks (more than the ring depth)
     (1, 8, 128), (4, 128, 128), (16, 136, 256), (64, 512, 512), (128, 256, 1152), (130, 264, 640),
     (300, 1000, 384), (257, 72, 2048), (64, 4096, 1024),
+    # CTA-pair kernel (M > 128, N >= 128): one tile, ragged halves, odd k-block counts, several
+    # tiles per pair and more k-blocks than the operand ring holds
+    (129, 128, 128), (256, 256, 128), (200, 136, 384), (384, 520, 1664), (1000, 1288, 896),
+    (513, 2304, 2176),
 ]
 
 
