@@ -13,7 +13,9 @@
 //   warps 6..13   B: staging -> registers -> widen -> swizzled operand ring  } leader's full[s]
 //   warp 1        (leader CTA only) 8 MMAs of K = 32 per block; commit frees the ring stage in
 //                 both CTAs; the last commit of a tile publishes the accumulator to both CTAs
-//   warps 14..17  epilogue: TMEM -> dequantise -> fp16 stores, then hand the accumulator back
+//   warps 14..21  epilogue: TMEM -> dequantise -> fp16 tile in shared memory -> TMA store (which
+//                 also clips the ragged edges); two warps per TMEM lane quarter, four 32-column
+//                 chunks each; the accumulator is handed back as soon as it has been read
 // Every hand-over costs each warp a few hundred cycles of barrier and fence latency whatever the
 // amount of data, which is why a ring stage holds two k-blocks.
 // The widening and the operand byte order are those of the single-CTA kernel (sq_gemm.cu).
@@ -28,7 +30,7 @@ namespace {
 
 constexpr int P_A_WARPS = 4;
 constexpr int P_B_WARPS = 8;
-constexpr int P_EPI_WARPS = 4;
+constexpr int P_EPI_WARPS = 8;
 constexpr int P_THREADS = (2 + P_A_WARPS + P_B_WARPS + P_EPI_WARPS) * 32;
 constexpr int P_TILE_M = 256;            // tokens per pair tile (128 per CTA)
 constexpr int P_TILE_N = 256;            // output channels per pair tile (128 staged per CTA)
@@ -49,17 +51,32 @@ struct PairSmem {
   static constexpr int OFF_B_OP = 0;
   static constexpr int OFF_A_ST = OFF_B_OP + S_OP * B_OP;
   static constexpr int OFF_B_ST = OFF_A_ST + S_ST * A_ST;
-  static constexpr int OFF_BAR = OFF_B_ST + S_ST * B_ST;
+  static constexpr int OUT_BUF = 32 * 64;            // fp16 [32 rows x 32 columns], 64-byte swizzle
+  static constexpr int OFF_OUT = OFF_B_ST + S_ST * B_ST;
+  static constexpr int OFF_BAR = OFF_OUT + P_EPI_WARPS * 2 * OUT_BUF;
   static constexpr int NUM_BARS = 2 * S_OP + 2 * S_ST + 2;
   static constexpr int OFF_TMEM = OFF_BAR + NUM_BARS * 8;
   static constexpr int TOTAL = OFF_TMEM + 16;
   static constexpr int DYN_BYTES = TOTAL + 1024;
 };
 
+// 2-D fp16 map over Y [M x N]; box = 32 rows x 32 columns (64 bytes) with the 64-byte swizzle.
+bool make_out_map(CUtensorMap* map, void* Y, uint64_t M, uint64_t N) {
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return false;
+  const cuuint64_t dims[2] = {N, M};
+  const cuuint64_t strides[1] = {N * 2};
+  const cuuint32_t box[2] = {32, 32};
+  const cuuint32_t estr[2] = {1, 1};
+  return enc(map, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, Y, dims, strides, box, estr, CU_TENSOR_MAP_INTERLEAVE_NONE,
+             CU_TENSOR_MAP_SWIZZLE_64B, CU_TENSOR_MAP_L2_PROMOTION_NONE,
+             CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
 template <int S_OP, int S_ST>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1)
 w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                      const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
+                      const __grid_constant__ CUtensorMap tmap_y, const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
                       __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
   using L = PairSmem<S_OP, S_ST>;
   extern __shared__ unsigned char smem_dyn[];
@@ -85,6 +102,7 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmap_x);
     tma_prefetch_desc(&tmap_w);
+    tma_prefetch_desc(&tmap_y);
     for (int s = 0; s < S_ST; ++s) {
       mbar_init(&st_full[s], 1);
       mbar_init(&st_empty[s], P_A_WARPS + P_B_WARPS);
@@ -222,8 +240,11 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     }
   } else {
     // ------------------------------ epilogue ----------------------------------------------------
-    const int q = warp & 3;
-    uint32_t tcount = 0;
+    const int e = warp - (2 + P_A_WARPS + P_B_WARPS);   // 0 .. 7
+    const int q = warp & 3;                             // TMEM lane quarter this warp may read
+    const int c_first = (e >> 2) * 4;                   // this warp's four 32-column chunks
+    unsigned char* obuf = smem + L::OFF_OUT + e * 2 * L::OUT_BUF;
+    uint32_t tcount = 0, nstore = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += npairs, ++tcount) {
       const int m0 = (tile / tiles_n) * P_TILE_M + static_cast<int>(rank) * 128;
@@ -231,43 +252,54 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
       ok = mbar_wait(tmem_full, tcount & 1, PSITE_TMEM_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
-      const int row = m0 + q * 32 + lane;
+      const int row0 = m0 + q * 32, row = row0 + lane;
       const float sxv = (row < M) ? __half2float(sx[row]) : 0.0f;
       const uint32_t tmem_d = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
 #pragma unroll 1
-      for (int c = 0; c < P_TILE_N / 32; ++c) {
+      for (int j = 0; j < 4; ++j, ++nstore) {
+        const int c = c_first + j;
         uint32_t r[32];
         tmem_ld_32x32b_x32(tmem_d + c * 32, r);
         tmem_wait_ld();
+        if (j == 3) {                                   // last read of this warp: hand the accumulator back
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(tmem_empty, 0);
+        }
         const int col0 = n0 + c * 32;
-        if (row < M && col0 < N) {
-          __half* yrow = Y + static_cast<size_t>(row) * N + col0;
-          int32_t* arow = accdbg ? accdbg + static_cast<size_t>(row) * N + col0 : nullptr;
+        unsigned char* buf = obuf + (nstore & 1) * L::OUT_BUF;
+        if (nstore >= 2) {                              // the store issued two chunks ago has read `buf`
+          if (lane == 0) tma_store_wait_read_1();
+          __syncwarp();
+        }
 #pragma unroll
-          for (int g = 0; g < 4; ++g) {                 // groups of 8 columns (N % 8 == 0)
-            if (col0 + g * 8 < N) {
-              const uint4 swraw = __ldg(reinterpret_cast<const uint4*>(sw + col0 + g * 8));
-              const __half* swh = reinterpret_cast<const __half*>(&swraw);
-              __align__(16) __half h[8];
-              int32_t a[8];
+        for (int g = 0; g < 4; ++g) {                   // groups of 8 columns (N % 8 == 0)
+          uint4 swraw = make_uint4(0u, 0u, 0u, 0u);
+          if (col0 + g * 8 < N) swraw = __ldg(reinterpret_cast<const uint4*>(sw + col0 + g * 8));
+          const __half* swh = reinterpret_cast<const __half*>(&swraw);
+          __align__(16) __half h[8];
+          int32_t a[8];
 #pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                a[e] = static_cast<int32_t>(r[g * 8 + e]) >> 8;          // exact: the accumulator is 256 * acc
-                h[e] = __float2half_rn(static_cast<float>(a[e]) * (sxv * __half2float(swh[e])));
-              }
-              *reinterpret_cast<uint4*>(yrow + g * 8) = *reinterpret_cast<const uint4*>(h);
-              if (arow) {
-                *reinterpret_cast<int4*>(arow + g * 8) = make_int4(a[0], a[1], a[2], a[3]);
-                *reinterpret_cast<int4*>(arow + g * 8 + 4) = make_int4(a[4], a[5], a[6], a[7]);
-              }
-            }
+          for (int x = 0; x < 8; ++x) {
+            a[x] = static_cast<int32_t>(r[g * 8 + x]) >> 8;              // exact: the accumulator is 256 * acc
+            h[x] = __float2half_rn(static_cast<float>(a[x]) * (sxv * __half2float(swh[x])));
+          }
+          *reinterpret_cast<uint4*>(buf + lane * 64 + ((g ^ ((lane >> 1) & 3)) << 4)) = *reinterpret_cast<const uint4*>(h);
+          if (accdbg != nullptr && row < M && col0 + g * 8 < N) {
+            int32_t* arow = accdbg + static_cast<size_t>(row) * N + col0 + g * 8;
+            *reinterpret_cast<int4*>(arow) = make_int4(a[0], a[1], a[2], a[3]);
+            *reinterpret_cast<int4*>(arow + 4) = make_int4(a[4], a[5], a[6], a[7]);
           }
         }
+        fence_proxy_async_smem();                       // the tile in `buf` -> visible to the TMA store
+        __syncwarp();
+        if (lane == 0) {
+          if (row0 < M && col0 < N) tma_store_2d(&tmap_y, buf, col0, row0);
+          tma_store_commit();
+        }
       }
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive_cluster(tmem_empty, 0);
     }
+    if (lane == 0) tma_store_wait_all();
   }
 
   // Neither CTA may leave while its partner can still reach its shared memory, barriers or TMEM.
@@ -290,8 +322,10 @@ sq_status_t launch_w4a4_gemm_pair(const void* Xq, const void* sx, const void* Wq
                                   int K, void* Y, int32_t* accdbg, cudaStream_t s) {
   constexpr int S_OP = 3, S_ST = 3;
   using L = PairSmem<S_OP, S_ST>;
-  CUtensorMap mx, mw;
-  if (!make_packed_map(&mx, Xq, M, K / 2, 128) || !make_packed_map(&mw, Wq, N, K / 2, 128)) return SQ_ERR_CUDA;
+  CUtensorMap mx, mw, my;
+  if (!make_packed_map(&mx, Xq, M, K / 2, 128) || !make_packed_map(&mw, Wq, N, K / 2, 128) ||
+      !make_out_map(&my, Y, M, N))
+    return SQ_ERR_CUDA;
   auto kern = w4a4_gemm_pair_kernel<S_OP, S_ST>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -305,7 +339,7 @@ sq_status_t launch_w4a4_gemm_pair(const void* Xq, const void* sx, const void* Wq
     return SQ_ERR_CUDA;
   const int tiles = ((N + P_TILE_N - 1) / P_TILE_N) * ((M + P_TILE_M - 1) / P_TILE_M);
   const int pairs = tiles < sms / 2 ? tiles : sms / 2;
-  kern<<<2 * pairs, P_THREADS, L::DYN_BYTES, s>>>(mx, mw, static_cast<const __half*>(sx),
+  kern<<<2 * pairs, P_THREADS, L::DYN_BYTES, s>>>(mx, mw, my, static_cast<const __half*>(sx),
                                                   static_cast<const __half*>(sw), M, N, K,
                                                   static_cast<__half*>(Y), accdbg);
   count_launch();
