@@ -92,6 +92,27 @@ __device__ __forceinline__ void unpack_tile(const unsigned char* __restrict__ st
   }
 }
 
+// Dequantises eight accumulators (each 256 * acc, |acc| <= 2^22) of one token: exact shift, exact
+// int -> float through the 1.5 * 2^23 trick (one integer add and one float subtract instead of a
+// conversion instruction, whose throughput is a quarter of the ALU's), one fp32 product with the
+// combined step, one rounding to fp16 (two values per cvt.rn.f16x2).
+__device__ __forceinline__ uint4 dequant8(const uint32_t* r, float sxv, uint4 swraw, int32_t* a) {
+  const __half2* swh = reinterpret_cast<const __half2*>(&swraw);
+  uint4 out;
+  uint32_t* o = reinterpret_cast<uint32_t*>(&out);
+#pragma unroll
+  for (int e = 0; e < 4; ++e) {
+    const float2 sc = __half22float2(swh[e]);
+    a[2 * e] = static_cast<int32_t>(r[2 * e]) >> 8;
+    a[2 * e + 1] = static_cast<int32_t>(r[2 * e + 1]) >> 8;
+    const float f0 = __int_as_float(0x4B400000 + a[2 * e]) - 12582912.0f;
+    const float f1 = __int_as_float(0x4B400000 + a[2 * e + 1]) - 12582912.0f;
+    const __half2 h = __floats2half2_rn(f0 * (sxv * sc.x), f1 * (sxv * sc.y));
+    o[e] = *reinterpret_cast<const uint32_t*>(&h);
+  }
+  return out;
+}
+
 // Persistent kernel: CTA b works on tiles b, b + gridDim.x, ...; tile index = m_tile * tiles_n +
 // n_tile.  Warp 0 lane 0: TMA producer.  Warp 1 lane 0: MMA issuer.  Warps 2..9: unpack.
 // Warps 10..13: epilogue (TMEM -> dequant -> fp16 stores), overlapped with the next tile's main
@@ -246,15 +267,8 @@ w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
           for (int g = 0; g < 4; ++g) {                 // groups of 8 columns (N % 8 == 0)
             if (col0 + g * 8 < N) {
               const uint4 swraw = __ldg(reinterpret_cast<const uint4*>(sw + col0 + g * 8));
-              const __half* swh = reinterpret_cast<const __half*>(&swraw);
-              __align__(16) __half h[8];
               int32_t a[8];
-#pragma unroll
-              for (int e = 0; e < 8; ++e) {
-                a[e] = static_cast<int32_t>(r[g * 8 + e]) >> 8;          // exact: the accumulator is 256 * acc
-                h[e] = __float2half_rn(static_cast<float>(a[e]) * (sxv * __half2float(swh[e])));
-              }
-              *reinterpret_cast<uint4*>(yrow + g * 8) = *reinterpret_cast<const uint4*>(h);
+              *reinterpret_cast<uint4*>(yrow + g * 8) = dequant8(&r[g * 8], sxv, swraw, a);
               if (arow) {
                 *reinterpret_cast<int4*>(arow + g * 8) = make_int4(a[0], a[1], a[2], a[3]);
                 *reinterpret_cast<int4*>(arow + g * 8 + 4) = make_int4(a[4], a[5], a[6], a[7]);

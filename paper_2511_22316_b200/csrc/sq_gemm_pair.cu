@@ -249,11 +249,15 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     for (int tile = pair; tile < num_tiles && ok; tile += npairs, ++tcount) {
       const int m0 = (tile / tiles_n) * P_TILE_M + static_cast<int>(rank) * 128;
       const int n0 = (tile % tiles_n) * P_TILE_N;
+      // Fetched while the MMAs still run: this row's token step, and the channel steps of the warp's
+      // 128 columns, four per lane (handed round by shuffles when a chunk needs them).
+      const int row0 = m0 + q * 32, row = row0 + lane;
+      const float sxv = (row < M) ? __half2float(sx[row]) : 0.0f;
+      const int swcol = n0 + c_first * 32 + 4 * lane;
+      const uint2 swp = (swcol < N) ? __ldg(reinterpret_cast<const uint2*>(sw + swcol)) : make_uint2(0u, 0u);
       ok = mbar_wait(tmem_full, tcount & 1, PSITE_TMEM_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
-      const int row0 = m0 + q * 32, row = row0 + lane;
-      const float sxv = (row < M) ? __half2float(sx[row]) : 0.0f;
       const uint32_t tmem_d = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
 #pragma unroll 1
       for (int j = 0; j < 4; ++j, ++nstore) {
@@ -274,17 +278,13 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         }
 #pragma unroll
         for (int g = 0; g < 4; ++g) {                   // groups of 8 columns (N % 8 == 0)
-          uint4 swraw = make_uint4(0u, 0u, 0u, 0u);
-          if (col0 + g * 8 < N) swraw = __ldg(reinterpret_cast<const uint4*>(sw + col0 + g * 8));
-          const __half* swh = reinterpret_cast<const __half*>(&swraw);
-          __align__(16) __half h[8];
+          uint4 swraw;
+          swraw.x = __shfl_sync(0xffffffffu, swp.x, 8 * j + 2 * g);
+          swraw.y = __shfl_sync(0xffffffffu, swp.y, 8 * j + 2 * g);
+          swraw.z = __shfl_sync(0xffffffffu, swp.x, 8 * j + 2 * g + 1);
+          swraw.w = __shfl_sync(0xffffffffu, swp.y, 8 * j + 2 * g + 1);
           int32_t a[8];
-#pragma unroll
-          for (int x = 0; x < 8; ++x) {
-            a[x] = static_cast<int32_t>(r[g * 8 + x]) >> 8;              // exact: the accumulator is 256 * acc
-            h[x] = __float2half_rn(static_cast<float>(a[x]) * (sxv * __half2float(swh[x])));
-          }
-          *reinterpret_cast<uint4*>(buf + lane * 64 + ((g ^ ((lane >> 1) & 3)) << 4)) = *reinterpret_cast<const uint4*>(h);
+          *reinterpret_cast<uint4*>(buf + lane * 64 + ((g ^ ((lane >> 1) & 3)) << 4)) = dequant8(&r[g * 8], sxv, swraw, a);
           if (accdbg != nullptr && row < M && col0 + g * 8 < N) {
             int32_t* arow = accdbg + static_cast<size_t>(row) * N + col0 + g * 8;
             *reinterpret_cast<int4*>(arow) = make_int4(a[0], a[1], a[2], a[3]);
