@@ -9,6 +9,20 @@
 namespace sq {
 std::atomic<uint64_t> g_launches{0};
 
+int sm_count() {
+  static std::atomic<int> cache[64];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return -1;
+  if (dev >= 0 && dev < 64) {
+    const int c = cache[dev].load(std::memory_order_relaxed);
+    if (c > 0) return c;
+  }
+  int sms = 0;
+  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return -1;
+  if (dev >= 0 && dev < 64) cache[dev].store(sms, std::memory_order_relaxed);
+  return sms;
+}
+
 sq_status_t read_and_clear_device_status(cudaStream_t s) {
   if (cudaStreamSynchronize(s) != cudaSuccess) return SQ_ERR_CUDA;
   unsigned int v = 0;

@@ -361,10 +361,8 @@ sq_status_t launch_tc(const void* Xq, const void* sx, const void* Wq, const void
       return SQ_ERR_CUDA;
     attr_set = true;
   }
-  int dev = 0, sms = 148;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return SQ_ERR_CUDA;
+  const int sms = sm_count();
+  if (sms <= 0) return SQ_ERR_CUDA;
   const int tiles = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
   const int grid = tiles < sms ? tiles : sms;
   kern<<<grid, GEMM_THREADS, L::DYN_BYTES, s>>>(mx, mw, static_cast<const __half*>(sx),

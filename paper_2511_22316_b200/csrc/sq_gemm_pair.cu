@@ -333,10 +333,8 @@ sq_status_t launch_w4a4_gemm_pair(const void* Xq, const void* sx, const void* Wq
       return SQ_ERR_CUDA;
     attr_set = true;
   }
-  int dev = 0, sms = 148;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return SQ_ERR_CUDA;
+  const int sms = sm_count();
+  if (sms <= 0) return SQ_ERR_CUDA;
   const int tiles = ((N + P_TILE_N - 1) / P_TILE_N) * ((M + P_TILE_M - 1) / P_TILE_M);
   const int pairs = tiles < sms / 2 ? tiles : sms / 2;
   kern<<<2 * pairs, P_THREADS, L::DYN_BYTES, s>>>(mx, mw, my, static_cast<const __half*>(sx),

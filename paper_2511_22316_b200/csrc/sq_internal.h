@@ -26,6 +26,9 @@ namespace sq {
 extern std::atomic<uint64_t> g_launches;
 inline void count_launch(uint64_t k = 1) { g_launches.fetch_add(k, std::memory_order_relaxed); }
 
+// Multiprocessor count of the current device (cached per device; <= 0 on failure).
+int sm_count();
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Host-side construction of the factors in float64 (sq_rotation_host.cu).

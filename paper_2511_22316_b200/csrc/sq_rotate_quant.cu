@@ -245,9 +245,8 @@ sq_status_t launch_rotate_quant(const float* dR1, const float* dR2, int n1, int 
                                 int64_t rows, void* Xq, void* scales, float* Zdbg, cudaStream_t s) {
   if (rows == 0) return SQ_OK;
   const long long n = static_cast<long long>(n1) * n2;
-  int dev = 0, sms = 148;
-  if (cudaGetDevice(&dev) != cudaSuccess) return SQ_ERR_CUDA;
-  if (cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess) return SQ_ERR_CUDA;
+  const int sms = sm_count();
+  if (sms <= 0) return SQ_ERR_CUDA;
 
   if (dR1 == nullptr || dR2 == nullptr) {
     const long long grid = std::min<long long>(rows, static_cast<long long>(sms) * 8);

@@ -114,6 +114,17 @@ __device__ __forceinline__ uint32_t pack8_codes(const float* t) {
   return (w - kBias) ^ 0x88888888u;
 }
 
+// max |r[e]| over 32 fp32 bit patterns, as a tree (four independent chains).
+__device__ __forceinline__ float absmax32(const uint32_t (&r)[32]) {
+  float m[4] = {0.0f, 0.0f, 0.0f, 0.0f};
+#pragma unroll
+  for (int e = 0; e < 32; e += 8)
+#pragma unroll
+    for (int x = 0; x < 4; ++x)
+      m[x] = fmaxf(m[x], fmaxf(fabsf(__uint_as_float(r[e + 2 * x])), fabsf(__uint_as_float(r[e + 2 * x + 1]))));
+  return fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
+}
+
 template <int N2>
 __global__ void __launch_bounds__((2 + 4 * (256 / N2)) * 32, 1)
 rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigned char* __restrict__ a1_img,
@@ -147,6 +158,18 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
   const long long my_groups = (ngroups > blockIdx.x) ? (ngroups - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
   const uint32_t limit = wait_limit();
 
+  // One X tile set per token group: G tokens, XQ 64-column blocks each.
+  auto load_group = [&](long long i) {
+    const long long g = blockIdx.x + i * gridDim.x;
+    const int s = static_cast<int>(i % L.XS);
+    mbar_arrive_expect_tx(&x_full[s], static_cast<uint32_t>(L.x_bytes));
+    for (int tk = 0; tk < G; ++tk)
+      for (int a = 0; a < XQ; ++a)
+        tma_load_3d(xs + s * L.x_bytes + tk * L.x_token + a * L.x_tile, &tmap_x, &x_full[s], a * 64, 0,
+                    static_cast<int32_t>(g * G + tk));
+  };
+  const long long preload = my_groups < L.XS ? my_groups : L.XS;
+
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmap_x);
     for (int b = 0; b < 4; ++b) {
@@ -159,8 +182,16 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
     }
     mbar_init(img_full, 1);
     mbar_fence_init();
+    // The first loads go out before the rest of the CTA has finished setting up: the whole X ring,
+    // then the factor images.
+    for (long long i = 0; i < preload; ++i) load_group(i);
+    mbar_arrive_expect_tx(img_full, static_cast<uint32_t>(L.a1_bytes + L.b2_bytes));
+    for (int o = 0; o < L.a1_bytes; o += 16384)
+      bulk_load_1d(a1s + o, a1_img + o, static_cast<uint32_t>(min(16384, L.a1_bytes - o)), img_full);
+    for (int o = 0; o < L.b2_bytes; o += 16384)
+      bulk_load_1d(b2s + o, b2_img + o, static_cast<uint32_t>(min(16384, L.b2_bytes - o)), img_full);
   }
-  if (warp == 0) {
+  if (warp == 1) {
     tmem_alloc(tmem_slot, 512);
     tmem_relinquish();
   }
@@ -170,22 +201,11 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
-    // ------------------------------ producer: factor images once, then one X tile set per group ------
-    if (elect_one()) {
-      mbar_arrive_expect_tx(img_full, static_cast<uint32_t>(L.a1_bytes + L.b2_bytes));
-      for (int o = 0; o < L.a1_bytes; o += 16384)
-        bulk_load_1d(a1s + o, a1_img + o, static_cast<uint32_t>(min(16384, L.a1_bytes - o)), img_full);
-      for (int o = 0; o < L.b2_bytes; o += 16384)
-        bulk_load_1d(b2s + o, b2_img + o, static_cast<uint32_t>(min(16384, L.b2_bytes - o)), img_full);
-      for (long long i = 0; i < my_groups; ++i) {
-        const long long g = blockIdx.x + i * gridDim.x;
-        const int s = static_cast<int>(i % L.XS);
-        if (!mbar_wait(&x_empty[s], ((i / L.XS) & 1) ^ 1, RQ_X_EMPTY, limit)) break;
-        mbar_arrive_expect_tx(&x_full[s], static_cast<uint32_t>(L.x_bytes));
-        for (int tk = 0; tk < G; ++tk)
-          for (int a = 0; a < XQ; ++a)
-            tma_load_3d(xs + s * L.x_bytes + tk * L.x_token + a * L.x_tile, &tmap_x, &x_full[s], a * 64, 0,
-                        static_cast<int32_t>(g * G + tk));
+    // ------------------------------ producer: keeps the X ring full -------------------------------------
+    if (lane == 0) {
+      for (long long i = preload; i < my_groups; ++i) {
+        if (!mbar_wait(&x_empty[i % L.XS], ((i / L.XS) & 1) ^ 1, RQ_X_EMPTY, limit)) break;
+        load_group(i);
       }
     }
   } else if (warp == 1) {
@@ -194,25 +214,23 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
       // stage 1: A K-major (shared), B MN-major (bit 16); stage 2: A from TMEM, B K-major
       const uint32_t idesc1 = umma_idesc(/*c=f32*/ 1, /*a=f16*/ 0, /*b=f16*/ 0, 128, N2) | (1u << 16);
       const uint32_t idesc2 = umma_idesc(/*c=f32*/ 1, /*a=f16*/ 0, /*b=f16*/ 0, 128, N2);
-      const uint32_t a1_addr = smem_u32(a1s), b2_addr = smem_u32(b2s), x_addr = smem_u32(xs);
+      const uint64_t a1_desc0 = umma_desc_sw128(smem_u32(a1s)), b2_desc0 = umma_desc_sw128(smem_u32(b2s));
+      const uint64_t x_desc0 = umma_desc_sw128_mn(smem_u32(xs), static_cast<uint32_t>(L.x_tile));
       const int ksteps1 = L.N1 / 16;                 // K = p, 16 per MMA
       bool ok = mbar_wait(img_full, 0, RQ_IMG, limit);
       auto stage1 = [&](long long i) {
         const int slot = static_cast<int>(i % S), xs_i = static_cast<int>(i % L.XS);
-        ok = mbar_wait(&x_full[xs_i], (i / L.XS) & 1, RQ_X_FULL, limit) &&
-             mbar_wait(&d_free[slot], ((i / S) & 1) ^ 1, RQ_D_FREE, limit);
-        if (!ok) return;
         tc_fence_after_sync();
         const uint32_t d1 = tmem_base + slot * SLOT_COLS;
         uint32_t acc = 0;
+        // descriptors differ only in their start-address field (16-byte units, no carry out of it)
         for (int tk = 0; tk < G; ++tk) {
-          const uint32_t xb = x_addr + xs_i * L.x_bytes + tk * L.x_token;
-          const uint32_t ab = a1_addr + (128 - LS - tk * LS) * 128;
-          for (int ks = 0; ks < ksteps1; ++ks) {
-            const uint64_t bd = umma_desc_sw128_mn(xb + ks * 2048, static_cast<uint32_t>(L.x_tile));
-            const uint32_t ao = ab + (ks >> 2) * L.a1_tile + (ks & 3) * 32;
-            umma_f16(d1, umma_desc_sw128(ao), bd, idesc1, acc);               // hi
-            umma_f16(d1, umma_desc_sw128(ao + L.a1_part), bd, idesc1, 1u);    // lo
+          uint64_t bd = x_desc0 + ((xs_i * L.x_bytes + tk * L.x_token) >> 4);
+          const uint64_t ad = a1_desc0 + (((128 - LS - tk * LS) * 128) >> 4);
+          for (int ks = 0; ks < ksteps1; ++ks, bd += 2048 >> 4) {
+            const uint64_t ah = ad + (((ks >> 2) * L.a1_tile + (ks & 3) * 32) >> 4);
+            umma_f16(d1, ah, bd, idesc1, acc);                         // hi
+            umma_f16(d1, ah + (L.a1_part >> 4), bd, idesc1, 1u);       // lo
             acc = 1;
           }
         }
@@ -221,25 +239,39 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
       };
       auto stage2 = [&](long long i) {
         const int slot = static_cast<int>(i % S);
-        ok = mbar_wait(&a2_ready[slot], (i / S) & 1, RQ_A2_READY, limit);
-        if (!ok) return;
         tc_fence_after_sync();
         const uint32_t d1 = tmem_base + slot * SLOT_COLS, d2 = d1 + N2;
 #pragma unroll
         for (int j = 0; j < N2 / 16; ++j) {
-          const uint32_t off = (j >> 2) * L.b2_tile + (j & 3) * 32;
-          const uint64_t bh = umma_desc_sw128(b2_addr + off), bl = umma_desc_sw128(b2_addr + L.b2_part + off);
+          const uint64_t bh = b2_desc0 + (((j >> 2) * L.b2_tile + (j & 3) * 32) >> 4), bl = bh + (L.b2_part >> 4);
           umma_f16_ts(d2, d1 + 16 * j, bh, idesc2, j > 0 ? 1u : 0u);      // hi * hi
           umma_f16_ts(d2, d1 + 16 * j + 8, bh, idesc2, 1u);               // lo * hi
           umma_f16_ts(d2, d1 + 16 * j, bl, idesc2, 1u);                   // hi * lo
         }
         umma_commit(&d2_full[slot]);
       };
-      for (long long i = 0; i < S - 1 && i < my_groups && ok; ++i) stage1(i);
-      for (long long i = 0; i < my_groups && ok; ++i) {
-        if (i + S - 1 < my_groups) stage1(i + S - 1);
-        if (!ok) break;
-        stage2(i);
+      // Whichever is ready goes: stage 1 of the next group whose X tile has landed and whose slot has
+      // been drained, and stage 2 of the oldest group whose operand has been converted.
+      long long i1 = 0, i2 = 0;
+      uint32_t idle = 0;
+      while (ok && i2 < my_groups) {
+        bool did = false;
+        if (i1 < my_groups && i1 < i2 + S &&
+            mbar_test_wait(&x_full[i1 % L.XS], (i1 / L.XS) & 1) &&
+            mbar_test_wait(&d_free[i1 % S], ((i1 / S) & 1) ^ 1)) {
+          stage1(i1++);
+          did = true;
+        }
+        if (i2 < i1 && mbar_test_wait(&a2_ready[i2 % S], (i2 / S) & 1)) {
+          stage2(i2++);
+          did = true;
+        }
+        if (did) {
+          idle = 0;
+        } else if (++idle > limit) {
+          atomicCAS(&g_device_status, 0u, (static_cast<uint32_t>(RQ_A2_READY) << 8) | 1u);
+          ok = false;
+        }
       }
     }
   } else {
@@ -268,9 +300,7 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
         uint32_t r[32];
         tmem_ld_32x32b_x32(d1 + 32 * c, r);
         tmem_wait_ld();
-#pragma unroll
-        for (int e = 0; e < 32; e += 2)
-          m = fmaxf(m, fmaxf(fabsf(__uint_as_float(r[e])), fabsf(__uint_as_float(r[e + 1]))));
+        m = fmaxf(m, absmax32(r));
       }
       // scale so that the lane's largest entry lands in [2^13, 2^14)
       int ebits = static_cast<int>((__float_as_uint(m) >> 23) & 0xFF);
@@ -313,9 +343,7 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
         uint32_t r[32];
         tmem_ld_32x32b_x32(d2 + 32 * c, r);
         tmem_wait_ld();
-#pragma unroll
-        for (int e = 0; e < 32; e += 2)
-          zm = fmaxf(zm, fmaxf(fabsf(__uint_as_float(r[e])), fabsf(__uint_as_float(r[e + 1]))));
+        zm = fmaxf(zm, absmax32(r));
       }
       zm *= un;                                      // lanes of padding rows hold exact zeros
 #pragma unroll
@@ -372,7 +400,7 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
 
   tc_fence_before_sync();
   __syncthreads();
-  if (warp == 0) {
+  if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, 512);
   }
@@ -450,10 +478,8 @@ sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t 
           CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return SQ_ERR_CUDA;
-  int dev = 0, sms = 148;
-  if (cudaGetDevice(&dev) != cudaSuccess ||
-      cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev) != cudaSuccess)
-    return SQ_ERR_CUDA;
+  const int sms = sm_count();
+  if (sms <= 0) return SQ_ERR_CUDA;
   // More than half of an SM's shared memory, so that two CTAs (each wanting all of TMEM) never share one.
   const int smem = std::max(L.total + 1024, 120 * 1024);
   const long long ngroups = (rows + L.G - 1) / L.G;
@@ -462,12 +488,20 @@ sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t 
   const unsigned char* b2 = static_cast<const unsigned char*>(h->dB2img);
   if (n2 == 64) {
     auto kern = rotate_quant_tc_kernel<64>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SQ_ERR_CUDA;
+    static int smem_set = 0;                      // largest size the attribute has been raised to
+    if (smem > smem_set) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SQ_ERR_CUDA;
+      smem_set = smem;
+    }
     kern<<<grid, (2 + 4 * 4) * 32, smem, s>>>(mx, a1, b2, n1, rows, static_cast<uint8_t*>(Xq),
                                               static_cast<__half*>(scales), Zdbg);
   } else {
     auto kern = rotate_quant_tc_kernel<128>;
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SQ_ERR_CUDA;
+    static int smem_set = 0;
+    if (smem > smem_set) {
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SQ_ERR_CUDA;
+      smem_set = smem;
+    }
     kern<<<grid, (2 + 4 * 2) * 32, smem, s>>>(mx, a1, b2, n1, rows, static_cast<uint8_t*>(Xq),
                                               static_cast<__half*>(scales), Zdbg);
   }
