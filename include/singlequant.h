@@ -130,6 +130,31 @@ sq_status_t sq_linear(const sq_rotation_t* rot, const void* X, int64_t M,
                       const void* Wq, const void* sw, int64_t N, int64_t K,
                       void* workspace, size_t workspace_bytes, void* Y, void* stream);
 
+/* sq_linear without a caller workspace and without any allocation on the call path.
+ * (The paper has no counterpart: this is a deployment variant of sq_linear.)
+ *
+ * For callers that cannot obtain device memory where they evaluate a layer: a serving loop that
+ * must stay out of cudaMalloc (which synchronises the device and may fail under memory pressure),
+ * a plugin that is handed input and output tensors by its host framework but no allocator, a
+ * process whose device memory is already split into fixed pools.  The packed activations and
+ * their steps go to a scratch array of SQ_LINEAR_STATIC_SCRATCH_BYTES that is part of the library
+ * image; every GPU that loads the library holds it until the process exits.
+ *   - Arguments as sq_linear, minus the workspace.  All pointers DEVICE; the caller owns X, Wq,
+ *     sw and Y.
+ *   - Limit: sq_linear_workspace_bytes(M, N, K) <= SQ_LINEAR_STATIC_SCRATCH_BYTES, i.e. roughly
+ *     M * K / 2 + 2 * M bytes (LLaMA-2-7B prefill, 2048 x 4096, needs 4.2 MB).  Larger problems
+ *     return SQ_ERR_UNSUPPORTED before anything is launched: split M, or use sq_linear.
+ *   - The first call on each device looks up the scratch's device address (a CUDA runtime query,
+ *     no allocation).  Make that first call outside any stream capture; later calls only launch.
+ *   - The call itself never calls cudaMalloc, cudaFree or any allocating routine.
+ *   - One array serves every call on a device, and it keeps what the last call wrote.  Nothing in
+ *     it needs clearing (each call rewrites all it reads), but two calls that overlap on the GPU
+ *     (different streams, or two host threads) race on it: serialise them, e.g. on one stream. */
+#define SQ_LINEAR_STATIC_SCRATCH_BYTES (8u << 20)
+sq_status_t sq_linear_static(const sq_rotation_t* rot, const void* X, int64_t M,
+                             const void* Wq, const void* sw, int64_t N, int64_t K,
+                             void* Y, void* stream);
+
 /* The whole layer from HOST activations to HOST outputs: copies X (HOST fp16 [M x n], pinned
  * memory recommended) to the device, runs sq_linear, copies Y back (HOST fp16 [M x N]) and
  * waits for the stream.  Weights stay on the device.

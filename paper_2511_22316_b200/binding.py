@@ -26,7 +26,7 @@ EXPORTS = (
     "sq_factorize", "sq_build_rotation", "sq_rotation_from_factors", "sq_rotation_get_factors",
     "sq_rotation_dims", "sq_rotation_destroy", "sq_rotate_quant_act", "sq_pack_weight",
     "sq_w4a4_gemm_workspace_bytes", "sq_w4a4_gemm", "sq_linear_workspace_bytes", "sq_linear",
-    "sq_linear_host_workspace_bytes", "sq_linear_host", "sq_last_device_status",
+    "sq_linear_static", "sq_linear_host_workspace_bytes", "sq_linear_host", "sq_last_device_status",
     "sq_kernel_launch_count", "sq_status_string",
 )
 
@@ -67,6 +67,8 @@ def load() -> ctypes.CDLL:
     lib.sq_linear_workspace_bytes.restype = c_size_t
     lib.sq_linear.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_int64,
                               c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.sq_linear_static.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_int64,
+                                     c_void_p, c_void_p]
     lib.sq_linear_host_workspace_bytes.argtypes = [c_int64, c_int64, c_int64]
     lib.sq_linear_host_workspace_bytes.restype = c_size_t
     lib.sq_linear_host.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_int64,
@@ -205,6 +207,17 @@ def sq_linear(rot: Rotation, X, M: int, Wq, sw, N: int, K: int, workspace, works
               stream=None) -> None:
     _check(load().sq_linear(rot.handle, _ptr(X), M, _ptr(Wq), _ptr(sw), N, K, _ptr(workspace), workspace_bytes,
                             _ptr(Y), _stream(stream)), "sq_linear")
+
+
+SQ_LINEAR_STATIC_SCRATCH_BYTES = 8 << 20
+
+
+def sq_linear_static(rot: Rotation, X, M: int, Wq, sw, N: int, K: int, Y, stream=None) -> None:
+    """sq_linear with the library's built-in scratch: no workspace argument, no allocation on the
+    call path (for callers that cannot allocate device memory; see the header).  Problems whose
+    workspace exceeds SQ_LINEAR_STATIC_SCRATCH_BYTES raise SingleQuantError(SQ_ERR_UNSUPPORTED)."""
+    _check(load().sq_linear_static(rot.handle, _ptr(X), M, _ptr(Wq), _ptr(sw), N, K, _ptr(Y), _stream(stream)),
+           "sq_linear_static")
 
 
 def sq_linear_host_workspace_bytes(M: int, N: int, K: int) -> int:

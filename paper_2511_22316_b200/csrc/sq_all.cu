@@ -6,3 +6,4 @@
 #include "sq_rotate_quant_tc.cu"
 #include "sq_rotation_host.cu"
 #include "sq_api.cu"
+#include "sq_noalloc.cu"
