@@ -128,3 +128,14 @@ def make_weights(w: Workload, N: Optional[int] = None) -> np.ndarray:
 
 def make_layer(w: Workload):
     return make_activations(w), make_weights(w)
+
+
+def shard_rows(M: int, world: int, rank: int) -> Tuple[int, int]:
+    """Token rows [start, start + count) owned by `rank` of `world` when a batch is split for
+    data-parallel inference: contiguous, sizes differing by at most one, earlier ranks larger.
+    Tokens are independent in every step of the path, so shards need no exchange."""
+    if world < 1 or not (0 <= rank < world) or M < 0:
+        raise ValueError("bad shard request")
+    base, extra = divmod(M, world)
+    start = rank * base + min(rank, extra)
+    return start, base + (1 if rank < extra else 0)
