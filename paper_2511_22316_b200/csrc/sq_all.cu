@@ -4,6 +4,7 @@
 #include "sq_gemm_pair.cu"
 #include "sq_rotate_quant.cu"
 #include "sq_rotate_quant_tc.cu"
+#include "sq_rotate_quant_pair.cu"
 #include "sq_rotation_host.cu"
 #include "sq_api.cu"
 #include "sq_noalloc.cu"

@@ -43,6 +43,7 @@ sq_status_t rotate_quant_dispatch(const sq_rotation* h, const void* X, int64_t r
                                   float* Zdbg, cudaStream_t s) {
   static const bool force_generic = getenv("SQ_ROTATE_GENERIC") != nullptr;
   if (h->tc_ready && !force_generic) return launch_rotate_quant_tc(h, X, rows, Xq, scales, Zdbg, s);
+  if (h->tc_pair && !force_generic) return launch_rotate_quant_pair(h, X, rows, Xq, scales, Zdbg, s);
   return launch_rotate_quant(h->dR1, h->dR2, h->n1, h->n2, X, rows, Xq, scales, Zdbg, s);
 }
 }  // namespace sq
@@ -77,7 +78,10 @@ sq_status_t make_handle(std::vector<float>&& R1, std::vector<float>&& R2, int32_
     delete h;
     return SQ_ERR_CUDA;
   }
-  if (sq::rotate_quant_tc_supported(n1, n2) && !sq::rotate_quant_tc_prepare(h)) {
+  const bool prepared = sq::rotate_quant_tc_supported(n1, n2)     ? sq::rotate_quant_tc_prepare(h)
+                        : sq::rotate_quant_pair_supported(n1, n2) ? sq::rotate_quant_pair_prepare(h)
+                                                                  : true;
+  if (!prepared) {
     sq_rotation_destroy(h);
     return SQ_ERR_CUDA;
   }

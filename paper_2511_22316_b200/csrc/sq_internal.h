@@ -18,7 +18,8 @@ struct sq_rotation {
   // tensor-core rotate+quant: shared-memory images of the split factors (device), if supported
   void* dA1img = nullptr;
   void* dB2img = nullptr;
-  bool tc_ready = false;
+  bool tc_ready = false;   // images for the single-CTA kernel (n1 <= 128)
+  bool tc_pair = false;    // images for the CTA-pair kernel (128 < n1 <= 256)
 };
 
 namespace sq {
@@ -45,6 +46,11 @@ bool rotate_quant_tc_supported(int n1, int n2);
 bool rotate_quant_tc_prepare(sq_rotation* h);
 sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
                                    float* Zdbg, cudaStream_t s);
+// Tensor-core variant for 128 < n1 <= 256 on CTA pairs (sq_rotate_quant_pair.cu).
+bool rotate_quant_pair_supported(int n1, int n2);
+bool rotate_quant_pair_prepare(sq_rotation* h);
+sq_status_t launch_rotate_quant_pair(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
+                                     float* Zdbg, cudaStream_t s);
 // Picks the tensor-core kernel when the handle has its images, else the generic fp32 kernel.
 sq_status_t rotate_quant_dispatch(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
                                   float* Zdbg, cudaStream_t s);

@@ -114,7 +114,9 @@ SMALL_ROT = [(2, 2, 1), (3, 4, 3), (5, 8, 2), (8, 2, 4), (12, 8, 5), (1, 8, 2), 
              (20, 16, 9), (64, 64, 37), (172, 64, 5), (112, 128, 4), (64, 128, 6), (224, 128, 3), (256, 128, 2),
              # tensor-core kernel: 4, 2 and 1 tokens per accumulator, ragged n1, ragged token groups
              (8, 64, 9), (24, 64, 7), (32, 128, 5), (48, 64, 11), (100, 128, 3), (128, 64, 5), (128, 128, 3),
-             (64, 64, 301)]
+             (64, 64, 301),
+             # CTA-pair tensor-core kernel (128 < n1 <= 256): 64- and 128-byte half tiles, ragged second block
+             (129, 64, 3), (160, 64, 75), (172, 64, 9), (224, 128, 5), (256, 64, 4), (144, 128, 150)]
 
 
 @pytest.mark.parametrize("n1,n2,M", SMALL_ROT)
