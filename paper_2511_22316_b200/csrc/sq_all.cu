@@ -2,6 +2,7 @@
 // file-scope device symbols, so everything is compiled together (no relocatable device code).
 #include "sq_gemm.cu"
 #include "sq_gemm_pair.cu"
+#include "sq_gemm_decode.cu"
 #include "sq_rotate_quant.cu"
 #include "sq_rotate_quant_tc.cu"
 #include "sq_rotate_quant_pair.cu"
