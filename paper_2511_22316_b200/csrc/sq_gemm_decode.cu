@@ -11,9 +11,11 @@
 // the item that completes a tile (a counter per tile) adds the partials in a fixed order,
 // dequantises and writes fp16 -- the result does not depend on which item came last.
 //
-// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..5 = weight converters,
-// warps 6..7 = token unpackers, warps 8..11 = epilogue (two accumulators, so an item's epilogue
-// overlaps the next item's main loop).
+// Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = two groups of weight
+// converters and warps 10..13 = two groups of token unpackers (a group takes every other block:
+// a block costs a warp several hundred cycles of waits and fences whatever its size), warps
+// 14..21 = two epilogue groups that take the items in turn (four accumulators, so epilogues,
+// whose global-memory round trips are long, overlap the main loop of the following items).
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -23,12 +25,15 @@
 namespace sq {
 namespace {
 
-constexpr int D_A_WARPS = 4, D_B_WARPS = 2, D_EPI_WARPS = 4;
+constexpr int D_CONV_GROUPS = 2;          // converter groups; group g takes the blocks g, g + 2, ...
+constexpr int D_A_WARPS = 4 * D_CONV_GROUPS, D_B_WARPS = 2 * D_CONV_GROUPS;
+constexpr int D_EPI_GROUPS = 2, D_EPI_WARPS = 4 * D_EPI_GROUPS;
 constexpr int D_THREADS = (2 + D_A_WARPS + D_B_WARPS + D_EPI_WARPS) * 32;
 constexpr int D_S_ST = 6;                // staging stages (256 channels each)
 constexpr int D_S_OP = 4;                // operand stages (TMEM A ring: 4 x 64 columns)
 constexpr int D_A_COL0 = 256;
-constexpr int D_MAX_SPLITS = 32;
+constexpr int D_MAX_SPLITS = 16;           // partial tiles of one output tile, all in flight when they are summed
+constexpr int D_ACCS = 4;                 // accumulators in TMEM (columns 0 .. 4 * NT)
 
 enum DecSite : uint32_t {
   DSITE_ST_EMPTY = 64, DSITE_ST_FULL_A, DSITE_ST_FULL_B, DSITE_EMPTY_A, DSITE_EMPTY_B, DSITE_FULL,
@@ -44,7 +49,7 @@ struct DecSmem {
   static constexpr int OFF_W_ST = OFF_X_OP + D_S_OP * X_OP;
   static constexpr int OFF_X_ST = OFF_W_ST + D_S_ST * W_ST;
   static constexpr int OFF_BAR = OFF_X_ST + D_S_ST * X_ST;
-  static constexpr int NUM_BARS = 2 * D_S_ST + 2 * D_S_OP + 4;
+  static constexpr int NUM_BARS = 2 * D_S_ST + 2 * D_S_OP + 2 * D_ACCS;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int TOTAL = OFF_MISC + 32;
   static constexpr int DYN_BYTES = TOTAL + 1024;
@@ -102,10 +107,10 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   uint64_t* st_empty = bars + D_S_ST;
   uint64_t* full = bars + 2 * D_S_ST;
   uint64_t* empty = bars + 2 * D_S_ST + D_S_OP;
-  uint64_t* tmem_full = bars + 2 * D_S_ST + 2 * D_S_OP;      // [2]
-  uint64_t* tmem_empty = tmem_full + 2;                       // [2]
+  uint64_t* tmem_full = bars + 2 * D_S_ST + 2 * D_S_OP;      // [D_ACCS]
+  uint64_t* tmem_empty = tmem_full + D_ACCS;                  // [D_ACCS]
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
-  uint32_t* last_flag = tmem_slot + 1;
+  uint32_t* last_flag = tmem_slot + 1;                        // [D_EPI_GROUPS]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = K / 128;
@@ -114,22 +119,56 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   const int num_items = tiles * splits;
   const uint32_t limit = wait_limit();
 
+  // item -> (tile, first block, one-past-last block)
+  auto item_range = [&](int item, int& tile, int& b0, int& b1) {
+    tile = item / splits;
+    const int sp = item % splits;
+    b0 = static_cast<int>(static_cast<long long>(sp) * num_sb / splits);
+    b1 = static_cast<int>(static_cast<long long>(sp + 1) * num_sb / splits);
+  };
+  // The producer's walk over (item, block); `budget` blocks are issued per call (waiting for the
+  // staging stage of each), so that the first ring-full can go out before the CTA has set up.
+  int p_item = blockIdx.x, p_sb = -1, p_b1 = 0, p_tile = 0;
+  uint32_t p_it = 0;
+  auto produce = [&](uint32_t budget) -> bool {
+    while (budget > 0 && p_item < num_items) {
+      if (p_sb < 0) {
+        int b0;
+        item_range(p_item, p_tile, b0, p_b1);
+        p_sb = b0;
+      }
+      const int ss = p_it % D_S_ST;
+      if (!mbar_wait(&st_empty[ss], ((p_it / D_S_ST) & 1) ^ 1, DSITE_ST_EMPTY, limit)) return false;
+      mbar_arrive_expect_tx(&st_full[ss], L::W_ST + L::X_ST);
+      tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, &tmap_w, &st_full[ss], p_sb * 128, p_tile * 128);
+      tma_load_2d(smem + L::OFF_X_ST + ss * L::X_ST, &tmap_x, &st_full[ss], p_sb * 128, 0);
+      ++p_it;
+      --budget;
+      if (++p_sb >= p_b1) {
+        p_sb = -1;
+        p_item += gridDim.x;
+      }
+    }
+    return true;
+  };
+
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmap_w);
     tma_prefetch_desc(&tmap_x);
     for (int s = 0; s < D_S_ST; ++s) {
       mbar_init(&st_full[s], 1);
-      mbar_init(&st_empty[s], D_A_WARPS + D_B_WARPS);
+      mbar_init(&st_empty[s], 6);                      // one converter group + one unpacker group
     }
     for (int s = 0; s < D_S_OP; ++s) {
-      mbar_init(&full[s], D_A_WARPS + D_B_WARPS);
+      mbar_init(&full[s], 6);
       mbar_init(&empty[s], 1);
     }
-    for (int b = 0; b < 2; ++b) {
+    for (int b = 0; b < D_ACCS; ++b) {
       mbar_init(&tmem_full[b], 1);
-      mbar_init(&tmem_empty[b], D_EPI_WARPS);
+      mbar_init(&tmem_empty[b], 4);
     }
     mbar_fence_init();
+    produce(D_S_ST);                                   // the whole staging ring, before anyone else is ready
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, 512);
@@ -140,32 +179,9 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
 
-  // item -> (tile, first block, one-past-last block)
-  auto item_range = [&](int item, int& tile, int& b0, int& b1) {
-    tile = item / splits;
-    const int sp = item % splits;
-    b0 = static_cast<int>(static_cast<long long>(sp) * num_sb / splits);
-    b1 = static_cast<int>(static_cast<long long>(sp + 1) * num_sb / splits);
-  };
-
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------------------------
-    if (lane == 0) {
-      uint32_t it = 0;
-      bool ok = true;
-      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
-        int tile, b0, b1;
-        item_range(item, tile, b0, b1);
-        for (int sb = b0; sb < b1; ++sb, ++it) {
-          const int ss = it % D_S_ST;
-          ok = mbar_wait(&st_empty[ss], ((it / D_S_ST) & 1) ^ 1, DSITE_ST_EMPTY, limit);
-          if (!ok) break;
-          mbar_arrive_expect_tx(&st_full[ss], L::W_ST + L::X_ST);
-          tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, &tmap_w, &st_full[ss], sb * 128, tile * 128);
-          tma_load_2d(smem + L::OFF_X_ST + ss * L::X_ST, &tmap_x, &st_full[ss], sb * 128, 0);
-        }
-      }
-    }
+    if (lane == 0) produce(0xFFFFFFFFu);
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------------------------
     if (elect_one()) {
@@ -175,8 +191,8 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
       for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++icount) {
         int tile, b0, b1;
         item_range(item, tile, b0, b1);
-        const uint32_t acc = icount & 1;
-        ok = mbar_wait(&tmem_empty[acc], ((icount >> 1) & 1) ^ 1, DSITE_TMEM_EMPTY, limit);
+        const uint32_t acc = icount % D_ACCS;
+        ok = mbar_wait(&tmem_empty[acc], ((icount / D_ACCS) & 1) ^ 1, DSITE_TMEM_EMPTY, limit);
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * NT;
@@ -200,6 +216,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   } else if (warp < 2 + D_A_WARPS) {
     // ------------------------------ weight converters: staging -> registers -> TMEM --------------
     const int q = warp & 3;
+    const int grp = (warp - 2) >> 2;                    // this group's blocks: it % D_CONV_GROUPS == grp
     const int r = q * 32 + lane;
     const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
     uint32_t it = 0;
@@ -208,6 +225,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
       int tile, b0, b1;
       item_range(item, tile, b0, b1);
       for (int sb = b0; sb < b1 && ok; ++sb, ++it) {
+        if ((it % D_CONV_GROUPS) != static_cast<uint32_t>(grp)) continue;
         const int ss = it % D_S_ST, s = it % D_S_OP;
         ok = mbar_wait(&st_full[ss], (it / D_S_ST) & 1, DSITE_ST_FULL_A, limit);
         if (!ok) break;
@@ -245,18 +263,20 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     }
   } else if (warp < 2 + D_A_WARPS + D_B_WARPS) {
     // ------------------------------ token unpackers: staging -> operand ring ----------------------
-    const int t = threadIdx.x - (2 + D_A_WARPS) * 32;
+    const int grp = (warp - (2 + D_A_WARPS)) >> 1;
+    const int t = (threadIdx.x - (2 + D_A_WARPS) * 32) & 63;
     uint32_t it = 0;
     bool ok = true;
     for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
       int tile, b0, b1;
       item_range(item, tile, b0, b1);
       for (int sb = b0; sb < b1 && ok; ++sb, ++it) {
+        if ((it % D_CONV_GROUPS) != static_cast<uint32_t>(grp)) continue;
         const int ss = it % D_S_ST, s = it % D_S_OP;
         ok = mbar_wait(&st_full[ss], (it / D_S_ST) & 1, DSITE_ST_FULL_B, limit) &&
              mbar_wait(&empty[s], ((it / D_S_OP) & 1) ^ 1, DSITE_EMPTY_B, limit);
         if (!ok) break;
-        unpack_rows(smem + L::OFF_X_ST + ss * L::X_ST, smem + L::OFF_X_OP + s * L::X_OP, NT, t, D_B_WARPS * 32,
+        unpack_rows(smem + L::OFF_X_ST + ss * L::X_ST, smem + L::OFF_X_OP + s * L::X_OP, NT, t, 64,
                     2 * sb + 1 < num_kb);
         fence_proxy_async_smem();
         __syncwarp();
@@ -267,70 +287,101 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
       }
     }
   } else {
-    // ------------------------------ epilogue ----------------------------------------------------
+    // ------------------------------ epilogue groups -----------------------------------------------
     const int q = warp & 3;
-    const int et = threadIdx.x - (2 + D_A_WARPS + D_B_WARPS) * 32;   // 0 .. 127
-    uint32_t icount = 0;
+    const int eg = (warp - (2 + D_A_WARPS + D_B_WARPS)) >> 2;        // this group takes items eg, eg + 2, ...
+    const int et = (threadIdx.x - (2 + D_A_WARPS + D_B_WARPS) * 32) & 127;
+    const int rowl = q * 32 + lane;                                  // row of the tile = TMEM lane
     bool ok = true;
+    uint32_t icount = 0;
     for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++icount) {
+      if ((icount % D_EPI_GROUPS) != static_cast<uint32_t>(eg)) continue;
       int tile, b0, b1;
       item_range(item, tile, b0, b1);
-      const uint32_t acc = icount & 1;
-      ok = mbar_wait(&tmem_full[acc], (icount >> 1) & 1, DSITE_TMEM_FULL, limit);
+      const uint32_t acc = icount % D_ACCS;
+      ok = mbar_wait(&tmem_full[acc], (icount / D_ACCS) & 1, DSITE_TMEM_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
-      uint32_t r[NT];
       const uint32_t tmem_d = tmem_base + acc * NT + (static_cast<uint32_t>(q * 32) << 16);
+      const int ch = tile * 128 + rowl;                    // output channel of this thread
+      const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;
+      // Partial tiles are stored as [item][4-column chunk][row][4]: a warp's 16-byte accesses are contiguous.
+      int4* mine = reinterpret_cast<int4*>(partials) + static_cast<size_t>(item) * (NT / 4) * 128 + rowl;
 #pragma unroll
-      for (int c = 0; c < NT / 16; ++c) tmem_ld_32x32b_x16(tmem_d + 16 * c, *reinterpret_cast<uint32_t(*)[16]>(&r[16 * c]));
-      tmem_wait_ld();
-      tc_fence_before_sync();
-      __syncwarp();
-      if (lane == 0) mbar_arrive(&tmem_empty[acc]);
-      const int ch = tile * 128 + q * 32 + lane;           // output channel of this thread
-      int32_t a[NT];
-#pragma unroll
-      for (int e = 0; e < NT; ++e) a[e] = static_cast<int32_t>(r[e]) >> 8;   // exact: the accumulator is 256 * acc
-      bool finish = (splits == 1);
-      if (splits > 1) {
-        int32_t* mine = partials + (static_cast<size_t>(item) * 128 + q * 32 + lane) * NT;
-#pragma unroll
-        for (int e = 0; e < NT; e += 4) *reinterpret_cast<int4*>(mine + e) = make_int4(a[e], a[e + 1], a[e + 2], a[e + 3]);
-        __threadfence();
-        named_barrier(1, D_EPI_WARPS * 32);
-        if (et == 0) {
-          const unsigned int old = atomicAdd(&counters[tile], 1u);
-          *last_flag = (old == static_cast<unsigned int>(splits - 1)) ? 1u : 0u;
-          if (old == static_cast<unsigned int>(splits - 1)) counters[tile] = 0u;    // ready for the next call
+      for (int c16 = 0; c16 < NT / 16; ++c16) {
+        uint32_t r[16];
+        tmem_ld_32x32b_x16(tmem_d + 16 * c16, r);
+        tmem_wait_ld();
+        if (c16 == NT / 16 - 1) {                          // last read: hand the accumulator back
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&tmem_empty[acc]);
         }
-        named_barrier(1, D_EPI_WARPS * 32);
-        finish = (*last_flag != 0u);
-        if (finish) {
-          __threadfence();
+        if (splits == 1) {
 #pragma unroll
-          for (int e = 0; e < NT; ++e) a[e] = 0;
-          for (int sp = 0; sp < splits; ++sp) {            // fixed order: the sum does not depend on who finishes
-            const int32_t* p = partials + (static_cast<size_t>(tile * splits + sp) * 128 + q * 32 + lane) * NT;
+          for (int x = 0; x < 16; ++x) {
+            const int e = 16 * c16 + x;
+            if (e < M && ch < N) {
+              const int32_t a = static_cast<int32_t>(r[x]) >> 8;          // exact: the accumulator is 256 * acc
+              const float f = __int_as_float(0x4B400000 + a) - 12582912.0f;
+              Y[static_cast<size_t>(e) * N + ch] = __float2half_rn(f * (__half2float(__ldg(sx + e)) * swv));
+              if (accdbg) accdbg[static_cast<size_t>(e) * N + ch] = a;
+            }
+          }
+        } else {
 #pragma unroll
-            for (int e = 0; e < NT; e += 4) {
-              const int4 v = __ldcg(reinterpret_cast<const int4*>(p + e));
-              a[e] += v.x; a[e + 1] += v.y; a[e + 2] += v.z; a[e + 3] += v.w;
+          for (int c = 0; c < 4; ++c)
+            mine[(4 * c16 + c) * 128] =
+                make_int4(static_cast<int32_t>(r[4 * c]) >> 8, static_cast<int32_t>(r[4 * c + 1]) >> 8,
+                          static_cast<int32_t>(r[4 * c + 2]) >> 8, static_cast<int32_t>(r[4 * c + 3]) >> 8);
+        }
+      }
+      if (splits == 1) continue;
+      named_barrier(1 + eg, 128);                            // the group's stores happen before ...
+      if (et == 0) {
+        __threadfence();                                     // ... this fence, which orders them before the count
+        const unsigned int old = atomicAdd(&counters[tile], 1u);
+        const bool last = (old == static_cast<unsigned int>(splits - 1));
+        if (last) {
+          counters[tile] = 0u;                               // ready for the next call
+          __threadfence();                                   // the other items' partials are visible from here on
+        }
+        last_flag[eg] = last ? 1u : 0u;
+      }
+      named_barrier(1 + eg, 128);
+      const bool finish = (last_flag[eg] != 0u);
+      if (finish) {
+        // Sum the tile's partials in the fixed order sp = 0, 1, ...: the result does not depend on
+        // which item came last.  All loads of a chunk are issued before any is used.
+        const int4* base = reinterpret_cast<const int4*>(partials) + static_cast<size_t>(tile) * splits * (NT / 4) * 128 + rowl;
+#pragma unroll 1
+        for (int c = 0; c < NT / 4; ++c) {
+          int4 a = make_int4(0, 0, 0, 0);
+#pragma unroll
+          for (int h = 0; h < D_MAX_SPLITS; h += 8) {      // eight loads in flight at a time
+            if (h < splits) {
+              int4 v[8];
+#pragma unroll
+              for (int sp = 0; sp < 8; ++sp)
+                if (h + sp < splits) v[sp] = __ldcg(base + (static_cast<size_t>(h + sp) * (NT / 4) + c) * 128);
+#pragma unroll
+              for (int sp = 0; sp < 8; ++sp)
+                if (h + sp < splits) { a.x += v[sp].x; a.y += v[sp].y; a.z += v[sp].z; a.w += v[sp].w; }
+            }
+          }
+          const int32_t av[4] = {a.x, a.y, a.z, a.w};
+#pragma unroll
+          for (int x = 0; x < 4; ++x) {
+            const int e = 4 * c + x;
+            if (e < M && ch < N) {
+              const float f = __int_as_float(0x4B400000 + av[x]) - 12582912.0f;
+              Y[static_cast<size_t>(e) * N + ch] = __float2half_rn(f * (__half2float(__ldg(sx + e)) * swv));
+              if (accdbg) accdbg[static_cast<size_t>(e) * N + ch] = av[x];
             }
           }
         }
-        named_barrier(1, D_EPI_WARPS * 32);                // last_flag may be rewritten by the next item
       }
-      if (finish && ch < N) {
-        const float swv = __half2float(sw[ch]);
-#pragma unroll
-        for (int e = 0; e < NT; ++e) {
-          if (e < M) {
-            const float f = __int_as_float(0x4B400000 + a[e]) - 12582912.0f;
-            Y[static_cast<size_t>(e) * N + ch] = __float2half_rn(f * (__half2float(__ldg(sx + e)) * swv));
-            if (accdbg) accdbg[static_cast<size_t>(e) * N + ch] = a[e];
-          }
-        }
-      }
+      named_barrier(1 + eg, 128);                            // last_flag may be rewritten by the group's next item
     }
   }
 
