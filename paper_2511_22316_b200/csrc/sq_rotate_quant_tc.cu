@@ -36,6 +36,7 @@ namespace {
 constexpr float kFactorScale = 1024.0f;           // 2^10 applied to R1 and R2 in the images
 constexpr int kFactorScaleLog2 = 10;
 constexpr int kMaxDynSmem = 227 * 1024;
+constexpr int kHalfDynSmem = 113 * 1024;        // two CTAs per SM
 
 enum RqSite : uint32_t { RQ_X_EMPTY = 16, RQ_X_FULL, RQ_D_FREE, RQ_A2_READY, RQ_D1_FULL, RQ_D2_FULL, RQ_IMG };
 
@@ -48,7 +49,7 @@ struct RqLayout {
   int off_a1, off_b2, off_x, off_misc, total;
 };
 
-__host__ __device__ inline RqLayout rq_layout(int n1, int n2) {
+__host__ __device__ inline RqLayout rq_layout(int n1, int n2, int budget = kMaxDynSmem) {
   RqLayout L;
   L.LS = n1 <= 32 ? 32 : (n1 <= 64 ? 64 : 128);   // TMEM lanes per token
   L.G = 128 / L.LS;                               // tokens per accumulator
@@ -69,7 +70,7 @@ __host__ __device__ inline RqLayout rq_layout(int n1, int n2) {
   L.off_a1 = 0;
   L.off_b2 = L.off_a1 + L.a1_bytes;
   L.off_x = L.off_b2 + L.b2_bytes;
-  const int room = kMaxDynSmem - 1024 - 512 - L.off_x;
+  const int room = budget - 1024 - 512 - L.off_x;
   const int xs = room / L.x_bytes;
   L.XS = xs > 4 ? 4 : xs;                         // X ring depth
   L.off_misc = L.off_x + L.XS * L.x_bytes;
@@ -125,15 +126,17 @@ __device__ __forceinline__ float absmax32(const uint32_t (&r)[32]) {
   return fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
 }
 
-template <int N2>
-__global__ void __launch_bounds__((2 + 4 * (256 / N2)) * 32, 1)
+// S accumulator slots (= compute groups) per CTA.  With S * 2 * N2 = 256 TMEM columns two CTAs share
+// an SM (each with its own producer and MMA issuer); with 512 a CTA has the SM to itself.
+template <int N2, int S>
+__global__ void __launch_bounds__((2 + 4 * S) * 32, (S * 2 * N2 <= 256) ? 2 : 1)
 rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigned char* __restrict__ a1_img,
                        const unsigned char* __restrict__ b2_img, int n1, long long rows,
                        uint8_t* __restrict__ Xq, __half* __restrict__ scales, float* __restrict__ Zdbg) {
-  constexpr int S = 256 / N2;                    // accumulator slots = compute groups
+  constexpr int TM_COLS = S * 2 * N2;             // 256 or 512
   constexpr int XQ = N2 / 64;
   constexpr int SLOT_COLS = 2 * N2;              // D1 (N2 columns) + D2 (N2 columns)
-  const RqLayout L = rq_layout(n1, N2);
+  const RqLayout L = rq_layout(n1, N2, TM_COLS == 512 ? kMaxDynSmem : kHalfDynSmem);
   const int n = n1 * N2;
   const int G = L.G, LS = L.LS;
 
@@ -192,7 +195,7 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
       bulk_load_1d(b2s + o, b2_img + o, static_cast<uint32_t>(min(16384, L.b2_bytes - o)), img_full);
   }
   if (warp == 1) {
-    tmem_alloc(tmem_slot, 512);
+    tmem_alloc(tmem_slot, TM_COLS);
     tmem_relinquish();
   }
   tc_fence_before_sync();
@@ -402,7 +405,7 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
   __syncthreads();
   if (warp == 1) {
     tc_fence_after_sync();
-    tmem_dealloc(tmem_base, 512);
+    tmem_dealloc(tmem_base, TM_COLS);
   }
 }
 
@@ -466,7 +469,10 @@ bool rotate_quant_tc_prepare(sq_rotation* h) {
 sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
                                    float* Zdbg, cudaStream_t s) {
   const int n1 = h->n1, n2 = h->n2;
-  const RqLayout L = rq_layout(n1, n2);
+  // n2 = 64 with images small enough: two CTAs per SM, two accumulator slots each.
+  const RqLayout Lh = rq_layout(n1, n2, kHalfDynSmem);
+  const bool dual = (n2 == 64) && Lh.XS >= 2;
+  const RqLayout L = dual ? Lh : rq_layout(n1, n2);
   EncodeTiledFn enc = get_encode_fn();
   if (!enc) return SQ_ERR_CUDA;
   CUtensorMap mx;
@@ -480,31 +486,27 @@ sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t 
     return SQ_ERR_CUDA;
   const int sms = sm_count();
   if (sms <= 0) return SQ_ERR_CUDA;
-  // More than half of an SM's shared memory, so that two CTAs (each wanting all of TMEM) never share one.
-  const int smem = std::max(L.total + 1024, 120 * 1024);
   const long long ngroups = (rows + L.G - 1) / L.G;
-  const unsigned grid = static_cast<unsigned>(std::min<long long>(ngroups, sms));
   const unsigned char* a1 = static_cast<const unsigned char*>(h->dA1img);
   const unsigned char* b2 = static_cast<const unsigned char*>(h->dB2img);
-  if (n2 == 64) {
-    auto kern = rotate_quant_tc_kernel<64>;
-    static int smem_set = 0;                      // largest size the attribute has been raised to
+  auto launch = [&](auto kern, int slots, int ctas_per_sm, int& smem_set) -> bool {
+    // A CTA that wants all of TMEM asks for more than half of the shared memory, so that it is alone.
+    const int smem = ctas_per_sm == 1 ? std::max(L.total + 1024, 120 * 1024) : L.total + 1024;
     if (smem > smem_set) {
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SQ_ERR_CUDA;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
       smem_set = smem;
     }
-    kern<<<grid, (2 + 4 * 4) * 32, smem, s>>>(mx, a1, b2, n1, rows, static_cast<uint8_t*>(Xq),
-                                              static_cast<__half*>(scales), Zdbg);
-  } else {
-    auto kern = rotate_quant_tc_kernel<128>;
-    static int smem_set = 0;
-    if (smem > smem_set) {
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SQ_ERR_CUDA;
-      smem_set = smem;
-    }
-    kern<<<grid, (2 + 4 * 2) * 32, smem, s>>>(mx, a1, b2, n1, rows, static_cast<uint8_t*>(Xq),
-                                              static_cast<__half*>(scales), Zdbg);
-  }
+    const unsigned grid = static_cast<unsigned>(std::min<long long>(ngroups, static_cast<long long>(sms) * ctas_per_sm));
+    kern<<<grid, (2 + 4 * slots) * 32, smem, s>>>(mx, a1, b2, n1, rows, static_cast<uint8_t*>(Xq),
+                                                  static_cast<__half*>(scales), Zdbg);
+    return true;
+  };
+  static int set_64_2 = 0, set_64_4 = 0, set_128_2 = 0;     // largest shared-memory size set per kernel
+  bool ok;
+  if (n2 == 64 && dual) ok = launch(rotate_quant_tc_kernel<64, 2>, 2, 2, set_64_2);
+  else if (n2 == 64) ok = launch(rotate_quant_tc_kernel<64, 4>, 4, 1, set_64_4);
+  else ok = launch(rotate_quant_tc_kernel<128, 2>, 2, 1, set_128_2);
+  if (!ok) return SQ_ERR_CUDA;
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
 }
