@@ -3,6 +3,7 @@
 #include "sq_gemm.cu"
 #include "sq_gemm_pair.cu"
 #include "sq_gemm_decode.cu"
+#include "sq_gemv.cu"
 #include "sq_rotate_quant.cu"
 #include "sq_rotate_quant_tc.cu"
 #include "sq_rotate_quant_pair.cu"

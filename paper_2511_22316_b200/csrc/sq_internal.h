@@ -72,6 +72,11 @@ size_t gemm_decode_workspace_bytes(int64_t M, int64_t N, int64_t K);
 sq_status_t launch_w4a4_gemm_decode(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N, int K,
                                     void* Y, int32_t* accdbg, void* workspace, size_t workspace_bytes, cudaStream_t s);
 
+// Step 3 for one to four tokens (sq_gemv.cu): dot products on the CUDA cores.
+bool gemv_supported(int64_t M, int64_t N, int64_t K);
+sq_status_t launch_w4a4_gemv(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N, int K,
+                             void* Y, int32_t* accdbg, cudaStream_t s);
+
 // Device status word helpers (sq_api.cu).
 sq_status_t read_and_clear_device_status(cudaStream_t s);
 

@@ -246,6 +246,8 @@ GEMM_SHAPES = [
     (513, 2304, 2176),
     # decode kernel (M <= 64, weights as the A operand, split K): all three token-count classes,
     # ragged channel tile, odd k-block count, the two decode layer shapes
+    # dot-product kernel (M <= 4): odd channel counts, every token-count class
+    (2, 1001, 2048), (3, 264, 14336), (4, 7, 96),
     (1, 4096, 4096), (17, 1000, 2048), (33, 384, 1664), (64, 2048, 2304), (4, 14336, 4096), (16, 4096, 14336),
 ]
 
