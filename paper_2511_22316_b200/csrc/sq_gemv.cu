@@ -15,8 +15,9 @@
 namespace sq {
 namespace {
 
-constexpr int GV_ROWS = 2;            // weight rows per warp task
 constexpr int GV_UNROLL = 4;          // 16-byte pieces of each row in flight per lane
+// Weight rows per warp task: four for one or two tokens (more bytes in flight per lane), two for four.
+template <int MT> struct GvRows { static constexpr int value = MT <= 2 ? 4 : 2; };
 
 __device__ __forceinline__ int dp4a_s8(uint32_t a, uint32_t b, int c) {
   int d;
@@ -32,13 +33,31 @@ w4a4_gemv_kernel(const uint8_t* __restrict__ Xq, const __half* __restrict__ sx, 
                  const __half* __restrict__ sw, int M, int N, int K, __half* __restrict__ Y,
                  int32_t* __restrict__ accdbg) {
   extern __shared__ __align__(16) uint32_t xs[];
+  constexpr int GV_ROWS = GvRows<MT>::value;
   const int kw = K / 8;                                  // packed words per row
   const int nchunk = K / 32;                             // 16-byte pieces per row
-  for (int i = threadIdx.x; i < MT * kw; i += blockDim.x) {
-    const int t = i / kw, j = i % kw;
-    const uint32_t w = (t < M) ? __ldg(reinterpret_cast<const uint32_t*>(Xq + static_cast<size_t>(t) * (K / 2)) + j) : 0u;
-    xs[(0 * MT + t) * kw + j] = (w << 4) & 0xF0F0F0F0u;
-    xs[(1 * MT + t) * kw + j] = w & 0xF0F0F0F0u;
+  // tokens -> shared memory, four 16-byte pieces per thread in flight
+  for (int i0 = threadIdx.x; i0 < MT * nchunk; i0 += 4 * blockDim.x) {
+    uint4 w[4];
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * blockDim.x;
+      const int t = i / nchunk, c = i % nchunk;
+      w[u] = (i < MT * nchunk && t < M) ? __ldg(reinterpret_cast<const uint4*>(Xq + static_cast<size_t>(t) * (K / 2)) + c)
+                                        : make_uint4(0u, 0u, 0u, 0u);
+    }
+#pragma unroll
+    for (int u = 0; u < 4; ++u) {
+      const int i = i0 + u * blockDim.x;
+      if (i < MT * nchunk) {
+        const int t = i / nchunk, c = i % nchunk;
+        *reinterpret_cast<uint4*>(xs + (0 * MT + t) * kw + 4 * c) =
+            make_uint4((w[u].x << 4) & 0xF0F0F0F0u, (w[u].y << 4) & 0xF0F0F0F0u, (w[u].z << 4) & 0xF0F0F0F0u,
+                       (w[u].w << 4) & 0xF0F0F0F0u);
+        *reinterpret_cast<uint4*>(xs + (1 * MT + t) * kw + 4 * c) =
+            make_uint4(w[u].x & 0xF0F0F0F0u, w[u].y & 0xF0F0F0F0u, w[u].z & 0xF0F0F0F0u, w[u].w & 0xF0F0F0F0u);
+      }
+    }
   }
   __syncthreads();
 
@@ -116,11 +135,11 @@ w4a4_gemv_kernel(const uint8_t* __restrict__ Xq, const __half* __restrict__ sx, 
   }
 }
 
-// Warps per CTA such that N / GV_ROWS tasks fill sms * warps warps as evenly as possible.
+// Warps per CTA such that the tasks fill sms * warps warps as evenly as possible.
 int gemv_warps(long long ntask, int sms) {
-  int best = 8;
+  int best = 16;
   double best_eff = 0.0;
-  for (int w = 8; w <= 16; ++w) {
+  for (int w = 16; w >= 8; --w) {                        // more warps = more bytes in flight: prefer many
     const long long total = static_cast<long long>(sms) * w;
     const long long waves = (ntask + total - 1) / total;
     const double eff = static_cast<double>(ntask) / static_cast<double>(waves * total);
@@ -137,6 +156,7 @@ sq_status_t launch_gemv(const void* Xq, const void* sx, const void* Wq, const vo
                         int32_t* accdbg, cudaStream_t s) {
   const int sms = sm_count();
   if (sms <= 0) return SQ_ERR_CUDA;
+  constexpr int GV_ROWS = GvRows<MT>::value;
   const long long ntask = (N + GV_ROWS - 1) / GV_ROWS;
   const int warps = gemv_warps(ntask, sms);
   const int smem = MT * K;                               // 2 * MT * (K / 8) words
