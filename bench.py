@@ -75,6 +75,8 @@ def gemm_bytes(w):
 def gemm_kernel_name(w):
     """The kernel sq_w4a4_gemm picks for this shape (mirrors the library's dispatch)."""
     fast = w.K % 128 == 0 and w.N % 8 == 0
+    if w.M <= 4 and w.K % 32 == 0 and w.K <= 32768:
+        return "w4a4_gemv_kernel"
     if fast and w.M <= 64 and w.N >= 128 and w.K >= 256:
         return "w4a4_gemm_decode_kernel"
     if fast and w.M > 128 and w.N >= 128:
@@ -323,31 +325,46 @@ def run_ours(args, w):
     rq_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
     gemm_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
 
-    # ---- the same steps replayed from a CUDA graph (launch overhead taken out; informative) ------
-    graph_ms = None
-    try:
-        gsteps = min(args.steps, 4 * nsets)
-        gstream = torch.cuda.Stream()
-        gstream.wait_stream(torch.cuda.current_stream())
-        graph = torch.cuda.CUDAGraph()
-        with torch.cuda.stream(gstream):
-            with torch.cuda.graph(graph, stream=gstream):
-                for i in range(gsteps):
-                    step(i)
-            graph.replay()
-            gstream.synchronize()
-            g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-            g0.record(gstream)
-            for _ in range(5):
+    # ---- the same calls replayed from CUDA graphs: launch overhead taken out.  Short kernels
+    # (decode shapes) are launch-bound when issued one by one, so the per-kernel figures below
+    # come from graphs of back-to-back launches when capture works, else from the events above.
+    def graph_time(fn, count):
+        try:
+            gstream = torch.cuda.Stream()
+            gstream.wait_stream(torch.cuda.current_stream())
+            graph = torch.cuda.CUDAGraph()
+            with torch.cuda.stream(gstream):
+                with torch.cuda.graph(graph, stream=gstream):
+                    for i in range(count):
+                        fn(i)
                 graph.replay()
-            g1.record(gstream)
-            gstream.synchronize()
-            graph_ms = g0.elapsed_time(g1) / (5 * gsteps)
-        torch.cuda.current_stream().wait_stream(gstream)
-    except Exception as exc:           # capture is optional: the timed region above stands on its own
-        graph_ms = None
-        sys.stderr.write(f"graph replay skipped: {exc}\n")
-    torch.cuda.synchronize()
+                gstream.synchronize()
+                g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+                g0.record(gstream)
+                for _ in range(5):
+                    graph.replay()
+                g1.record(gstream)
+                gstream.synchronize()
+                ms = g0.elapsed_time(g1) / (5 * count)
+            torch.cuda.current_stream().wait_stream(gstream)
+            torch.cuda.synchronize()
+            return ms
+        except Exception as exc:       # capture is optional: the event timings stand on their own
+            sys.stderr.write(f"graph replay skipped: {exc}\n")
+            torch.cuda.synchronize()
+            return None
+
+    gsteps = min(args.steps, 4 * nsets)
+    graph_ms = graph_time(step, gsteps)
+    rq_graph = graph_time(lambda i: sq.sq_rotate_quant_act(rot, sets[i % nsets]["X"], M, sets[i % nsets]["Xq"],
+                                                           sets[i % nsets]["sx"]), gsteps)
+    gemm_graph = graph_time(lambda i: sq.sq_w4a4_gemm(sets[i % nsets]["Xq"], sets[i % nsets]["sx"], sets[i % nsets]["Wq"],
+                                                      sets[i % nsets]["sw"], M, N, K, sets[i % nsets]["Y"], None,
+                                                      gws if gws_bytes else None, gws_bytes), gsteps)
+    kernel_timing = "cuda events around single launches"
+    if rq_graph is not None and gemm_graph is not None:
+        rq_ms, gemm_ms = rq_graph, gemm_graph
+        kernel_timing = "cuda events around graph replays of back-to-back launches"
 
     # ---- end to end: host activations in, host outputs out, through sq_linear_host ------------
     hws_bytes = sq.sq_linear_host_workspace_bytes(M, N, K)
@@ -429,7 +446,7 @@ def run_ours(args, w):
             "roofline": dominant,
             "roofline_other": other,
             "kernel_ms": {"rotate_quant": rq_ms, "w4a4_gemm": gemm_ms, "sum": rq_ms + gemm_ms,
-                          "step": ms_per_step, "step_graph_replay": graph_ms},
+                          "step": ms_per_step, "step_graph_replay": graph_ms, "how": kernel_timing},
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": M * K * 2,
                     "d2h_bytes_per_step": M * N * 2, "api": "sq_linear_host (pinned host X -> host Y)"},
             "gpu_launches": int(launches),
