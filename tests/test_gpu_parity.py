@@ -155,6 +155,16 @@ def test_rotate_quant_70b_shapes_sampled_rows(sq, w):
     check_rotate_quant(sq, X, R1, R2, rows=rows)
 
 
+def test_rotate_quant_many_short_rows(sq):
+    """More token rows than 16 bits can index, four tokens per accumulator, a ragged last group."""
+    w = wl.small("many", 70001, 8, 64, 8, 77)
+    X = wl.make_activations(w)
+    R1, R2 = ora.build_rotation(X.astype(np.float32), w.n1, w.n2)
+    rng = np.random.default_rng(2)
+    rows = np.unique(np.concatenate([[0, 1, 2, 3, 65535, 65536, 69999, 70000], rng.integers(0, w.M, size=120)]))
+    check_rotate_quant(sq, X, R1, R2, rows=rows)
+
+
 def test_quantiser_is_bit_exact_under_identity_rotation(sq):
     """With R1 = R2 = I the rotated row equals the fp16 input exactly, so codes and steps must
     match the oracle's fp32-decision quantiser bit for bit (both the rotating kernel with
@@ -278,6 +288,25 @@ def test_gemm_extreme_codes_do_not_overflow(sq):
     Y, acc = run_gemm(sq, Xc, Wc, sx, sw)
     assert np.all(acc[:, 0] == 64 * K) and np.all(acc[:, 1] == -56 * K)
     assert np.array_equal(acc, ora.gemm_i32(Xc, Wc))
+
+
+@pytest.mark.parametrize("M,N", [(2, 8), (3, 136), (40, 256), (100, 128), (130, 128)])
+def test_gemm_largest_k_and_largest_accumulator(sq, M, N):
+    """K = 65536 is the largest supported contraction; with every code at -8 the accumulator reaches
+    64 K = 2^22, the top of the range the exact int -> float step of the epilogues is built for."""
+    K = 65536
+    rng = np.random.default_rng(M * 31 + N)
+    Xc, Wc = random_codes(rng, M, K), random_codes(rng, N, K)
+    Xc[0] = -8
+    Wc[0] = -8
+    Wc[N - 1] = 7
+    sx = np.full(M, 2.0 ** -12, np.float16)
+    sw = np.full(N, 2.0 ** -12, np.float16)
+    Y, acc = run_gemm(sq, Xc, Wc, sx, sw)
+    acc_o = ora.gemm_i32(Xc, Wc)
+    assert acc_o[0, 0] == 64 * K and acc_o[0, N - 1] == -56 * K
+    assert np.array_equal(acc, acc_o)
+    assert np.array_equal(Y.view(np.uint16), ora.dequant(acc_o, sx, sw).view(np.uint16))
 
 
 def test_gemm_prefill_config_sampled_rows(sq):
