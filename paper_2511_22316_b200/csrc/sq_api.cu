@@ -8,6 +8,7 @@
 
 namespace sq {
 std::atomic<uint64_t> g_launches{0};
+thread_local bool g_pdl_next = false;
 
 int sm_count() {
   static std::atomic<int> cache[64];
@@ -241,7 +242,11 @@ sq_status_t sq_linear(const sq_rotation_t* rot, const void* X, int64_t M, const 
   const size_t gws_bytes = sq::gemm_workspace_bytes(M, N, K);
   sq_status_t st = sq_rotate_quant_act(rot, X, M, Xq, sx, nullptr, stream);
   if (st != SQ_OK) return st;
-  return sq_w4a4_gemm(Xq, sx, Wq, sw, M, N, K, Y, nullptr, gws_bytes ? gws : nullptr, gws_bytes, stream);
+  // The split-K decode kernel is preceded by a memset of its counters, so it is launched normally.
+  sq::g_pdl_next = sq::gemv_supported(M, N, K) || !sq::gemm_decode_supported(M, N, K);
+  st = sq_w4a4_gemm(Xq, sx, Wq, sw, M, N, K, Y, nullptr, gws_bytes ? gws : nullptr, gws_bytes, stream);
+  sq::g_pdl_next = false;
+  return st;
 }
 
 // Workspace layout of sq_linear_host: [X: 2*M*K][Y: 2*M*N][sq_linear workspace].

@@ -166,6 +166,7 @@ w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
   __syncthreads();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();                                     // Xq and sx may come from the kernel launched before this one
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------------------
@@ -365,11 +366,11 @@ sq_status_t launch_tc(const void* Xq, const void* sx, const void* Wq, const void
   if (sms <= 0) return SQ_ERR_CUDA;
   const int tiles = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);
   const int grid = tiles < sms ? tiles : sms;
-  kern<<<grid, GEMM_THREADS, L::DYN_BYTES, s>>>(mx, mw, static_cast<const __half*>(sx),
-                                                static_cast<const __half*>(sw), M, N, K, static_cast<__half*>(Y),
-                                                accdbg);
+  const cudaError_t err = launch_maybe_pdl(kern, dim3(grid), dim3(GEMM_THREADS), L::DYN_BYTES, s, mx, mw,
+                                           static_cast<const __half*>(sx), static_cast<const __half*>(sw), M, N, K,
+                                           static_cast<__half*>(Y), accdbg);
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
 }
 
 }  // namespace

@@ -123,6 +123,7 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   __syncthreads();
   cluster_sync_all();                                 // both CTAs' barriers exist before any remote arrival
   tc_fence_after_sync();
+  griddep_wait();                                     // Xq and sx may come from the kernel launched before this one
   const uint32_t tmem_base = *tmem_slot;
 
   if (warp == 0) {
@@ -337,11 +338,11 @@ sq_status_t launch_w4a4_gemm_pair(const void* Xq, const void* sx, const void* Wq
   if (sms <= 0) return SQ_ERR_CUDA;
   const int tiles = ((N + P_TILE_N - 1) / P_TILE_N) * ((M + P_TILE_M - 1) / P_TILE_M);
   const int pairs = tiles < sms / 2 ? tiles : sms / 2;
-  kern<<<2 * pairs, P_THREADS, L::DYN_BYTES, s>>>(mx, mw, my, static_cast<const __half*>(sx),
-                                                  static_cast<const __half*>(sw), M, N, K,
-                                                  static_cast<__half*>(Y), accdbg);
+  const cudaError_t err = launch_maybe_pdl(kern, dim3(2 * pairs), dim3(P_THREADS), L::DYN_BYTES, s, mx, mw, my,
+                                           static_cast<const __half*>(sx), static_cast<const __half*>(sw), M, N, K,
+                                           static_cast<__half*>(Y), accdbg);
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
 }
 
 }  // namespace sq

@@ -11,6 +11,7 @@
 #include <cuda_fp16.h>
 
 #include "sq_internal.h"
+#include "sq_ptx.cuh"
 
 namespace sq {
 namespace {
@@ -32,6 +33,7 @@ __global__ void __launch_bounds__(512)
 w4a4_gemv_kernel(const uint8_t* __restrict__ Xq, const __half* __restrict__ sx, const uint8_t* __restrict__ Wq,
                  const __half* __restrict__ sw, int M, int N, int K, __half* __restrict__ Y,
                  int32_t* __restrict__ accdbg) {
+  griddep_wait();                                        // Xq and sx may come from the kernel launched before this one
   extern __shared__ __align__(16) uint32_t xs[];
   constexpr int GV_ROWS = GvRows<MT>::value;
   const int kw = K / 8;                                  // packed words per row
@@ -167,11 +169,12 @@ sq_status_t launch_gemv(const void* Xq, const void* sx, const void* Wq, const vo
     smem_set = smem;
   }
   const unsigned grid = static_cast<unsigned>(std::min<long long>(sms, (ntask + warps - 1) / warps));
-  kern<<<grid, warps * 32, smem, s>>>(static_cast<const uint8_t*>(Xq), static_cast<const __half*>(sx),
-                                      static_cast<const uint8_t*>(Wq), static_cast<const __half*>(sw), M, N, K,
-                                      static_cast<__half*>(Y), accdbg);
+  const cudaError_t err = launch_maybe_pdl(kern, dim3(grid), dim3(warps * 32), static_cast<size_t>(smem), s,
+                                           static_cast<const uint8_t*>(Xq), static_cast<const __half*>(sx),
+                                           static_cast<const uint8_t*>(Wq), static_cast<const __half*>(sw), M, N, K,
+                                           static_cast<__half*>(Y), accdbg);
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
 }
 
 }  // namespace

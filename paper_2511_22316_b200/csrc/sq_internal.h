@@ -4,6 +4,7 @@
 #include <stdint.h>
 
 #include <atomic>
+#include <utility>
 #include <vector>
 
 #include "../../include/singlequant.h"
@@ -29,6 +30,26 @@ inline void count_launch(uint64_t k = 1) { g_launches.fetch_add(k, std::memory_o
 
 // Multiprocessor count of the current device (cached per device; <= 0 on failure).
 int sm_count();
+
+// Set by sq_linear around its GEMM launch: the GEMM may then start while the rotate+quant kernel
+// before it in the stream is still running (it waits on the device before reading Xq and sx).
+extern thread_local bool g_pdl_next;
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_maybe_pdl(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                    Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = g_pdl_next ? 1 : 0;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 

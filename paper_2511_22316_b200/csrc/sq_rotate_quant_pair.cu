@@ -77,6 +77,7 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
                          uint8_t* __restrict__ Xq, __half* __restrict__ scales, float* __restrict__ Zdbg) {
   constexpr int S = 256 / N2;
   constexpr int SLOT_COLS = 2 * N2;
+  griddep_launch_dependents();                   // a GEMM launched behind this kernel may set itself up
   const RqPairLayout L = rq_pair_layout(n1, N2);
   const int n = n1 * N2;
 

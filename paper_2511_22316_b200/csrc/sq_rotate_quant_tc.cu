@@ -134,6 +134,7 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
                        const unsigned char* __restrict__ b2_img, int n1, long long rows,
                        uint8_t* __restrict__ Xq, __half* __restrict__ scales, float* __restrict__ Zdbg) {
   constexpr int TM_COLS = S * 2 * N2;             // 256 or 512
+  griddep_launch_dependents();                   // a GEMM launched behind this kernel may set itself up
   constexpr int XQ = N2 / 64;
   constexpr int SLOT_COLS = 2 * N2;              // D1 (N2 columns) + D2 (N2 columns)
   const RqLayout L = rq_layout(n1, N2, TM_COLS == 512 ? kMaxDynSmem : kHalfDynSmem);
