@@ -104,10 +104,16 @@ def _ptr(t) -> Optional[int]:
     return t.data_ptr()
 
 
+_torch = None
+
+
 def _stream(stream) -> Optional[int]:
     if stream is None:
-        import torch
-        return torch.cuda.current_stream().cuda_stream or None
+        global _torch
+        if _torch is None:
+            import torch
+            _torch = torch
+        return _torch.cuda.current_stream().cuda_stream or None
     if isinstance(stream, int):
         return stream or None
     return stream.cuda_stream or None
