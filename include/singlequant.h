@@ -56,6 +56,11 @@ typedef struct sq_rotation sq_rotation_t;   /* opaque: host + device copies of R
 /* Components of R = (R1^U R^A)^T (x) (H R2^U); a cleared bit replaces that component by the
  * identity (the paper's ablation of ART and URT). */
 enum { SQ_ROT_ART = 1, SQ_ROT_URT = 2, SQ_ROT_HADAMARD = 4, SQ_ROT_DEFAULT = 7 };
+/* Repeated ART rotations (paragraph "Effect of ART Steps"): OR this into `flags` to apply k >= 1
+ * ART steps (k <= 2048); each step after the first is the closed-form Givens rotation of Lemma 1
+ * in the plane (outlier, minimum) of the column as rotated so far.  The paper finds one step
+ * sufficient; the default is one. */
+#define SQ_ROT_ART_STEPS(k) ((uint32_t)((k) - 1) << 8)
 
 /* Algorithm 1 (Kronecker Dimension Factorization).  Host only.  n2 = the power of two dividing
  * n closest to sqrt(n), the first found winning ties; n1 = n / n2.  n >= 1. */

@@ -95,14 +95,23 @@ def haar_orthogonal(m: int, rng: np.random.Generator) -> np.ndarray:
 
 def art_indices(c: np.ndarray) -> Tuple[int, int]:
     """ART paragraph: i = dimension of the outlier (largest |c|), j = dimension of the minimum
-    value, read as the smallest magnitude among the others; ties go to the lowest index."""
+    value, read as the smallest magnitude among the others; ties go to the lowest index.
+    Magnitudes within a relative 1e-9 of each other count as tied: after an ART step two entries
+    are equal in exact arithmetic, and rounding must not decide which of them is "the" outlier."""
     n = c.shape[0]
-    i = int(np.argmax(np.abs(c)))
+    mag = np.abs(np.asarray(c, dtype=np.float64))
+    i = 0
+    for k in range(1, n):
+        if mag[k] > mag[i] * (1.0 + 1e-9):
+            i = k
     if n < 2:
         return i, i
-    mag = np.abs(c).astype(np.float64).copy()
-    mag[i] = np.inf
-    j = int(np.argmin(mag))
+    j = -1
+    for k in range(n):
+        if k == i:
+            continue
+        if j < 0 or mag[k] < mag[j] * (1.0 - 1e-9):
+            j = k
     return i, j
 
 
@@ -136,6 +145,36 @@ def art_matrix(c: np.ndarray, O: Optional[np.ndarray]) -> np.ndarray:
     return D @ P
 
 
+def art_repeat_step(c: np.ndarray) -> np.ndarray:
+    """One further ART step ("Effect of ART Steps": repeated ART rotations): the plane rotation in
+    coordinates (i, j) = (outlier, minimum) of the CURRENT column c that sends (c_i, c_j) to
+    (r, r)/sqrt(2) (Lemma 1) and leaves every other coordinate alone.  The paper does not say how
+    a repeated step treats the permutation and the random block of the first one; this reading
+    repeats only the closed-form Givens rotation, which is what its ablation varies."""
+    c = np.asarray(c, dtype=np.float64)
+    n = c.shape[0]
+    M = np.eye(n, dtype=np.float64)
+    if n < 2:
+        return M
+    i, j = art_indices(c)
+    a, b = float(c[i]), float(c[j])
+    if a == 0.0 and b == 0.0:
+        return M
+    th = equalizing_angle(a, b)
+    cs, sn = math.cos(th), math.sin(th)
+    M[i, i], M[i, j], M[j, i], M[j, j] = cs, sn, -sn, cs
+    return M
+
+
+def art_matrix_steps(c: np.ndarray, O: Optional[np.ndarray], steps: int) -> np.ndarray:
+    """R^A for `steps` >= 1 ART steps: the first is art_matrix, each further one art_repeat_step
+    on the column as rotated so far."""
+    RA = art_matrix(c, O)
+    for _ in range(steps - 1):
+        RA = art_repeat_step(RA @ np.asarray(c, dtype=np.float64)) @ RA
+    return RA
+
+
 # --------------------------------------------------------------------------------------
 # URT: uniformity rotation (normal outliers)
 # --------------------------------------------------------------------------------------
@@ -159,7 +198,9 @@ def map_to_e1(V: np.ndarray) -> Tuple[np.ndarray, int]:
 
 def uniform_target(V: np.ndarray) -> np.ndarray:
     """U of the URT paragraph: q_k = (2k - n - 1)/n for k = 1..n, assigned by the rank order
-    of V (stable ascending sort pi) and scaled so that ||U|| = ||V||."""
+    of V (stable ascending sort pi) and scaled so that ||U|| = ||V||.  Entries closer than
+    1e-9 max|V| count as equal and keep their index order (after ART two entries of the column
+    are equal in exact arithmetic; rounding must not decide their rank)."""
     V = np.asarray(V, dtype=np.float64)
     n = V.shape[0]
     k = np.arange(1, n + 1, dtype=np.float64)
@@ -168,7 +209,9 @@ def uniform_target(V: np.ndarray) -> np.ndarray:
     U = np.zeros(n, dtype=np.float64)
     if qn == 0.0:
         return U
-    pi = np.argsort(V, kind="stable")
+    vmax = float(np.max(np.abs(V)))
+    keys = np.rint(V / (1e-9 * vmax)) if vmax > 0.0 else np.zeros(n)
+    pi = np.argsort(keys, kind="stable")
     U[pi] = np.linalg.norm(V) / qn * q
     return U
 
@@ -201,7 +244,7 @@ def hadamard(n: int) -> np.ndarray:
 # --------------------------------------------------------------------------------------
 def build_rotation(calib: np.ndarray, n1: int, n2: int, flags: int = ROT_DEFAULT,
                    O: Optional[np.ndarray] = None, seed: int = 0,
-                   return_f64: bool = False):
+                   return_f64: bool = False, art_steps: int = 1):
     """Paragraph "The Overall SingleQuant Method": R1 = (R1^U R^A)^T, R2 = H R2^U.
 
     The paper builds ART/URT "according to" the activation X without saying which vectors; the
@@ -213,7 +256,8 @@ def build_rotation(calib: np.ndarray, n1: int, n2: int, flags: int = ROT_DEFAULT
          L = (R^U)^T R^A is R1^T; R1 = L^T.
       4. A' = L A; r = the row of A' with the largest |entry|; R2^U = URT for the row r H;
          R2 = H R2^U.
-    `flags` switches components to the identity (the paper's ablation of ART / URT).
+    `flags` switches components to the identity (the paper's ablation of ART / URT);
+    `art_steps` > 1 repeats the ART rotation (the paper's ablation of ART steps).
     Factors are built in float64 and returned rounded to float32 (the stored precision);
     with return_f64 the unrounded pair is returned as well."""
     calib = np.asarray(calib, dtype=np.float64)
@@ -230,7 +274,7 @@ def build_rotation(calib: np.ndarray, n1: int, n2: int, flags: int = ROT_DEFAULT
     if flags & ROT_ART:
         if O is None and n1 > 2:
             O = haar_orthogonal(n1 - 2, np.random.default_rng(seed))
-        RA = art_matrix(c, O)
+        RA = art_matrix_steps(c, O, art_steps)
     else:
         RA = np.eye(n1)
     c_prime = RA @ c

@@ -156,6 +156,11 @@ def sq_factorize(n: int) -> Tuple[int, int]:
     return a.value, b.value
 
 
+def SQ_ROT_ART_STEPS(k: int) -> int:
+    """Flag bits for k >= 1 ART steps (OR into `flags`)."""
+    return (int(k) - 1) << 8
+
+
 def sq_build_rotation(calib: np.ndarray, n1: int, n2: int, flags: int = SQ_ROT_DEFAULT, seed: int = 0,
                       O: Optional[np.ndarray] = None) -> Rotation:
     calib = np.ascontiguousarray(calib, dtype=np.float32)

@@ -136,7 +136,7 @@ sq_status_t sq_build_rotation(const float* calib, int64_t T, int64_t n, int32_t 
                               uint64_t seed, const double* O_or_null, sq_rotation_t** out) {
   if (!out) return SQ_ERR_INVALID_ARG;
   *out = nullptr;
-  if (!calib || T < 1 || n1 < 1 || n2 < 1 || (flags & ~7u)) return SQ_ERR_INVALID_ARG;
+  if (!calib || T < 1 || n1 < 1 || n2 < 1 || (flags & ~(7u | (0x7FFu << 8)))) return SQ_ERR_INVALID_ARG;
   if (static_cast<int64_t>(n1) * n2 != n) return SQ_ERR_SHAPE;
   if ((flags & SQ_ROT_HADAMARD) && (n2 & (n2 - 1)) != 0) return SQ_ERR_SHAPE;
   if (n1 > 4096 || n2 > 4096) return SQ_ERR_UNSUPPORTED;

@@ -76,7 +76,12 @@ Mat urt(const std::vector<double>& v) {
   if (n < 2 || !any) return identity(n);
   std::vector<int> order(n);
   std::iota(order.begin(), order.end(), 0);
-  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return v[a] < v[b]; });
+  // entries closer than 1e-9 max|v| count as equal and keep their index order
+  double vmax = 0.0;
+  for (double x : v) vmax = std::max(vmax, std::fabs(x));
+  std::vector<double> key(n);
+  for (int k = 0; k < n; ++k) key[k] = std::nearbyint(v[k] / (1e-9 * vmax));
+  std::stable_sort(order.begin(), order.end(), [&](int a, int b) { return key[a] < key[b]; });
   double vnorm2 = 0.0, qnorm2 = 0.0;
   for (double x : v) vnorm2 += x * x;
   std::vector<double> q(n);
@@ -92,18 +97,27 @@ Mat urt(const std::vector<double>& v) {
   return matmul(Rv, transpose(Ru, n), n);
 }
 
+// The (outlier, minimum) pair of ART: largest and smallest magnitude, ties to the lowest index.
+// Magnitudes within a relative 1e-9 count as tied (after an ART step two entries are equal in exact
+// arithmetic; rounding must not pick between them).
+void art_pair(const std::vector<double>& c, int& i, int& j) {
+  const int n = static_cast<int>(c.size());
+  i = 0;
+  for (int k = 1; k < n; ++k)
+    if (std::fabs(c[k]) > std::fabs(c[i]) * (1.0 + 1e-9)) i = k;
+  j = -1;
+  for (int k = 0; k < n; ++k) {
+    if (k == i) continue;
+    if (j < 0 || std::fabs(c[k]) < std::fabs(c[j]) * (1.0 - 1e-9)) j = k;
+  }
+}
+
 // ART matrix acting on the left of the column c: diag(G2, O) P_ij.
 Mat art(const std::vector<double>& c, const double* O) {
   const int n = static_cast<int>(c.size());
   if (n < 2) return identity(n);
-  int i = 0;
-  for (int k = 1; k < n; ++k)
-    if (std::fabs(c[k]) > std::fabs(c[i])) i = k;
-  int j = -1;
-  for (int k = 0; k < n; ++k) {
-    if (k == i) continue;
-    if (j < 0 || std::fabs(c[k]) < std::fabs(c[j])) j = k;
-  }
+  int i, j;
+  art_pair(c, i, j);
   std::vector<int> order;
   order.reserve(n);
   order.push_back(i);
@@ -132,6 +146,25 @@ Mat art(const std::vector<double>& c, const double* O) {
   for (int r = 0; r < n; ++r)
     for (int k = 0; k < n; ++k) RA[static_cast<size_t>(r) * n + order[k]] = D[static_cast<size_t>(r) * n + k];
   return RA;
+}
+
+// One further ART step: the plane rotation in coordinates (outlier, minimum) of the current column
+// that equalises the two (Lemma 1); every other coordinate is left alone.
+Mat art_repeat_step(const std::vector<double>& c) {
+  const int n = static_cast<int>(c.size());
+  Mat M = identity(n);
+  if (n < 2) return M;
+  int i, j;
+  art_pair(c, i, j);
+  const double a = c[i], b = c[j];
+  if (a == 0.0 && b == 0.0) return M;
+  const double th = std::atan2(b, a) - M_PI / 4.0;
+  const double cs = std::cos(th), sn = std::sin(th);
+  M[static_cast<size_t>(i) * n + i] = cs;
+  M[static_cast<size_t>(i) * n + j] = sn;
+  M[static_cast<size_t>(j) * n + i] = -sn;
+  M[static_cast<size_t>(j) * n + j] = cs;
+  return M;
 }
 
 // Counter-based generator for the library's own random orthogonal block.
@@ -215,6 +248,13 @@ sq_status_t build_factors_host(const float* calib, int64_t T, int64_t n, int32_t
       Ouse = Oown.data();
     }
     RA = art(col, Ouse);
+    const int art_steps = static_cast<int>((flags >> 8) & 0x7FFu) + 1;
+    for (int step = 1; step < art_steps; ++step) {         // repeated ART rotations on the column so far
+      std::vector<double> cur(n1, 0.0);
+      for (int r = 0; r < n1; ++r)
+        for (int k = 0; k < n1; ++k) cur[r] += RA[static_cast<size_t>(r) * n1 + k] * col[k];
+      RA = matmul(art_repeat_step(cur), RA, n1);
+    }
   } else {
     RA = identity(n1);
   }

@@ -93,6 +93,21 @@ def test_build_rotation_matches_oracle(sq, w, flags):
     rot.close()
 
 
+@pytest.mark.parametrize("steps", [2, 5, 16])
+def test_build_rotation_with_repeated_art_steps_matches_oracle(sq, steps):
+    w = wl.small("arts", 6, 64, 64, 8, 17)
+    X = wl.make_activations(w).astype(np.float32)
+    O = ora.haar_orthogonal(w.n1 - 2, np.random.default_rng(5))
+    R1o, R2o = ora.build_rotation(X, w.n1, w.n2, O=O, art_steps=steps)
+    rot = sq.sq_build_rotation(X, w.n1, w.n2, flags=sq.SQ_ROT_DEFAULT | sq.SQ_ROT_ART_STEPS(steps), O=O)
+    R1, R2 = rot.factors()
+    assert np.max(np.abs(R1.astype(np.float64) - R1o)) <= 1e-6
+    assert np.max(np.abs(R2.astype(np.float64) - R2o)) <= 1e-6
+    one = sq.sq_build_rotation(X, w.n1, w.n2, O=O).factors()[0]
+    assert not np.array_equal(one, R1)
+    rot.close()
+
+
 def test_build_rotation_own_generator_gives_orthogonal_factors(sq):
     w = wl.TINY
     X = wl.make_activations(w).astype(np.float32)

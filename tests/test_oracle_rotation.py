@@ -100,6 +100,43 @@ def test_givens_embedding():
 
 
 # ---------------------------------------------------------------- ART (P4)
+@pytest.mark.parametrize("steps", [2, 3, 8, 33])
+def test_repeated_art_steps_equalise_one_pair_each(steps):
+    """Paragraph "Effect of ART Steps": every further step is a rotation in the plane of the
+    current (outlier, minimum) pair that leaves both at r/sqrt(2) (Lemma 1) and touches nothing
+    else; the product stays orthogonal, keeps the norm and never raises the column's absmax."""
+    rng = np.random.default_rng(steps)
+    n = 24
+    c = rng.standard_normal(n)
+    c[5] = 800.0
+    c[11] = -300.0
+    O = ora.haar_orthogonal(n - 2, rng)
+    prev = ora.art_matrix_steps(c, O, steps - 1)
+    full = ora.art_matrix_steps(c, O, steps)
+    assert np.allclose(full.T @ full, np.eye(n), atol=1e-12)
+    before, after = prev @ c, full @ c
+    i, j = ora.art_indices(before)
+    r = math.hypot(before[i], before[j])
+    assert abs(after[i] - r / math.sqrt(2)) < 1e-9 and abs(after[j] - r / math.sqrt(2)) < 1e-9
+    others = [k for k in range(n) if k not in (i, j)]
+    assert np.allclose(after[others], before[others], atol=1e-12)
+    assert abs(np.linalg.norm(after) - np.linalg.norm(c)) < 1e-9
+    assert np.max(np.abs(after)) <= np.max(np.abs(before)) + 1e-12
+    # one step is the plain ART
+    assert np.array_equal(ora.art_matrix_steps(c, O, 1), ora.art_matrix(c, O))
+
+
+def test_repeated_art_steps_lower_the_massive_outlier_further():
+    c = np.array([800.0, 0.3, -1.0, 2.0, 0.5, -0.7, 1.5, 0.1])
+    peaks = [np.max(np.abs(ora.art_matrix_steps(c, None, k) @ c)) for k in (1, 2, 3, 4)]
+    assert abs(peaks[0] - math.hypot(800.0, 0.1) / math.sqrt(2)) < 1e-9      # (800, 0.1): smallest magnitude is index 7
+    assert all(b <= a + 1e-12 for a, b in zip(peaks, peaks[1:]))
+    # two equal halves of 800/sqrt(2) are each halved again against a small entry: 800/2 after three steps
+    assert abs(peaks[1] - peaks[0]) < 1e-9 and abs(peaks[2] - 400.0) < 1e-2
+    R1, R2 = ora.build_rotation(np.tile(c, (2, 4)).reshape(2, 32), 8, 4, art_steps=3)
+    assert np.allclose(R1.astype(np.float64).T @ R1.astype(np.float64), np.eye(8), atol=1e-6)
+
+
 @pytest.mark.parametrize("n", [2, 3, 8, 16, 64])
 def test_art_equalises_outlier_pair(n):
     rng = np.random.default_rng(n)
