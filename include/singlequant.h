@@ -119,7 +119,10 @@ sq_status_t sq_pack_weight(const sq_rotation_t* rot_or_null, const void* W, int6
  *   Y   DEVICE fp16  [M x N] (out)
  *   accdbg_or_null  DEVICE int32 [M x N] (out, optional: the raw accumulators)
  *   workspace       DEVICE scratch of at least sq_w4a4_gemm_workspace_bytes(M,N,K) bytes, or
- *                   NULL (then small-M problems run without split-K, slower but identical)
+ *                   NULL.  Every kernel of this version keeps its intermediates on chip (split-K
+ *                   partial tiles are exchanged through cluster shared memory), so the size is 0
+ *                   for all shapes and the argument is not read; it stays in the signature so
+ *                   that callers need not change if a later kernel wants scratch.
  * Supported: K even, K <= 65536 (so that the 256x-scaled int32 accumulator cannot overflow).
  * The tensor-core path needs K % 128 == 0 and N % 8 == 0; other shapes run a plain integer
  * kernel with the same results. */

@@ -242,8 +242,9 @@ sq_status_t sq_linear(const sq_rotation_t* rot, const void* X, int64_t M, const 
   const size_t gws_bytes = sq::gemm_workspace_bytes(M, N, K);
   sq_status_t st = sq_rotate_quant_act(rot, X, M, Xq, sx, nullptr, stream);
   if (st != SQ_OK) return st;
-  // The split-K decode kernel is preceded by a memset of its counters, so it is launched normally.
-  sq::g_pdl_next = sq::gemv_supported(M, N, K) || !sq::gemm_decode_supported(M, N, K);
+  // Every tensor-core GEMM kernel and the dot-product kernel start their set-up (and their weight
+  // loads) while the rotate kernel drains; they wait for it before they read Xq or sx.
+  sq::g_pdl_next = true;
   st = sq_w4a4_gemm(Xq, sx, Wq, sw, M, N, K, Y, nullptr, gws_bytes ? gws : nullptr, gws_bytes, stream);
   sq::g_pdl_next = false;
   return st;

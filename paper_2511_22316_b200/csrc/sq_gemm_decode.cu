@@ -6,18 +6,24 @@
 // TMEM lanes), the tokens are the MMA's N (16, 32 or 64).  Four warps read the packed bytes of
 // "their" weight row from the TMA staging ring, widen them in registers and store the int8
 // operand into a TMEM ring (tcgen05.st); the few token rows are widened through shared memory.
-// A work item is (tile of 128 channels, chunk of K); the chunk count is chosen so that the items
-// fill the SMs evenly.  Each item leaves an exact int32 partial tile in the caller's workspace;
-// the item that completes a tile (a counter per tile) adds the partials in a fixed order,
-// dequantises and writes fp16 -- the result does not depend on which item came last.
+//
+// Where the tiles alone do not fill the SMs, K is split over a thread-block cluster of 2, 4 or 8
+// CTAs: every CTA of the cluster accumulates its chunk of K for the same tile, then the cluster
+// reduce-scatters the exact int32 partial tiles through distributed shared memory -- CTA r of s
+// receives, from each of the others, the 128 / s rows it finishes (one slot per source, written
+// with st.shared::cluster and handed over with a cluster-scope release/acquire barrier), adds
+// them to its own rows, dequantises and writes fp16.  Integer addition makes the result
+// independent of any order; no partial tile, counter or workspace exists in global memory.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = two groups of weight
 // converters and warps 10..13 = two groups of token unpackers (a group takes every other block:
 // a block costs a warp several hundred cycles of waits and fences whatever its size), warps
-// 14..21 = two epilogue groups that take the items in turn (four accumulators, so epilogues,
-// whose global-memory round trips are long, overlap the main loop of the following items).
+// 14..21 = two epilogue groups that take the tiles in turn (four accumulators, so epilogues
+// overlap the main loop of the following tiles).
 #include <cuda.h>
 #include <cuda_fp16.h>
+
+#include <atomic>
 
 #include "sq_internal.h"
 #include "sq_ptx.cuh"
@@ -29,51 +35,34 @@ constexpr int D_CONV_GROUPS = 2;          // converter groups; group g takes the
 constexpr int D_A_WARPS = 4 * D_CONV_GROUPS, D_B_WARPS = 2 * D_CONV_GROUPS;
 constexpr int D_EPI_GROUPS = 2, D_EPI_WARPS = 4 * D_EPI_GROUPS;
 constexpr int D_THREADS = (2 + D_A_WARPS + D_B_WARPS + D_EPI_WARPS) * 32;
-constexpr int D_S_ST = 6;                // staging stages (256 channels each)
 constexpr int D_S_OP = 4;                // operand stages (TMEM A ring: 4 x 64 columns)
 constexpr int D_A_COL0 = 256;
-constexpr int D_MAX_SPLITS = 16;           // partial tiles of one output tile, all in flight when they are summed
+constexpr int D_MAX_SPLITS = 8;            // largest cluster (the portable limit)
 constexpr int D_ACCS = 4;                 // accumulators in TMEM (columns 0 .. 4 * NT)
 
 enum DecSite : uint32_t {
   DSITE_ST_EMPTY = 64, DSITE_ST_FULL_A, DSITE_ST_FULL_B, DSITE_EMPTY_A, DSITE_EMPTY_B, DSITE_FULL,
-  DSITE_TMEM_FULL, DSITE_TMEM_EMPTY
+  DSITE_TMEM_FULL, DSITE_TMEM_EMPTY, DSITE_RED_FULL, DSITE_RED_EMPTY
 };
 
 template <int NT>
 struct DecSmem {
+  static constexpr int S_ST = NT == 64 ? 4 : 6;      // staging stages (256 channels each)
   static constexpr int W_ST = 128 * 128;             // packed weight rows, two k-blocks
   static constexpr int X_ST = NT * 128;              // packed token rows, two k-blocks
   static constexpr int X_OP = 2 * NT * 128;          // int8 token rows, two k-block tiles
+  // Reduce-scatter slots of one epilogue group: (s - 1) sources x 128 / s rows x NT int32, largest at s = 8.
+  static constexpr int RED_GROUP = 128 * NT * 4 / D_MAX_SPLITS * (D_MAX_SPLITS - 1);
   static constexpr int OFF_X_OP = 0;
   static constexpr int OFF_W_ST = OFF_X_OP + D_S_OP * X_OP;
-  static constexpr int OFF_X_ST = OFF_W_ST + D_S_ST * W_ST;
-  static constexpr int OFF_BAR = OFF_X_ST + D_S_ST * X_ST;
-  static constexpr int NUM_BARS = 2 * D_S_ST + 2 * D_S_OP + 2 * D_ACCS;
+  static constexpr int OFF_X_ST = OFF_W_ST + S_ST * W_ST;
+  static constexpr int OFF_RED = OFF_X_ST + S_ST * X_ST;
+  static constexpr int OFF_BAR = OFF_RED + D_EPI_GROUPS * RED_GROUP;
+  static constexpr int NUM_BARS = 2 * S_ST + 2 * D_S_OP + 2 * D_ACCS + 2 * D_EPI_GROUPS;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int TOTAL = OFF_MISC + 32;
   static constexpr int DYN_BYTES = TOTAL + 1024;
 };
-
-// Splits the K blocks of every tile into `splits` chunks.  Cost model (cycles, measured): a block of
-// 256 channels takes about 1250 cycles of the main loop; splitting K adds about 8000 cycles once
-// (partial tiles, fence, counter, the sum by the last item).  The cheapest count wins.
-int choose_splits(int tiles, int blocks, int sms) {
-  int best = 1;
-  double best_cost = 0.0;
-  for (int s = 1; s <= D_MAX_SPLITS && s * 2 <= blocks + 1; ++s) {
-    if (s > 1 && blocks / s < 2) break;
-    const long long items = static_cast<long long>(tiles) * s;
-    const long long waves = (items + sms - 1) / sms;
-    const double per_item = static_cast<double>((blocks + s - 1) / s);
-    const double cost = static_cast<double>(waves) * per_item * 1250.0 + (s > 1 ? 8000.0 : 0.0);
-    if (s == 1 || cost < best_cost * 0.97) {
-      best_cost = cost;
-      best = s;
-    }
-  }
-  return best;
-}
 
 // Widens the 128 staged bytes of `rows` token rows into two int8 k-block tiles (rows x 128 B each,
 // 128-byte swizzle), same byte order as unpack_tile.  Task = (row, 16-byte chunk).
@@ -99,56 +88,54 @@ template <int NT>
 __global__ void __launch_bounds__(D_THREADS, 1)
 w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
                         const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
-                        int splits, __half* __restrict__ Y, int32_t* __restrict__ accdbg,
-                        int32_t* __restrict__ partials, unsigned int* __restrict__ counters) {
+                        int splits, __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
   using L = DecSmem<NT>;
+  constexpr int S_ST = L::S_ST;
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
   uint64_t* st_full = bars;
-  uint64_t* st_empty = bars + D_S_ST;
-  uint64_t* full = bars + 2 * D_S_ST;
-  uint64_t* empty = bars + 2 * D_S_ST + D_S_OP;
-  uint64_t* tmem_full = bars + 2 * D_S_ST + 2 * D_S_OP;      // [D_ACCS]
+  uint64_t* st_empty = bars + S_ST;
+  uint64_t* full = bars + 2 * S_ST;
+  uint64_t* empty = bars + 2 * S_ST + D_S_OP;
+  uint64_t* tmem_full = bars + 2 * S_ST + 2 * D_S_OP;        // [D_ACCS]
   uint64_t* tmem_empty = tmem_full + D_ACCS;                  // [D_ACCS]
+  uint64_t* red_full = tmem_empty + D_ACCS;                   // [D_EPI_GROUPS] the others' rows have arrived here
+  uint64_t* red_empty = red_full + D_EPI_GROUPS;              // [D_EPI_GROUPS] the others have read what this CTA sent
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
-  uint32_t* last_flag = tmem_slot + 1;                        // [D_EPI_GROUPS]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = K / 128;
   const int num_sb = (num_kb + 1) / 2;                 // blocks of 256 channels (the last may be half)
   const int tiles = (N + 127) / 128;
-  const int num_items = tiles * splits;
   const uint32_t limit = wait_limit();
 
-  // item -> (tile, first block, one-past-last block)
-  auto item_range = [&](int item, int& tile, int& b0, int& b1) {
-    tile = item / splits;
-    const int sp = item % splits;
-    b0 = static_cast<int>(static_cast<long long>(sp) * num_sb / splits);
-    b1 = static_cast<int>(static_cast<long long>(sp + 1) * num_sb / splits);
-  };
-  // The producer's walk over (item, block); `budget` blocks are issued per call (waiting for the
-  // staging stage of each), so that the first ring-full can go out before the CTA has set up.
-  int p_item = blockIdx.x, p_sb = -1, p_b1 = 0, p_tile = 0;
+  // The cluster (a single CTA when splits == 1) takes the tiles cid, cid + ncl, ...; CTA `crank`
+  // of it accumulates the blocks [b0, b1) of every one of them.
+  const uint32_t crank = (splits > 1) ? cluster_ctarank() : 0u;
+  const int cid = static_cast<int>(blockIdx.x) / splits, ncl = static_cast<int>(gridDim.x) / splits;
+  const int b0 = static_cast<int>(static_cast<long long>(crank) * num_sb / splits);
+  const int b1 = static_cast<int>(static_cast<long long>(crank + 1) * num_sb / splits);
+
+  // The producer's walk over (tile, block); `budget` blocks are issued per call (waiting for the
+  // staging stage of each).  The weights do not depend on the kernel before this one, the tokens
+  // do: with `defer_x` only the weights are requested and the blocks are noted in pre_sb.
+  int p_tile = cid, p_sb = b0, pre_n = 0;
+  int pre_sb[S_ST];
   uint32_t p_it = 0;
-  auto produce = [&](uint32_t budget) -> bool {
-    while (budget > 0 && p_item < num_items) {
-      if (p_sb < 0) {
-        int b0;
-        item_range(p_item, p_tile, b0, p_b1);
-        p_sb = b0;
-      }
-      const int ss = p_it % D_S_ST;
-      if (!mbar_wait(&st_empty[ss], ((p_it / D_S_ST) & 1) ^ 1, DSITE_ST_EMPTY, limit)) return false;
+  auto produce = [&](uint32_t budget, bool defer_x) -> bool {
+    while (budget > 0 && p_tile < tiles) {
+      const int ss = p_it % S_ST;
+      if (!mbar_wait(&st_empty[ss], ((p_it / S_ST) & 1) ^ 1, DSITE_ST_EMPTY, limit)) return false;
       mbar_arrive_expect_tx(&st_full[ss], L::W_ST + L::X_ST);
       tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, &tmap_w, &st_full[ss], p_sb * 128, p_tile * 128);
-      tma_load_2d(smem + L::OFF_X_ST + ss * L::X_ST, &tmap_x, &st_full[ss], p_sb * 128, 0);
+      if (defer_x) pre_sb[pre_n++] = p_sb;
+      else tma_load_2d(smem + L::OFF_X_ST + ss * L::X_ST, &tmap_x, &st_full[ss], p_sb * 128, 0);
       ++p_it;
       --budget;
-      if (++p_sb >= p_b1) {
-        p_sb = -1;
-        p_item += gridDim.x;
+      if (++p_sb >= b1) {
+        p_sb = b0;
+        p_tile += ncl;
       }
     }
     return true;
@@ -157,7 +144,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmap_w);
     tma_prefetch_desc(&tmap_x);
-    for (int s = 0; s < D_S_ST; ++s) {
+    for (int s = 0; s < S_ST; ++s) {
       mbar_init(&st_full[s], 1);
       mbar_init(&st_empty[s], 6);                      // one converter group + one unpacker group
     }
@@ -169,8 +156,14 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
       mbar_init(&tmem_full[b], 1);
       mbar_init(&tmem_empty[b], 4);
     }
+    // One arrival per row that crosses CTAs: (s - 1) sources x 128 / s rows, both ways.
+    const uint32_t crossing = splits > 1 ? static_cast<uint32_t>((splits - 1) * (128 / splits)) : 1u;
+    for (int g = 0; g < D_EPI_GROUPS; ++g) {
+      mbar_init(&red_full[g], crossing);
+      mbar_init(&red_empty[g], crossing);
+    }
     mbar_fence_init();
-    produce(D_S_ST);                                   // the whole staging ring, before anyone else is ready
+    produce(S_ST, true);                               // the weights of the whole staging ring, before anyone else is ready
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, 512);
@@ -178,21 +171,25 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   }
   tc_fence_before_sync();
   __syncthreads();
+  if (splits > 1) cluster_sync_all();                  // every CTA's barriers exist before anyone arrives on them
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();                                      // the tokens and their scales come from the kernel before
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------------------------
-    if (lane == 0) produce(0xFFFFFFFFu);
+    if (lane == 0) {
+      for (int i = 0; i < pre_n; ++i)
+        tma_load_2d(smem + L::OFF_X_ST + i * L::X_ST, &tmap_x, &st_full[i], pre_sb[i] * 128, 0);
+      produce(0xFFFFFFFFu, false);
+    }
   } else if (warp == 1) {
     // ------------------------------ MMA issuer --------------------------------------------------
     if (elect_one()) {
       constexpr uint32_t idesc = umma_idesc(/*c=s32*/ 2, /*a=s8*/ 1, /*b=s8*/ 1, 128, NT);
       uint32_t it = 0, icount = 0;
       bool ok = true;
-      for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++icount) {
-        int tile, b0, b1;
-        item_range(item, tile, b0, b1);
+      for (int tile = cid; tile < tiles && ok; tile += ncl, ++icount) {
         const uint32_t acc = icount % D_ACCS;
         ok = mbar_wait(&tmem_empty[acc], ((icount / D_ACCS) & 1) ^ 1, DSITE_TMEM_EMPTY, limit);
         if (!ok) break;
@@ -223,13 +220,11 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
     uint32_t it = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
-      int tile, b0, b1;
-      item_range(item, tile, b0, b1);
+    for (int tile = cid; tile < tiles && ok; tile += ncl) {
       for (int sb = b0; sb < b1 && ok; ++sb, ++it) {
         if ((it % D_CONV_GROUPS) != static_cast<uint32_t>(grp)) continue;
-        const int ss = it % D_S_ST, s = it % D_S_OP;
-        ok = mbar_wait(&st_full[ss], (it / D_S_ST) & 1, DSITE_ST_FULL_A, limit);
+        const int ss = it % S_ST, s = it % D_S_OP;
+        ok = mbar_wait(&st_full[ss], (it / S_ST) & 1, DSITE_ST_FULL_A, limit);
         if (!ok) break;
         const unsigned char* row = smem + L::OFF_W_ST + ss * L::W_ST + r * 128;
         const int nh = (2 * sb + 1 < num_kb) ? 2 : 1;
@@ -269,13 +264,11 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     const int t = (threadIdx.x - (2 + D_A_WARPS) * 32) & 63;
     uint32_t it = 0;
     bool ok = true;
-    for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x) {
-      int tile, b0, b1;
-      item_range(item, tile, b0, b1);
+    for (int tile = cid; tile < tiles && ok; tile += ncl) {
       for (int sb = b0; sb < b1 && ok; ++sb, ++it) {
         if ((it % D_CONV_GROUPS) != static_cast<uint32_t>(grp)) continue;
-        const int ss = it % D_S_ST, s = it % D_S_OP;
-        ok = mbar_wait(&st_full[ss], (it / D_S_ST) & 1, DSITE_ST_FULL_B, limit) &&
+        const int ss = it % S_ST, s = it % D_S_OP;
+        ok = mbar_wait(&st_full[ss], (it / S_ST) & 1, DSITE_ST_FULL_B, limit) &&
              mbar_wait(&empty[s], ((it / D_S_OP) & 1) ^ 1, DSITE_EMPTY_B, limit);
         if (!ok) break;
         unpack_rows(smem + L::OFF_X_ST + ss * L::X_ST, smem + L::OFF_X_OP + s * L::X_OP, NT, t, 64,
@@ -291,27 +284,70 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   } else {
     // ------------------------------ epilogue groups -----------------------------------------------
     const int q = warp & 3;
-    const int eg = (warp - (2 + D_A_WARPS + D_B_WARPS)) >> 2;        // this group takes items eg, eg + 2, ...
-    const int et = (threadIdx.x - (2 + D_A_WARPS + D_B_WARPS) * 32) & 127;
+    const int eg = (warp - (2 + D_A_WARPS + D_B_WARPS)) >> 2;        // this group takes tiles eg, eg + 2, ... of the CTA's
     const int rowl = q * 32 + lane;                                  // row of the tile = TMEM lane
+    // Reduce-scatter geometry: CTA `owner` finishes this thread's row; this CTA finishes the rows
+    // [crank * rows_per, (crank + 1) * rows_per).  Slots are [source][4-column chunk][row][4] int32:
+    // a warp's 16-byte accesses are contiguous.
+    const int rows_per = 128 / splits;
+    const uint32_t owner = static_cast<uint32_t>(rowl / rows_per);
+    const int rloc = rowl % rows_per;
+    const bool mine = (owner == crank);
+    const bool warp_owns = __any_sync(0xFFFFFFFFu, mine);
+    const bool warp_sends = __any_sync(0xFFFFFFFFu, !mine);
+    unsigned char* red = smem + L::OFF_RED + eg * L::RED_GROUP;
+    const uint32_t my_slot = crank < owner ? crank : crank - 1u;     // this CTA's slot in `owner`'s buffer
+    const uint32_t send_addr = mine ? 0u : cluster_map(red, owner) + ((my_slot * (NT / 4)) * rows_per + rloc) * 16u;
+    const uint32_t send_bar = mine ? 0u : cluster_map(&red_full[eg], owner);
     bool ok = true;
     uint32_t icount = 0;
-    for (int item = blockIdx.x; item < num_items && ok; item += gridDim.x, ++icount) {
+    for (int tile = cid; tile < tiles && ok; tile += ncl, ++icount) {
       if ((icount % D_EPI_GROUPS) != static_cast<uint32_t>(eg)) continue;
-      int tile, b0, b1;
-      item_range(item, tile, b0, b1);
       const uint32_t acc = icount % D_ACCS;
+      const uint32_t g = icount / D_EPI_GROUPS;                      // the group's tile count
       ok = mbar_wait(&tmem_full[acc], (icount / D_ACCS) & 1, DSITE_TMEM_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t tmem_d = tmem_base + acc * NT + (static_cast<uint32_t>(q * 32) << 16);
       const int ch = tile * 128 + rowl;                    // output channel of this thread
       const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;
-      // Partial tiles are stored as [item][4-column chunk][row][4]: a warp's 16-byte accesses are contiguous.
-      int4* mine = reinterpret_cast<int4*>(partials) + static_cast<size_t>(item) * (NT / 4) * 128 + rowl;
+      if (warp_sends) {
+        // This CTA's chunk of K for rows that another CTA finishes: into that CTA's slot, once it
+        // has read what was sent for the group's previous tile.
+        if (!mine) ok = mbar_wait_acq_cluster(&red_empty[eg], (g & 1) ^ 1, DSITE_RED_EMPTY, limit);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+#pragma unroll
+        for (int c16 = 0; c16 < NT / 16; ++c16) {
+          uint32_t r[16];
+          __syncwarp();
+          tmem_ld_32x32b_x16(tmem_d + 16 * c16, r);
+          tmem_wait_ld();
+          if (!mine) {
+#pragma unroll
+            for (int c = 0; c < 4; ++c)
+              st_v4_cluster(send_addr + static_cast<uint32_t>((4 * c16 + c) * rows_per) * 16u,
+                            static_cast<int32_t>(r[4 * c]) >> 8, static_cast<int32_t>(r[4 * c + 1]) >> 8,
+                            static_cast<int32_t>(r[4 * c + 2]) >> 8, static_cast<int32_t>(r[4 * c + 3]) >> 8);
+          }
+        }
+        if (!mine) mbar_arrive_release_cluster(send_bar);
+      }
+      if (!warp_owns) {                                      // nothing to finish here: hand the accumulator back
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&tmem_empty[acc]);
+        continue;
+      }
+      if (splits > 1) {
+        if (mine) ok = mbar_wait_acq_cluster(&red_full[eg], g & 1, DSITE_RED_FULL, limit);
+        ok = __all_sync(0xFFFFFFFFu, ok);
+        if (!ok) break;
+      }
 #pragma unroll
       for (int c16 = 0; c16 < NT / 16; ++c16) {
         uint32_t r[16];
+        __syncwarp();
         tmem_ld_32x32b_x16(tmem_d + 16 * c16, r);
         tmem_wait_ld();
         if (c16 == NT / 16 - 1) {                          // last read: hand the accumulator back
@@ -319,62 +355,21 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
           __syncwarp();
           if (lane == 0) mbar_arrive(&tmem_empty[acc]);
         }
-        if (splits == 1) {
+        if (!mine) continue;
 #pragma unroll
-          for (int x = 0; x < 16; ++x) {
-            const int e = 16 * c16 + x;
-            if (e < M && ch < N) {
-              const int32_t a = static_cast<int32_t>(r[x]) >> 8;          // exact: the accumulator is 256 * acc
-              const float f = __int_as_float(0x4B400000 + a) - 12582912.0f;
-              Y[static_cast<size_t>(e) * N + ch] = __float2half_rn(f * (__half2float(__ldg(sx + e)) * swv));
-              if (accdbg) accdbg[static_cast<size_t>(e) * N + ch] = a;
-            }
-          }
-        } else {
-#pragma unroll
-          for (int c = 0; c < 4; ++c)
-            mine[(4 * c16 + c) * 128] =
-                make_int4(static_cast<int32_t>(r[4 * c]) >> 8, static_cast<int32_t>(r[4 * c + 1]) >> 8,
-                          static_cast<int32_t>(r[4 * c + 2]) >> 8, static_cast<int32_t>(r[4 * c + 3]) >> 8);
-        }
-      }
-      if (splits == 1) continue;
-      named_barrier(1 + eg, 128);                            // the group's stores happen before ...
-      if (et == 0) {
-        __threadfence();                                     // ... this fence, which orders them before the count
-        const unsigned int old = atomicAdd(&counters[tile], 1u);
-        const bool last = (old == static_cast<unsigned int>(splits - 1));
-        if (last) {
-          counters[tile] = 0u;                               // ready for the next call
-          __threadfence();                                   // the other items' partials are visible from here on
-        }
-        last_flag[eg] = last ? 1u : 0u;
-      }
-      named_barrier(1 + eg, 128);
-      const bool finish = (last_flag[eg] != 0u);
-      if (finish) {
-        // Sum the tile's partials in the fixed order sp = 0, 1, ...: the result does not depend on
-        // which item came last.  All loads of a chunk are issued before any is used.
-        const int4* base = reinterpret_cast<const int4*>(partials) + static_cast<size_t>(tile) * splits * (NT / 4) * 128 + rowl;
-#pragma unroll 1
-        for (int c = 0; c < NT / 4; ++c) {
-          int4 a = make_int4(0, 0, 0, 0);
-#pragma unroll
-          for (int h = 0; h < D_MAX_SPLITS; h += 8) {      // eight loads in flight at a time
-            if (h < splits) {
-              int4 v[8];
-#pragma unroll
-              for (int sp = 0; sp < 8; ++sp)
-                if (h + sp < splits) v[sp] = __ldcg(base + (static_cast<size_t>(h + sp) * (NT / 4) + c) * 128);
-#pragma unroll
-              for (int sp = 0; sp < 8; ++sp)
-                if (h + sp < splits) { a.x += v[sp].x; a.y += v[sp].y; a.z += v[sp].z; a.w += v[sp].w; }
-            }
+        for (int c = 0; c < 4; ++c) {
+          // exact: the accumulator is 256 * (sum of products)
+          int4 a = make_int4(static_cast<int32_t>(r[4 * c]) >> 8, static_cast<int32_t>(r[4 * c + 1]) >> 8,
+                             static_cast<int32_t>(r[4 * c + 2]) >> 8, static_cast<int32_t>(r[4 * c + 3]) >> 8);
+          const int4* slot = reinterpret_cast<const int4*>(red) + (4 * c16 + c) * rows_per + rloc;
+          for (int sp = 0; sp + 1 < splits; ++sp) {
+            const int4 v = slot[sp * (NT / 4) * rows_per];
+            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
           }
           const int32_t av[4] = {a.x, a.y, a.z, a.w};
 #pragma unroll
           for (int x = 0; x < 4; ++x) {
-            const int e = 4 * c + x;
+            const int e = 16 * c16 + 4 * c + x;
             if (e < M && ch < N) {
               const float f = __int_as_float(0x4B400000 + av[x]) - 12582912.0f;
               Y[static_cast<size_t>(e) * N + ch] = __float2half_rn(f * (__half2float(__ldg(sx + e)) * swv));
@@ -383,38 +378,82 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
           }
         }
       }
-      named_barrier(1 + eg, 128);                            // last_flag may be rewritten by the group's next item
+      if (splits > 1 && mine) {                              // the slots may be rewritten
+        for (uint32_t d = 0; d < static_cast<uint32_t>(splits); ++d)
+          if (d != crank) mbar_arrive_release_cluster(cluster_map(&red_empty[eg], d));
+      }
     }
   }
 
   tc_fence_before_sync();
   __syncthreads();
+  if (splits > 1) cluster_sync_all();                  // nobody leaves while another CTA may still write or arrive here
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, 512);
   }
 }
 
+// Largest number of clusters of `s` CTAs of this kernel that the device holds at once.
+template <int NT>
+int max_clusters(int s, int sms) {
+  using L = DecSmem<NT>;
+  static std::atomic<int> cache[64][4];
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return 0;
+  const int slot = s == 2 ? 1 : (s == 4 ? 2 : (s == 8 ? 3 : 0));
+  if (slot == 0) return sms;
+  int v = cache[dev][slot].load(std::memory_order_relaxed);
+  if (v != 0) return v > 0 ? v : 0;
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = dim3(static_cast<unsigned>(sms / s * s));
+  cfg.blockDim = dim3(D_THREADS);
+  cfg.dynamicSmemBytes = L::DYN_BYTES;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeClusterDimension;
+  attr[0].val.clusterDim.x = static_cast<unsigned>(s);
+  attr[0].val.clusterDim.y = 1;
+  attr[0].val.clusterDim.z = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  int n = 0;
+  if (cudaOccupancyMaxActiveClusters(&n, w4a4_gemm_decode_kernel<NT>, &cfg) != cudaSuccess) {
+    cudaGetLastError();
+    n = 0;
+  }
+  cache[dev][slot].store(n > 0 ? n : -1, std::memory_order_relaxed);
+  return n;
+}
+
+// Chooses the cluster size s in {1, 2, 4, 8} over which K is split.  Cost model (cycles, measured):
+// a block of 256 channels costs the main loop BLOCK_CYCLES; the exchange through shared memory
+// adds SPLIT_CYCLES once; tiles beyond the clusters the device holds at once take further waves.
+template <int NT>
+int choose_splits(int tiles, int blocks, int sms) {
+  constexpr double BLOCK_CYCLES = NT == 64 ? 1100.0 : (NT == 32 ? 900.0 : 700.0);
+  constexpr double SPLIT_CYCLES = 2500.0;
+  int best = 1;
+  double best_cost = 0.0;
+  for (int s = 1; s <= D_MAX_SPLITS; s *= 2) {
+    if (s > 1 && blocks / s < 2) break;
+    const int ncl = max_clusters<NT>(s, sms);
+    if (ncl <= 0) continue;
+    const int waves = (tiles + ncl - 1) / ncl;
+    const double cost = static_cast<double>(waves) * ((blocks + s - 1) / s) * BLOCK_CYCLES + (s > 1 ? SPLIT_CYCLES : 0.0);
+    if (s == 1 || cost < best_cost * 0.97) {
+      best_cost = cost;
+      best = s;
+    }
+  }
+  return best;
+}
+
 template <int NT>
 sq_status_t launch_decode(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N, int K, void* Y,
-                          int32_t* accdbg, void* workspace, size_t workspace_bytes, cudaStream_t s) {
+                          int32_t* accdbg, cudaStream_t s) {
   using L = DecSmem<NT>;
   const int sms = sm_count();
   if (sms <= 0) return SQ_ERR_CUDA;
-  const int tiles = (N + 127) / 128, blocks = (K / 128 + 1) / 2;
-  int splits = choose_splits(tiles, blocks, sms);
-  const size_t part_bytes = static_cast<size_t>(tiles) * splits * 128 * NT * sizeof(int32_t);
-  const size_t cnt_off = (part_bytes + 255) / 256 * 256;
-  if (splits > 1 && (workspace == nullptr || workspace_bytes < cnt_off + static_cast<size_t>(tiles) * 4)) splits = 1;
-  int32_t* partials = nullptr;
-  unsigned int* counters = nullptr;
-  if (splits > 1) {
-    partials = static_cast<int32_t*>(workspace);
-    counters = reinterpret_cast<unsigned int*>(static_cast<unsigned char*>(workspace) + cnt_off);
-    if (cudaMemsetAsync(counters, 0, static_cast<size_t>(tiles) * 4, s) != cudaSuccess) return SQ_ERR_CUDA;
-  }
-  CUtensorMap mw, mx;
-  if (!make_packed_map(&mw, Wq, N, K / 2, 128) || !make_packed_map(&mx, Xq, M, K / 2, NT)) return SQ_ERR_CUDA;
   auto kern = w4a4_gemm_decode_kernel<NT>;
   static bool attr_set = false;
   if (!attr_set) {
@@ -422,12 +461,19 @@ sq_status_t launch_decode(const void* Xq, const void* sx, const void* Wq, const 
       return SQ_ERR_CUDA;
     attr_set = true;
   }
-  const int items = tiles * splits;
-  const int grid = items < sms ? items : sms;
-  kern<<<grid, D_THREADS, L::DYN_BYTES, s>>>(mw, mx, static_cast<const __half*>(sx), static_cast<const __half*>(sw), M, N,
-                                             K, splits, static_cast<__half*>(Y), accdbg, partials, counters);
+  const int tiles = (N + 127) / 128, blocks = (K / 128 + 1) / 2;
+  const int splits = choose_splits<NT>(tiles, blocks, sms);
+  const int ncl_max = max_clusters<NT>(splits, sms);
+  if (ncl_max <= 0) return SQ_ERR_CUDA;
+  CUtensorMap mw, mx;
+  if (!make_packed_map(&mw, Wq, N, K / 2, 128) || !make_packed_map(&mx, Xq, M, K / 2, NT)) return SQ_ERR_CUDA;
+  const int ncl = tiles < ncl_max ? tiles : ncl_max;
+  const cudaError_t err = launch_cluster_maybe_pdl(kern, dim3(static_cast<unsigned>(ncl * splits)), dim3(D_THREADS),
+                                                   static_cast<size_t>(L::DYN_BYTES), s, static_cast<unsigned>(splits), mw,
+                                                   mx, static_cast<const __half*>(sx), static_cast<const __half*>(sw), M, N,
+                                                   K, splits, static_cast<__half*>(Y), accdbg);
   count_launch();
-  return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+  return err == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
 }
 
 }  // namespace
@@ -436,24 +482,14 @@ bool gemm_decode_supported(int64_t M, int64_t N, int64_t K) {
   return M >= 1 && M <= 64 && N >= 128 && (K % 128 == 0) && K >= 256 && (N % 8 == 0);
 }
 
-// Workspace of the split-K path: int32 partial tiles, then one counter per tile.
-size_t gemm_decode_workspace_bytes(int64_t M, int64_t N, int64_t K) {
-  if (!gemm_decode_supported(M, N, K)) return 0;
-  const int sms = sm_count();
-  if (sms <= 0) return 0;
-  const int NT = M <= 16 ? 16 : (M <= 32 ? 32 : 64);
-  const int tiles = static_cast<int>((N + 127) / 128), blocks = static_cast<int>((K / 128 + 1) / 2);
-  const int splits = choose_splits(tiles, blocks, sms);
-  if (splits == 1) return 0;
-  const size_t part_bytes = static_cast<size_t>(tiles) * splits * 128 * NT * sizeof(int32_t);
-  return (part_bytes + 255) / 256 * 256 + (static_cast<size_t>(tiles) * 4 + 255) / 256 * 256;
-}
+// The split-K exchange lives in shared memory: no workspace.
+size_t gemm_decode_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
 
 sq_status_t launch_w4a4_gemm_decode(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N, int K,
-                                    void* Y, int32_t* accdbg, void* workspace, size_t workspace_bytes, cudaStream_t s) {
-  if (M <= 16) return launch_decode<16>(Xq, sx, Wq, sw, M, N, K, Y, accdbg, workspace, workspace_bytes, s);
-  if (M <= 32) return launch_decode<32>(Xq, sx, Wq, sw, M, N, K, Y, accdbg, workspace, workspace_bytes, s);
-  return launch_decode<64>(Xq, sx, Wq, sw, M, N, K, Y, accdbg, workspace, workspace_bytes, s);
+                                    void* Y, int32_t* accdbg, void*, size_t, cudaStream_t s) {
+  if (M <= 16) return launch_decode<16>(Xq, sx, Wq, sw, M, N, K, Y, accdbg, s);
+  if (M <= 32) return launch_decode<32>(Xq, sx, Wq, sw, M, N, K, Y, accdbg, s);
+  return launch_decode<64>(Xq, sx, Wq, sw, M, N, K, Y, accdbg, s);
 }
 
 }  // namespace sq

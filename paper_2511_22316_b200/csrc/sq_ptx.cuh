@@ -385,6 +385,21 @@ __device__ __forceinline__ void st_f32_peer_and_arrive(float* slot, float v, uin
       "mbarrier.arrive.release.cluster.shared::cluster.b64 _, [rb];\n\t}"
       ::"r"(smem_u32(slot)), "r"(smem_u32(bar)), "f"(v), "r"(rank) : "memory");
 }
+// Address, in the cluster's shared window, of the location at the same offset in CTA `rank`.
+__device__ __forceinline__ uint32_t cluster_map(const void* p, uint32_t rank) {
+  uint32_t r;
+  asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
+  return r;
+}
+__device__ __forceinline__ void st_v4_cluster(uint32_t addr, int32_t a, int32_t b, int32_t c, int32_t d) {
+  asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+}
+// Arrival with cluster-scope release on a barrier given by its address in the cluster's window:
+// the arriving thread's earlier loads and stores (to any CTA's shared memory) happen before
+// whatever a thread does after an acquire wait that sees the arrival.
+__device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t bar_addr) {
+  asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_addr) : "memory");
+}
 __device__ __forceinline__ bool mbar_wait_acq_cluster(uint64_t* bar, uint32_t parity, uint32_t site, uint32_t limit) {
   for (uint32_t it = 0; it < limit; ++it) {
     uint32_t ok;

@@ -269,8 +269,10 @@ GEMM_SHAPES = [
     # tiles per pair and more k-blocks than the operand ring holds
     (129, 128, 128), (256, 256, 128), (200, 136, 384), (384, 520, 1664), (1000, 1288, 896),
     (513, 2304, 2176),
-    # decode kernel (M <= 64, weights as the A operand, split K): all three token-count classes,
-    # ragged channel tile, odd k-block count, the two decode layer shapes
+    # decode kernel (M <= 64, weights as the A operand, K split over a cluster): all three
+    # token-count classes, ragged channel tile, odd k-block count, the two decode layer shapes;
+    # clusters of 2, 4 and 8, and more tiles than the device holds clusters (slots reused)
+    (9, 264, 1280), (64, 640, 2560), (40, 136, 8192), (16, 5120, 14336), (33, 2432, 6144), (64, 5120, 14336),
     # dot-product kernel (M <= 4): odd channel counts, every token-count class
     (2, 1001, 2048), (3, 264, 14336), (4, 7, 96),
     (1, 4096, 4096), (17, 1000, 2048), (33, 384, 1664), (64, 2048, 2304), (4, 14336, 4096), (16, 4096, 14336),
@@ -340,14 +342,15 @@ def test_gemm_prefill_config_sampled_rows(sq):
     assert _fp16_ulps_apart(Y[rows], Yo).max() <= 1
 
 
-def test_gemm_decode_without_workspace_gives_the_same_result(sq):
-    """With no workspace the decode kernel cannot split K; the result must not change."""
+def test_gemm_decode_needs_no_workspace(sq):
+    """The decode kernel splits K over a cluster and exchanges partial tiles on chip: it asks for
+    no workspace and gives the same result with and without one."""
     rng = np.random.default_rng(9)
     M, N, K = 8, 4096, 4096
     Xc, Wc = random_codes(rng, M, K), random_codes(rng, N, K)
     sx = rng.uniform(0.01, 2.0, size=M).astype(np.float16)
     sw = rng.uniform(0.001, 0.1, size=N).astype(np.float16)
-    assert sq.sq_w4a4_gemm_workspace_bytes(M, N, K) > 0
+    assert sq.sq_w4a4_gemm_workspace_bytes(M, N, K) == 0
     Y1, acc1 = run_gemm(sq, Xc, Wc, sx, sw)
     y, a = Guarded(M * N * 2), Guarded(M * N * 4)
     sq.sq_w4a4_gemm(dev(ora.pack_int4(Xc)), dev(sx), dev(ora.pack_int4(Wc)), dev(sw), M, N, K, y, a, None, 0)
