@@ -60,7 +60,7 @@ struct DecSmem {
   static constexpr int OFF_BAR = OFF_RED + D_EPI_GROUPS * RED_GROUP;
   static constexpr int NUM_BARS = 2 * S_ST + 2 * D_S_OP + 2 * D_ACCS + 2 * D_EPI_GROUPS;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
-  static constexpr int TOTAL = OFF_MISC + 32;
+  static constexpr int TOTAL = OFF_MISC + 32 + NT * 4;   // TMEM address, then the tokens' scales as floats
   static constexpr int DYN_BYTES = TOTAL + 1024;
 };
 
@@ -103,6 +103,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   uint64_t* red_full = tmem_empty + D_ACCS;                   // [D_EPI_GROUPS] the others' rows have arrived here
   uint64_t* red_empty = red_full + D_EPI_GROUPS;              // [D_EPI_GROUPS] the others have read what this CTA sent
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
+  float* sxs = reinterpret_cast<float*>(smem + L::OFF_MISC + 32);   // [NT], zero beyond M
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = K / 128;
@@ -118,15 +119,17 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   const int b1 = static_cast<int>(static_cast<long long>(crank + 1) * num_sb / splits);
 
   // The producer's walk over (tile, block); `budget` blocks are issued per call (waiting for the
-  // staging stage of each).  The weights do not depend on the kernel before this one, the tokens
-  // do: with `defer_x` only the weights are requested and the blocks are noted in pre_sb.
+  // staging stage of each, except on the first lap of the ring, when every stage is free and the
+  // "empty" barriers may not exist yet).  The weights do not depend on the kernel before this
+  // one, the tokens do: with `defer_x` only the weights are requested and the blocks are noted.
   int p_tile = cid, p_sb = b0, pre_n = 0;
   int pre_sb[S_ST];
   uint32_t p_it = 0;
   auto produce = [&](uint32_t budget, bool defer_x) -> bool {
     while (budget > 0 && p_tile < tiles) {
       const int ss = p_it % S_ST;
-      if (!mbar_wait(&st_empty[ss], ((p_it / S_ST) & 1) ^ 1, DSITE_ST_EMPTY, limit)) return false;
+      if (p_it >= static_cast<uint32_t>(S_ST) &&
+          !mbar_wait(&st_empty[ss], ((p_it / S_ST) & 1) ^ 1, DSITE_ST_EMPTY, limit)) return false;
       mbar_arrive_expect_tx(&st_full[ss], L::W_ST + L::X_ST);
       tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, &tmap_w, &st_full[ss], p_sb * 128, p_tile * 128);
       if (defer_x) pre_sb[pre_n++] = p_sb;
@@ -142,12 +145,12 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   };
 
   if (threadIdx.x == 0) {
-    tma_prefetch_desc(&tmap_w);
+    // First of all the weights of the whole staging ring: nothing else is on the critical path.
+    for (int s = 0; s < S_ST; ++s) mbar_init(&st_full[s], 1);
+    mbar_fence_init();
+    produce(S_ST, true);
     tma_prefetch_desc(&tmap_x);
-    for (int s = 0; s < S_ST; ++s) {
-      mbar_init(&st_full[s], 1);
-      mbar_init(&st_empty[s], 6);                      // one converter group + one unpacker group
-    }
+    for (int s = 0; s < S_ST; ++s) mbar_init(&st_empty[s], 6);   // one converter group + one unpacker group
     for (int s = 0; s < D_S_OP; ++s) {
       mbar_init(&full[s], 6);
       mbar_init(&empty[s], 1);
@@ -156,14 +159,14 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
       mbar_init(&tmem_full[b], 1);
       mbar_init(&tmem_empty[b], 4);
     }
-    // One arrival per row that crosses CTAs: (s - 1) sources x 128 / s rows, both ways.
+    // red_full: armed by one thread with the bytes that cross into this CTA; red_empty: one
+    // arrival per row that crossed out of it, (s - 1) readers x 128 / s rows.
     const uint32_t crossing = splits > 1 ? static_cast<uint32_t>((splits - 1) * (128 / splits)) : 1u;
     for (int g = 0; g < D_EPI_GROUPS; ++g) {
-      mbar_init(&red_full[g], crossing);
+      mbar_init(&red_full[g], 1);
       mbar_init(&red_empty[g], crossing);
     }
     mbar_fence_init();
-    produce(S_ST, true);                               // the weights of the whole staging ring, before anyone else is ready
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, 512);
@@ -171,7 +174,9 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   }
   tc_fence_before_sync();
   __syncthreads();
-  if (splits > 1) cluster_sync_all();                  // every CTA's barriers exist before anyone arrives on them
+  // Every CTA's barriers must exist before another CTA stores or arrives on them: only the
+  // epilogue warps do that, so only they wait here; the others pick the barrier up at the end.
+  if (splits > 1) cluster_arrive_release();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
   griddep_wait();                                      // the tokens and their scales come from the kernel before
@@ -285,6 +290,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     // ------------------------------ epilogue groups -----------------------------------------------
     const int q = warp & 3;
     const int eg = (warp - (2 + D_A_WARPS + D_B_WARPS)) >> 2;        // this group takes tiles eg, eg + 2, ... of the CTA's
+    const int et = static_cast<int>(threadIdx.x) - (2 + D_A_WARPS + D_B_WARPS) * 32;   // 0 .. 255
     const int rowl = q * 32 + lane;                                  // row of the tile = TMEM lane
     // Reduce-scatter geometry: CTA `owner` finishes this thread's row; this CTA finishes the rows
     // [crank * rows_per, (crank + 1) * rows_per).  Slots are [source][4-column chunk][row][4] int32:
@@ -299,18 +305,24 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     const uint32_t my_slot = crank < owner ? crank : crank - 1u;     // this CTA's slot in `owner`'s buffer
     const uint32_t send_addr = mine ? 0u : cluster_map(red, owner) + ((my_slot * (NT / 4)) * rows_per + rloc) * 16u;
     const uint32_t send_bar = mine ? 0u : cluster_map(&red_full[eg], owner);
+    const uint32_t red_bytes = static_cast<uint32_t>((splits - 1) * rows_per * NT * 4);   // what crosses into this CTA per tile
+    // The tokens' scales as floats (zero beyond M): read once, before any accumulator is ready.
+    if (et < NT) sxs[et] = (et < M) ? __half2float(sx[et]) : 0.0f;
+    named_barrier(1, D_EPI_WARPS * 32);
+    if (splits > 1) cluster_wait_acquire();                            // the other CTAs' barriers exist
     bool ok = true;
     uint32_t icount = 0;
     for (int tile = cid; tile < tiles && ok; tile += ncl, ++icount) {
       if ((icount % D_EPI_GROUPS) != static_cast<uint32_t>(eg)) continue;
       const uint32_t acc = icount % D_ACCS;
       const uint32_t g = icount / D_EPI_GROUPS;                      // the group's tile count
+      const int ch = tile * 128 + rowl;                    // output channel of this thread
+      const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;      // in flight while the accumulator is awaited
+      if (splits > 1 && mine && rloc == 0) mbar_arrive_expect_tx(&red_full[eg], red_bytes);
       ok = mbar_wait(&tmem_full[acc], (icount / D_ACCS) & 1, DSITE_TMEM_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t tmem_d = tmem_base + acc * NT + (static_cast<uint32_t>(q * 32) << 16);
-      const int ch = tile * 128 + rowl;                    // output channel of this thread
-      const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;
       if (warp_sends) {
         // This CTA's chunk of K for rows that another CTA finishes: into that CTA's slot, once it
         // has read what was sent for the group's previous tile.
@@ -326,12 +338,12 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
           if (!mine) {
 #pragma unroll
             for (int c = 0; c < 4; ++c)
-              st_v4_cluster(send_addr + static_cast<uint32_t>((4 * c16 + c) * rows_per) * 16u,
-                            static_cast<int32_t>(r[4 * c]) >> 8, static_cast<int32_t>(r[4 * c + 1]) >> 8,
-                            static_cast<int32_t>(r[4 * c + 2]) >> 8, static_cast<int32_t>(r[4 * c + 3]) >> 8);
+              st_async_v4_cluster(send_addr + static_cast<uint32_t>((4 * c16 + c) * rows_per) * 16u,
+                                  static_cast<int32_t>(r[4 * c]) >> 8, static_cast<int32_t>(r[4 * c + 1]) >> 8,
+                                  static_cast<int32_t>(r[4 * c + 2]) >> 8, static_cast<int32_t>(r[4 * c + 3]) >> 8,
+                                  send_bar);
           }
         }
-        if (!mine) mbar_arrive_release_cluster(send_bar);
       }
       if (!warp_owns) {                                      // nothing to finish here: hand the accumulator back
         tc_fence_before_sync();
@@ -366,19 +378,27 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
             const int4 v = slot[sp * (NT / 4) * rows_per];
             a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
           }
+          const int e0 = 16 * c16 + 4 * c;
+          const float4 s4 = *reinterpret_cast<const float4*>(sxs + e0);
           const int32_t av[4] = {a.x, a.y, a.z, a.w};
+          const float sv[4] = {s4.x, s4.y, s4.z, s4.w};
+          __half h[4];
 #pragma unroll
-          for (int x = 0; x < 4; ++x) {
-            const int e = 16 * c16 + 4 * c + x;
-            if (e < M && ch < N) {
-              const float f = __int_as_float(0x4B400000 + av[x]) - 12582912.0f;
-              Y[static_cast<size_t>(e) * N + ch] = __float2half_rn(f * (__half2float(__ldg(sx + e)) * swv));
-              if (accdbg) accdbg[static_cast<size_t>(e) * N + ch] = av[x];
+          for (int x = 0; x < 4; ++x)
+            h[x] = __float2half_rn((__int_as_float(0x4B400000 + av[x]) - 12582912.0f) * (sv[x] * swv));
+          if (ch < N) {
+#pragma unroll
+            for (int x = 0; x < 4; ++x) {
+              if (e0 + x < M) {
+                Y[static_cast<size_t>(e0 + x) * N + ch] = h[x];
+                if (accdbg) accdbg[static_cast<size_t>(e0 + x) * N + ch] = av[x];
+              }
             }
           }
         }
       }
-      if (splits > 1 && mine) {                              // the slots may be rewritten
+      // The slots may be rewritten -- if the group has another tile (nobody waits otherwise).
+      if (splits > 1 && mine && tile + D_EPI_GROUPS * ncl < tiles) {
         for (uint32_t d = 0; d < static_cast<uint32_t>(splits); ++d)
           if (d != crank) mbar_arrive_release_cluster(cluster_map(&red_empty[eg], d));
       }
@@ -387,10 +407,16 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
 
   tc_fence_before_sync();
   __syncthreads();
-  if (splits > 1) cluster_sync_all();                  // nobody leaves while another CTA may still write or arrive here
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, 512);
+  }
+  if (splits > 1) {
+    // Nobody leaves while another CTA may still store or arrive here.  No memory is ordered by
+    // this barrier: what crossed CTAs was handed over by the red_* barriers.
+    if (warp < 2 + D_A_WARPS + D_B_WARPS) cluster_wait_acquire();      // the set-up barrier, long complete
+    cluster_arrive_relaxed();
+    cluster_wait_acquire();
   }
 }
 

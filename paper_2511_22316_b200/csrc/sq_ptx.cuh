@@ -314,6 +314,17 @@ __device__ __forceinline__ void mbar_arrive_cluster(uint64_t* bar, uint32_t rank
 __device__ __forceinline__ void cluster_sync_all() {
   asm volatile("barrier.cluster.arrive.release.aligned;\n\tbarrier.cluster.wait.acquire.aligned;" ::: "memory");
 }
+// The two halves of the cluster barrier.  A thread alternates arrive and wait; work between the
+// two overlaps the other CTAs' way to the barrier.  The relaxed arrival orders no memory.
+__device__ __forceinline__ void cluster_arrive_release() {
+  asm volatile("barrier.cluster.arrive.release.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_arrive_relaxed() {
+  asm volatile("barrier.cluster.arrive.relaxed.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void cluster_wait_acquire() {
+  asm volatile("barrier.cluster.wait.acquire.aligned;" ::: "memory");
+}
 __device__ __forceinline__ void tmem_alloc_pair(uint32_t* smem_result, uint32_t ncols) {
   asm volatile("tcgen05.alloc.cta_group::2.sync.aligned.shared::cta.b32 [%0], %1;"
                ::"r"(smem_u32(smem_result)), "r"(ncols) : "memory");
@@ -391,12 +402,17 @@ __device__ __forceinline__ uint32_t cluster_map(const void* p, uint32_t rank) {
   asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(smem_u32(p)), "r"(rank));
   return r;
 }
-__device__ __forceinline__ void st_v4_cluster(uint32_t addr, int32_t a, int32_t b, int32_t c, int32_t d) {
-  asm volatile("st.shared::cluster.v4.b32 [%0], {%1, %2, %3, %4};" ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d) : "memory");
+// Asynchronous 16-byte store into another CTA's shared memory (address in the cluster's window)
+// that, once performed, takes its 16 bytes off the transaction count of the barrier `bar_addr` in
+// the same CTA: a thread that has waited for that barrier's phase sees the data.
+__device__ __forceinline__ void st_async_v4_cluster(uint32_t addr, int32_t a, int32_t b, int32_t c, int32_t d,
+                                                    uint32_t bar_addr) {
+  asm volatile("st.async.weak.shared::cluster.mbarrier::complete_tx::bytes.v4.b32 [%0], {%1, %2, %3, %4}, [%5];"
+               ::"r"(addr), "r"(a), "r"(b), "r"(c), "r"(d), "r"(bar_addr) : "memory");
 }
 // Arrival with cluster-scope release on a barrier given by its address in the cluster's window:
-// the arriving thread's earlier loads and stores (to any CTA's shared memory) happen before
-// whatever a thread does after an acquire wait that sees the arrival.
+// the arriving thread's earlier loads and stores happen before whatever a thread does after an
+// acquire wait that sees the arrival.
 __device__ __forceinline__ void mbar_arrive_release_cluster(uint32_t bar_addr) {
   asm volatile("mbarrier.arrive.release.cluster.shared::cluster.b64 _, [%0];" ::"r"(bar_addr) : "memory");
 }
