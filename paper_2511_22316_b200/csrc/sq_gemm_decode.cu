@@ -18,8 +18,8 @@
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = two groups of weight
 // converters and warps 10..13 = two groups of token unpackers (a group takes every other block:
 // a block costs a warp several hundred cycles of waits and fences whatever its size), warps
-// 14..21 = two epilogue groups that take the tiles in turn (four accumulators, so epilogues
-// overlap the main loop of the following tiles).
+// 14..21 = epilogue: all eight work on every tile, each on a quarter of the channels and half of
+// the tokens (four accumulators, so the epilogue overlaps the main loop of the following tiles).
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -57,7 +57,8 @@ struct DecSmem {
   static constexpr int OFF_W_ST = OFF_X_OP + D_S_OP * X_OP;
   static constexpr int OFF_X_ST = OFF_W_ST + S_ST * W_ST;
   static constexpr int OFF_RED = OFF_X_ST + S_ST * X_ST;
-  static constexpr int OFF_BAR = OFF_RED + D_EPI_GROUPS * RED_GROUP;
+  static constexpr int OFF_OUT = OFF_RED + D_EPI_GROUPS * RED_GROUP;     // per epilogue warp: 16 tokens x 32 channels fp16
+  static constexpr int OFF_BAR = OFF_OUT + D_EPI_WARPS * 1024;
   static constexpr int NUM_BARS = 2 * S_ST + 2 * D_S_OP + 2 * D_ACCS + 2 * D_EPI_GROUPS;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int TOTAL = OFF_MISC + 32 + NT * 4;   // TMEM address, then the tokens' scales as floats
@@ -100,8 +101,8 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   uint64_t* empty = bars + 2 * S_ST + D_S_OP;
   uint64_t* tmem_full = bars + 2 * S_ST + 2 * D_S_OP;        // [D_ACCS]
   uint64_t* tmem_empty = tmem_full + D_ACCS;                  // [D_ACCS]
-  uint64_t* red_full = tmem_empty + D_ACCS;                   // [D_EPI_GROUPS] the others' rows have arrived here
-  uint64_t* red_empty = red_full + D_EPI_GROUPS;              // [D_EPI_GROUPS] the others have read what this CTA sent
+  uint64_t* red_full = tmem_empty + D_ACCS;                   // [2] the others' rows have arrived in buffer 0 / 1
+  uint64_t* red_empty = red_full + D_EPI_GROUPS;              // [2] the others have read what this CTA sent there
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
   float* sxs = reinterpret_cast<float*>(smem + L::OFF_MISC + 32);   // [NT], zero beyond M
 
@@ -157,11 +158,11 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     }
     for (int b = 0; b < D_ACCS; ++b) {
       mbar_init(&tmem_full[b], 1);
-      mbar_init(&tmem_empty[b], 4);
+      mbar_init(&tmem_empty[b], D_EPI_WARPS);
     }
     // red_full: armed by one thread with the bytes that cross into this CTA; red_empty: one
-    // arrival per row that crossed out of it, (s - 1) readers x 128 / s rows.
-    const uint32_t crossing = splits > 1 ? static_cast<uint32_t>((splits - 1) * (128 / splits)) : 1u;
+    // arrival per epilogue group and row that crossed out of it, (s - 1) readers x 128 / s rows.
+    const uint32_t crossing = splits > 1 ? static_cast<uint32_t>(D_EPI_GROUPS * (splits - 1) * (128 / splits)) : 1u;
     for (int g = 0; g < D_EPI_GROUPS; ++g) {
       mbar_init(&red_full[g], 1);
       mbar_init(&red_empty[g], crossing);
@@ -287,25 +288,37 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
       }
     }
   } else {
-    // ------------------------------ epilogue groups -----------------------------------------------
+    // ------------------------------ epilogue ------------------------------------------------------
+    // Eight warps share every tile: warp q of group eg reads the TMEM lanes 32 q .. 32 q + 31 (all a
+    // warp may touch) of the columns [eg * NT / 2, (eg + 1) * NT / 2) -- a single warp per scheduler
+    // is bound by its own instruction issue, so the columns are spread over as many as there are.
+    constexpr int HALF = NT / 2;                                     // columns (tokens) per group
+    constexpr int CH = HALF >= 16 ? 16 : 8;                          // columns per TMEM load
     const int q = warp & 3;
-    const int eg = (warp - (2 + D_A_WARPS + D_B_WARPS)) >> 2;        // this group takes tiles eg, eg + 2, ... of the CTA's
+    const int eg = (warp - (2 + D_A_WARPS + D_B_WARPS)) >> 2;
     const int et = static_cast<int>(threadIdx.x) - (2 + D_A_WARPS + D_B_WARPS) * 32;   // 0 .. 255
     const int rowl = q * 32 + lane;                                  // row of the tile = TMEM lane
     // Reduce-scatter geometry: CTA `owner` finishes this thread's row; this CTA finishes the rows
     // [crank * rows_per, (crank + 1) * rows_per).  Slots are [source][4-column chunk][row][4] int32:
-    // a warp's 16-byte accesses are contiguous.
+    // a warp's 16-byte accesses are contiguous.  Two buffers, used by the CTA's tiles in turn.
     const int rows_per = 128 / splits;
     const uint32_t owner = static_cast<uint32_t>(rowl / rows_per);
     const int rloc = rowl % rows_per;
     const bool mine = (owner == crank);
     const bool warp_owns = __any_sync(0xFFFFFFFFu, mine);
     const bool warp_sends = __any_sync(0xFFFFFFFFu, !mine);
-    unsigned char* red = smem + L::OFF_RED + eg * L::RED_GROUP;
     const uint32_t my_slot = crank < owner ? crank : crank - 1u;     // this CTA's slot in `owner`'s buffer
-    const uint32_t send_addr = mine ? 0u : cluster_map(red, owner) + ((my_slot * (NT / 4)) * rows_per + rloc) * 16u;
-    const uint32_t send_bar = mine ? 0u : cluster_map(&red_full[eg], owner);
+    const uint32_t send_base = mine ? 0u : cluster_map(smem + L::OFF_RED, owner) + ((my_slot * (NT / 4)) * rows_per + rloc) * 16u;
+    const uint32_t send_bar0 = mine ? 0u : cluster_map(&red_full[0], owner);
     const uint32_t red_bytes = static_cast<uint32_t>((splits - 1) * rows_per * NT * 4);   // what crosses into this CTA per tile
+    // Output staging of this warp: the accumulator has one channel per thread and the tokens along
+    // its registers, Y has the channels contiguous.  A chunk of CH tokens x 32 channels is turned in
+    // shared memory -- written as words of two tokens, [token pair][channel] -- so that a thread
+    // stores 8 channels (16 bytes) of one token.
+    uint32_t* outw = reinterpret_cast<uint32_t*>(smem + L::OFF_OUT + (warp - (2 + D_A_WARPS + D_B_WARPS)) * 1024);
+    const int piece = lane & 3, prow = lane >> 2;                    // reader: channels 8 * piece .., token prow (+ 8)
+    const bool piece_mine = static_cast<uint32_t>((q * 32 + piece * 8) / rows_per) == crank;
+    const uint32_t pick = (prow & 1) ? 0x7632u : 0x5410u;            // the odd or the even token of a pair
     // The tokens' scales as floats (zero beyond M): read once, before any accumulator is ready.
     if (et < NT) sxs[et] = (et < M) ? __half2float(sx[et]) : 0.0f;
     named_barrier(1, D_EPI_WARPS * 32);
@@ -313,35 +326,35 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     bool ok = true;
     uint32_t icount = 0;
     for (int tile = cid; tile < tiles && ok; tile += ncl, ++icount) {
-      if ((icount % D_EPI_GROUPS) != static_cast<uint32_t>(eg)) continue;
       const uint32_t acc = icount % D_ACCS;
-      const uint32_t g = icount / D_EPI_GROUPS;                      // the group's tile count
+      const uint32_t par = icount & 1u, g = icount >> 1;             // reduce buffer and its use count
       const int ch = tile * 128 + rowl;                    // output channel of this thread
       const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;      // in flight while the accumulator is awaited
-      if (splits > 1 && mine && rloc == 0) mbar_arrive_expect_tx(&red_full[eg], red_bytes);
+      if (splits > 1 && eg == 0 && mine && rloc == 0) mbar_arrive_expect_tx(&red_full[par], red_bytes);
       ok = mbar_wait(&tmem_full[acc], (icount / D_ACCS) & 1, DSITE_TMEM_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t tmem_d = tmem_base + acc * NT + (static_cast<uint32_t>(q * 32) << 16);
+      const uint32_t tmem_d = tmem_base + acc * NT + eg * HALF + (static_cast<uint32_t>(q * 32) << 16);
       if (warp_sends) {
         // This CTA's chunk of K for rows that another CTA finishes: into that CTA's slot, once it
-        // has read what was sent for the group's previous tile.
-        if (!mine) ok = mbar_wait_acq_cluster(&red_empty[eg], (g & 1) ^ 1, DSITE_RED_EMPTY, limit);
+        // has read what was sent two tiles ago.
+        if (!mine) ok = mbar_wait_acq_cluster(&red_empty[par], (g & 1) ^ 1, DSITE_RED_EMPTY, limit);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
+        const uint32_t dst = send_base + par * L::RED_GROUP, bar = send_bar0 + par * 8u;
 #pragma unroll
-        for (int c16 = 0; c16 < NT / 16; ++c16) {
-          uint32_t r[16];
+        for (int k = 0; k < HALF / CH; ++k) {
+          uint32_t r[CH];
           __syncwarp();
-          tmem_ld_32x32b_x16(tmem_d + 16 * c16, r);
+          if constexpr (CH == 16) tmem_ld_32x32b_x16(tmem_d + CH * k, r);
+          else tmem_ld_32x32b_x8(tmem_d + CH * k, r);
           tmem_wait_ld();
           if (!mine) {
 #pragma unroll
-            for (int c = 0; c < 4; ++c)
-              st_async_v4_cluster(send_addr + static_cast<uint32_t>((4 * c16 + c) * rows_per) * 16u,
+            for (int c = 0; c < CH / 4; ++c)
+              st_async_v4_cluster(dst + static_cast<uint32_t>(((eg * HALF + CH * k) / 4 + c) * rows_per) * 16u,
                                   static_cast<int32_t>(r[4 * c]) >> 8, static_cast<int32_t>(r[4 * c + 1]) >> 8,
-                                  static_cast<int32_t>(r[4 * c + 2]) >> 8, static_cast<int32_t>(r[4 * c + 3]) >> 8,
-                                  send_bar);
+                                  static_cast<int32_t>(r[4 * c + 2]) >> 8, static_cast<int32_t>(r[4 * c + 3]) >> 8, bar);
           }
         }
       }
@@ -352,55 +365,72 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
         continue;
       }
       if (splits > 1) {
-        if (mine) ok = mbar_wait_acq_cluster(&red_full[eg], g & 1, DSITE_RED_FULL, limit);
+        if (mine) ok = mbar_wait_acq_cluster(&red_full[par], g & 1, DSITE_RED_FULL, limit);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
       }
+      const int4* red = reinterpret_cast<const int4*>(smem + L::OFF_RED + par * L::RED_GROUP);
 #pragma unroll
-      for (int c16 = 0; c16 < NT / 16; ++c16) {
-        uint32_t r[16];
+      for (int k = 0; k < HALF / CH; ++k) {
+        uint32_t r[CH];
         __syncwarp();
-        tmem_ld_32x32b_x16(tmem_d + 16 * c16, r);
+        if constexpr (CH == 16) tmem_ld_32x32b_x16(tmem_d + CH * k, r);
+        else tmem_ld_32x32b_x8(tmem_d + CH * k, r);
         tmem_wait_ld();
-        if (c16 == NT / 16 - 1) {                          // last read: hand the accumulator back
+        if (k == HALF / CH - 1) {                          // last read: hand the accumulator back
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive(&tmem_empty[acc]);
         }
-        if (!mine) continue;
+        const int t0 = eg * HALF + CH * k;                 // first token of the chunk
+        if (mine) {
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-          // exact: the accumulator is 256 * (sum of products)
-          int4 a = make_int4(static_cast<int32_t>(r[4 * c]) >> 8, static_cast<int32_t>(r[4 * c + 1]) >> 8,
-                             static_cast<int32_t>(r[4 * c + 2]) >> 8, static_cast<int32_t>(r[4 * c + 3]) >> 8);
-          const int4* slot = reinterpret_cast<const int4*>(red) + (4 * c16 + c) * rows_per + rloc;
-          for (int sp = 0; sp + 1 < splits; ++sp) {
-            const int4 v = slot[sp * (NT / 4) * rows_per];
-            a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
-          }
-          const int e0 = 16 * c16 + 4 * c;
-          const float4 s4 = *reinterpret_cast<const float4*>(sxs + e0);
-          const int32_t av[4] = {a.x, a.y, a.z, a.w};
-          const float sv[4] = {s4.x, s4.y, s4.z, s4.w};
-          __half h[4];
+          for (int c = 0; c < CH / 4; ++c) {
+            // exact: the accumulator is 256 * (sum of products)
+            int4 a = make_int4(static_cast<int32_t>(r[4 * c]) >> 8, static_cast<int32_t>(r[4 * c + 1]) >> 8,
+                               static_cast<int32_t>(r[4 * c + 2]) >> 8, static_cast<int32_t>(r[4 * c + 3]) >> 8);
+            const int4* slot = red + (t0 / 4 + c) * rows_per + rloc;
+            for (int sp = 0; sp + 1 < splits; ++sp) {
+              const int4 v = slot[sp * (NT / 4) * rows_per];
+              a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+            }
+            const int e0 = t0 + 4 * c;
+            const float4 s4 = *reinterpret_cast<const float4*>(sxs + e0);
+            const __half2 h01 = __floats2half2_rn((__int_as_float(0x4B400000 + a.x) - 12582912.0f) * (s4.x * swv),
+                                                  (__int_as_float(0x4B400000 + a.y) - 12582912.0f) * (s4.y * swv));
+            const __half2 h23 = __floats2half2_rn((__int_as_float(0x4B400000 + a.z) - 12582912.0f) * (s4.z * swv),
+                                                  (__int_as_float(0x4B400000 + a.w) - 12582912.0f) * (s4.w * swv));
+            outw[(2 * c) * 32 + lane] = *reinterpret_cast<const uint32_t*>(&h01);
+            outw[(2 * c + 1) * 32 + lane] = *reinterpret_cast<const uint32_t*>(&h23);
+            if (accdbg && ch < N) {
+              const int32_t av[4] = {a.x, a.y, a.z, a.w};
 #pragma unroll
-          for (int x = 0; x < 4; ++x)
-            h[x] = __float2half_rn((__int_as_float(0x4B400000 + av[x]) - 12582912.0f) * (sv[x] * swv));
-          if (ch < N) {
-#pragma unroll
-            for (int x = 0; x < 4; ++x) {
-              if (e0 + x < M) {
-                Y[static_cast<size_t>(e0 + x) * N + ch] = h[x];
-                if (accdbg) accdbg[static_cast<size_t>(e0 + x) * N + ch] = av[x];
-              }
+              for (int x = 0; x < 4; ++x)
+                if (e0 + x < M) accdbg[static_cast<size_t>(e0 + x) * N + ch] = av[x];
             }
           }
         }
+        __syncwarp();
+        {
+          const int ch0 = tile * 128 + q * 32 + piece * 8;
+#pragma unroll
+          for (int pass = 0; pass < CH / 8; ++pass) {
+            const int e = t0 + 8 * pass + prow;
+            const uint4* src = reinterpret_cast<const uint4*>(outw + (4 * pass + (prow >> 1)) * 32 + piece * 8);
+            const uint4 w0 = src[0], w1 = src[1];
+            uint4 v;
+            v.x = __byte_perm(w0.x, w0.y, pick);
+            v.y = __byte_perm(w0.z, w0.w, pick);
+            v.z = __byte_perm(w1.x, w1.y, pick);
+            v.w = __byte_perm(w1.z, w1.w, pick);
+            if (piece_mine && e < M && ch0 < N) *reinterpret_cast<uint4*>(Y + static_cast<size_t>(e) * N + ch0) = v;
+          }
+        }
       }
-      // The slots may be rewritten -- if the group has another tile (nobody waits otherwise).
-      if (splits > 1 && mine && tile + D_EPI_GROUPS * ncl < tiles) {
+      // The slots may be rewritten -- if the CTA has another tile for this buffer (nobody waits otherwise).
+      if (splits > 1 && mine && tile + 2 * ncl < tiles) {
         for (uint32_t d = 0; d < static_cast<uint32_t>(splits); ++d)
-          if (d != crank) mbar_arrive_release_cluster(cluster_map(&red_empty[eg], d));
+          if (d != crank) mbar_arrive_release_cluster(cluster_map(&red_empty[par], d));
       }
     }
   }
