@@ -116,8 +116,8 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   // of it accumulates the blocks [b0, b1) of every one of them.
   const uint32_t crank = (splits > 1) ? cluster_ctarank() : 0u;
   const int cid = static_cast<int>(blockIdx.x) / splits, ncl = static_cast<int>(gridDim.x) / splits;
-  const int b0 = static_cast<int>(static_cast<long long>(crank) * num_sb / splits);
-  const int b1 = static_cast<int>(static_cast<long long>(crank + 1) * num_sb / splits);
+  const int b0 = static_cast<int>(crank * static_cast<uint32_t>(num_sb) / static_cast<uint32_t>(splits));
+  const int b1 = static_cast<int>((crank + 1u) * static_cast<uint32_t>(num_sb) / static_cast<uint32_t>(splits));
 
   // The producer's walk over (tile, block); `budget` blocks are issued per call (waiting for the
   // staging stage of each, except on the first lap of the ring, when every stage is free and the
@@ -389,10 +389,20 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
             // exact: the accumulator is 256 * (sum of products)
             int4 a = make_int4(static_cast<int32_t>(r[4 * c]) >> 8, static_cast<int32_t>(r[4 * c + 1]) >> 8,
                                static_cast<int32_t>(r[4 * c + 2]) >> 8, static_cast<int32_t>(r[4 * c + 3]) >> 8);
+            // The other CTAs' partial sums, four loads in flight at a time.
             const int4* slot = red + (t0 / 4 + c) * rows_per + rloc;
-            for (int sp = 0; sp + 1 < splits; ++sp) {
-              const int4 v = slot[sp * (NT / 4) * rows_per];
-              a.x += v.x; a.y += v.y; a.z += v.z; a.w += v.w;
+#pragma unroll
+            for (int h = 0; h < D_MAX_SPLITS - 1; h += 4) {
+              if (h + 1 < splits) {
+                int4 v[4];
+#pragma unroll
+                for (int sp = 0; sp < 4; ++sp)
+                  v[sp] = (h + sp + 1 < splits) ? slot[(h + sp) * (NT / 4) * rows_per] : make_int4(0, 0, 0, 0);
+#pragma unroll
+                for (int sp = 0; sp < 4; ++sp) {
+                  a.x += v[sp].x; a.y += v[sp].y; a.z += v[sp].z; a.w += v[sp].w;
+                }
+              }
             }
             const int e0 = t0 + 4 * c;
             const float4 s4 = *reinterpret_cast<const float4*>(sxs + e0);
