@@ -40,7 +40,8 @@ INT8_OVER_BF16 = 2.0      # nominal dense ratio (4.5 POPS int8 : 2.25 PFLOP/s bf
 NCU_TRAFFIC = {
     ("gemm", "llama2_7b_qkvo_prefill"): 12629504,           # w4a4_gemm_pair_kernel: reads (Y stays in L2)
     ("rotate_quant", "llama2_7b_qkvo_prefill"): 16887040,   # rotate_quant_tc_kernel
-    ("gemm", "llama3_8b_up_decode_m16"): 29469184,          # w4a4_gemm_decode_kernel
+    ("gemm", "llama3_8b_up_decode_m16"): 29457920,          # w4a4_gemm_decode_kernel, K not split
+    ("gemm", "llama3_8b_down_decode_m16"): 29518848,        # w4a4_gemm_decode_kernel, K over clusters of 4
     ("gemm", "llama3_8b_up_decode_m1"): 29409280,           # w4a4_gemv_kernel
     ("rotate_quant", "llama2_7b_down_prefill"): 45398528,   # rotate_quant_pair_kernel
 }
@@ -76,9 +77,10 @@ def gemm_bytes(w):
 def gemm_kernel_name(w):
     """The kernel sq_w4a4_gemm picks for this shape (mirrors the library's dispatch)."""
     fast = w.K % 128 == 0 and w.N % 8 == 0
-    if w.M <= 4 and w.K % 32 == 0 and w.K <= 32768:
+    decode = fast and w.M <= 64 and w.N >= 128 and w.K >= 256
+    if w.M <= 4 and w.K % 32 == 0 and w.K <= 32768 and (w.M <= 2 or not decode):
         return "w4a4_gemv_kernel"
-    if fast and w.M <= 64 and w.N >= 128 and w.K >= 256:
+    if decode:
         return "w4a4_gemm_decode_kernel"
     if fast and w.M > 128 and w.N >= 128:
         return "w4a4_gemm_pair_kernel"

@@ -375,15 +375,22 @@ sq_status_t launch_tc(const void* Xq, const void* sx, const void* Wq, const void
 
 }  // namespace
 
+// One or two tokens are pure streaming: dot products on the CUDA cores.  With three or four the
+// dot-product kernel is bound by its dp4a and shared-memory issue and the tensor-core decode kernel
+// (whose time does not depend on M up to 16) is as fast or faster, where it supports the shape.
+static bool use_gemv(int64_t M, int64_t N, int64_t K) {
+  return gemv_supported(M, N, K) && (M <= 2 || !gemm_decode_supported(M, N, K));
+}
+
 size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
-  return gemv_supported(M, N, K) ? 0 : gemm_decode_workspace_bytes(M, N, K);
+  return use_gemv(M, N, K) ? 0 : gemm_decode_workspace_bytes(M, N, K);
 }
 
 sq_status_t launch_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw, int64_t M, int64_t N,
                              int64_t K, void* Y, int32_t* accdbg, void* workspace, size_t workspace_bytes,
                              cudaStream_t s) {
   if (M == 0 || N == 0) return SQ_OK;
-  if (gemv_supported(M, N, K)) return launch_w4a4_gemv(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
+  if (use_gemv(M, N, K)) return launch_w4a4_gemv(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
   if (gemm_decode_supported(M, N, K))
     return launch_w4a4_gemm_decode(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, workspace, workspace_bytes, s);
   const bool tc_ok = (K % BK == 0) && (N % 8 == 0) && K >= BK;

@@ -273,8 +273,9 @@ GEMM_SHAPES = [
     # token-count classes, ragged channel tile, odd k-block count, the two decode layer shapes;
     # clusters of 2, 4 and 8, and more tiles than the device holds clusters (slots reused)
     (9, 264, 1280), (64, 640, 2560), (40, 136, 8192), (16, 5120, 14336), (33, 2432, 6144), (64, 5120, 14336),
-    # dot-product kernel (M <= 4): odd channel counts, every token-count class
-    (2, 1001, 2048), (3, 264, 14336), (4, 7, 96),
+    # dot-product kernel (M <= 2, and M <= 4 where the decode kernel does not take the shape): odd
+    # channel counts, every token-count class
+    (2, 1001, 2048), (2, 264, 14336), (3, 1001, 2048), (4, 7, 96), (3, 264, 14336),
     (1, 4096, 4096), (17, 1000, 2048), (33, 384, 1664), (64, 2048, 2304), (4, 14336, 4096), (16, 4096, 14336),
 ]
 
