@@ -65,23 +65,32 @@ struct DecSmem {
   static constexpr int DYN_BYTES = TOTAL + 1024;
 };
 
-// Widens the 128 staged bytes of `rows` token rows into two int8 k-block tiles (rows x 128 B each,
-// 128-byte swizzle), same byte order as unpack_tile.  Task = (row, 16-byte chunk).
+// Widens the 128 staged bytes of NT token rows into two int8 k-block tiles (NT x 128 B each,
+// 128-byte swizzle), same byte order as unpack_tile.  64 threads: thread t takes NT / 8 16-byte
+// chunks of row t % NT, all loads first.  `second` false: only the first k-block is there.
+template <int NT>
 __device__ __forceinline__ void unpack_rows(const unsigned char* __restrict__ st, unsigned char* __restrict__ op,
-                                            int rows, int t, int nthreads, bool second) {
-  const int ntask = rows * (second ? 8 : 4);
-  for (int task = t; task < ntask; task += nthreads) {
-    const int r = task % rows, c = task / rows;          // c: chunk of the staged row (0..7)
-    const int h = c >> 2, j = c & 3, sw = r & 7;
-    const uint4 w = *reinterpret_cast<const uint4*>(st + r * 128 + ((c ^ sw) << 4));
-    uint4 lo, hi;
-    lo.x = (w.x << 4) & 0xF0F0F0F0u; hi.x = w.x & 0xF0F0F0F0u;
-    lo.y = (w.y << 4) & 0xF0F0F0F0u; hi.y = w.y & 0xF0F0F0F0u;
-    lo.z = (w.z << 4) & 0xF0F0F0F0u; hi.z = w.z & 0xF0F0F0F0u;
-    lo.w = (w.w << 4) & 0xF0F0F0F0u; hi.w = w.w & 0xF0F0F0F0u;
-    unsigned char* tile = op + h * (rows * 128) + r * 128;
-    *reinterpret_cast<uint4*>(tile + ((j ^ sw) << 4)) = lo;
-    *reinterpret_cast<uint4*>(tile + (((4 + j) ^ sw) << 4)) = hi;
+                                            int t, bool second) {
+  constexpr int CPT = NT / 8;                              // chunks per thread: 2, 4 or 8
+  const int r = t % NT, c0 = (t / NT) * CPT, sw = r & 7;
+  const unsigned char* row = st + r * 128;
+  uint4 w[CPT];
+#pragma unroll
+  for (int i = 0; i < CPT; ++i)
+    if (second || c0 + i < 4) w[i] = *reinterpret_cast<const uint4*>(row + (((c0 + i) ^ sw) << 4));
+#pragma unroll
+  for (int i = 0; i < CPT; ++i) {
+    const int c = c0 + i, h = c >> 2, j = c & 3;
+    if (second || c < 4) {
+      uint4 lo, hi;
+      lo.x = (w[i].x << 4) & 0xF0F0F0F0u; hi.x = w[i].x & 0xF0F0F0F0u;
+      lo.y = (w[i].y << 4) & 0xF0F0F0F0u; hi.y = w[i].y & 0xF0F0F0F0u;
+      lo.z = (w[i].z << 4) & 0xF0F0F0F0u; hi.z = w[i].z & 0xF0F0F0F0u;
+      lo.w = (w[i].w << 4) & 0xF0F0F0F0u; hi.w = w[i].w & 0xF0F0F0F0u;
+      unsigned char* tile = op + h * (NT * 128) + r * 128;
+      *reinterpret_cast<uint4*>(tile + ((j ^ sw) << 4)) = lo;
+      *reinterpret_cast<uint4*>(tile + (((4 + j) ^ sw) << 4)) = hi;
+    }
   }
 }
 
@@ -193,6 +202,11 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     // ------------------------------ MMA issuer --------------------------------------------------
     if (elect_one()) {
       constexpr uint32_t idesc = umma_idesc(/*c=s32*/ 2, /*a=s8*/ 1, /*b=s8*/ 1, 128, NT);
+      // One thread issues every MMA, and each instruction it executes costs it several cycles: the
+      // descriptors are formed once (those of a block differ from the ring's first by constants in
+      // the start-address field, 16-byte units, no carry out of it) and the block's MMAs unrolled.
+      const uint64_t b_desc0 = umma_desc_sw128(smem_u32(smem + L::OFF_X_OP));
+      constexpr uint32_t KB1 = (NT * 128) >> 4;           // second k-block tile of a stage
       uint32_t it = 0, icount = 0;
       bool ok = true;
       for (int tile = cid; tile < tiles && ok; tile += ncl, ++icount) {
@@ -202,17 +216,22 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
         tc_fence_after_sync();
         const uint32_t d_tmem = tmem_base + acc * NT;
         for (int sb = b0; sb < b1; ++sb, ++it) {
-          const int s = it % D_S_OP;
+          const uint32_t s = it % D_S_OP;
           ok = mbar_wait(&full[s], (it / D_S_OP) & 1, DSITE_FULL, limit);
           if (!ok) break;
           tc_fence_after_sync();
           const uint32_t a_tmem = tmem_base + D_A_COL0 + s * 64;
-          const uint32_t b_base = smem_u32(smem + L::OFF_X_OP + s * L::X_OP);
-          const int nk = (2 * sb + 1 < num_kb) ? 8 : 4;
-#pragma unroll 4
-          for (int k = 0; k < nk; ++k)
-            umma_i8_ts(d_tmem, a_tmem + k * 8, umma_desc_sw128(b_base + (k >> 2) * (NT * 128) + (k & 3) * 32), idesc,
-                       (sb > b0 || k > 0) ? 1u : 0u);
+          const uint64_t bd = b_desc0 + static_cast<uint64_t>(s * (L::X_OP >> 4));
+          umma_i8_ts(d_tmem, a_tmem, bd, idesc, sb > b0 ? 1u : 0u);
+          umma_i8_ts(d_tmem, a_tmem + 8, bd + 2, idesc, 1u);
+          umma_i8_ts(d_tmem, a_tmem + 16, bd + 4, idesc, 1u);
+          umma_i8_ts(d_tmem, a_tmem + 24, bd + 6, idesc, 1u);
+          if (2 * sb + 1 < num_kb) {
+            umma_i8_ts(d_tmem, a_tmem + 32, bd + KB1, idesc, 1u);
+            umma_i8_ts(d_tmem, a_tmem + 40, bd + (KB1 + 2), idesc, 1u);
+            umma_i8_ts(d_tmem, a_tmem + 48, bd + (KB1 + 4), idesc, 1u);
+            umma_i8_ts(d_tmem, a_tmem + 56, bd + (KB1 + 6), idesc, 1u);
+          }
           umma_commit(&empty[s]);
         }
         umma_commit(&tmem_full[acc]);
@@ -277,8 +296,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
         ok = mbar_wait(&st_full[ss], (it / S_ST) & 1, DSITE_ST_FULL_B, limit) &&
              mbar_wait(&empty[s], ((it / D_S_OP) & 1) ^ 1, DSITE_EMPTY_B, limit);
         if (!ok) break;
-        unpack_rows(smem + L::OFF_X_ST + ss * L::X_ST, smem + L::OFF_X_OP + s * L::X_OP, NT, t, 64,
-                    2 * sb + 1 < num_kb);
+        unpack_rows<NT>(smem + L::OFF_X_ST + ss * L::X_ST, smem + L::OFF_X_OP + s * L::X_OP, t, 2 * sb + 1 < num_kb);
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) {
