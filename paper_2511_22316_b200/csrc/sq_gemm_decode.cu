@@ -47,7 +47,7 @@ enum DecSite : uint32_t {
 
 template <int NT>
 struct DecSmem {
-  static constexpr int S_ST = NT == 64 ? 4 : 6;      // staging stages (256 channels each)
+  static constexpr int S_ST = NT == 64 ? 5 : 6;      // staging stages (256 channels each)
   static constexpr int W_ST = 128 * 128;             // packed weight rows, two k-blocks
   static constexpr int X_ST = NT * 128;              // packed token rows, two k-blocks
   static constexpr int X_OP = 2 * NT * 128;          // int8 token rows, two k-block tiles
@@ -57,7 +57,7 @@ struct DecSmem {
   static constexpr int OFF_W_ST = OFF_X_OP + D_S_OP * X_OP;
   static constexpr int OFF_X_ST = OFF_W_ST + S_ST * W_ST;
   static constexpr int OFF_RED = OFF_X_ST + S_ST * X_ST;
-  static constexpr int OFF_OUT = OFF_RED + D_EPI_GROUPS * RED_GROUP;     // per epilogue warp: 16 tokens x 32 channels fp16
+  static constexpr int OFF_OUT = OFF_RED + RED_GROUP;     // per epilogue warp: 16 tokens x 32 channels fp16
   static constexpr int OFF_BAR = OFF_OUT + D_EPI_WARPS * 1024;
   static constexpr int NUM_BARS = 2 * S_ST + 2 * D_S_OP + 2 * D_ACCS + 2 * D_EPI_GROUPS;
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
@@ -110,8 +110,8 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   uint64_t* empty = bars + 2 * S_ST + D_S_OP;
   uint64_t* tmem_full = bars + 2 * S_ST + 2 * D_S_OP;        // [D_ACCS]
   uint64_t* tmem_empty = tmem_full + D_ACCS;                  // [D_ACCS]
-  uint64_t* red_full = tmem_empty + D_ACCS;                   // [2] the others' rows have arrived in buffer 0 / 1
-  uint64_t* red_empty = red_full + D_EPI_GROUPS;              // [2] the others have read what this CTA sent there
+  uint64_t* red_full = tmem_empty + D_ACCS;                   // the others' rows have arrived in this CTA's slots (entry 0; entry 1 unused)
+  uint64_t* red_empty = red_full + D_EPI_GROUPS;              // the others have read what this CTA sent them
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
   float* sxs = reinterpret_cast<float*>(smem + L::OFF_MISC + 32);   // [NT], zero beyond M
 
@@ -318,7 +318,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     const int rowl = q * 32 + lane;                                  // row of the tile = TMEM lane
     // Reduce-scatter geometry: CTA `owner` finishes this thread's row; this CTA finishes the rows
     // [crank * rows_per, (crank + 1) * rows_per).  Slots are [source][4-column chunk][row][4] int32:
-    // a warp's 16-byte accesses are contiguous.  Two buffers, used by the CTA's tiles in turn.
+    // a warp's 16-byte accesses are contiguous.  One buffer, reused by the CTA's tiles in turn.
     const int rows_per = 128 / splits;
     const uint32_t owner = static_cast<uint32_t>(rowl / rows_per);
     const int rloc = rowl % rows_per;
@@ -345,7 +345,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     uint32_t icount = 0;
     for (int tile = cid; tile < tiles && ok; tile += ncl, ++icount) {
       const uint32_t acc = icount % D_ACCS;
-      const uint32_t par = icount & 1u, g = icount >> 1;             // reduce buffer and its use count
+      const uint32_t par = 0u, g = icount;                            // reduce buffer and its use count
       const int ch = tile * 128 + rowl;                    // output channel of this thread
       const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;      // in flight while the accumulator is awaited
       if (splits > 1 && eg == 0 && mine && rloc == 0) mbar_arrive_expect_tx(&red_full[par], red_bytes);
@@ -355,7 +355,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
       const uint32_t tmem_d = tmem_base + acc * NT + eg * HALF + (static_cast<uint32_t>(q * 32) << 16);
       if (warp_sends) {
         // This CTA's chunk of K for rows that another CTA finishes: into that CTA's slot, once it
-        // has read what was sent two tiles ago.
+        // has read what was sent for the CTA's previous tile.
         if (!mine) ok = mbar_wait_acq_cluster(&red_empty[par], (g & 1) ^ 1, DSITE_RED_EMPTY, limit);
         ok = __all_sync(0xFFFFFFFFu, ok);
         if (!ok) break;
@@ -455,8 +455,8 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
           }
         }
       }
-      // The slots may be rewritten -- if the CTA has another tile for this buffer (nobody waits otherwise).
-      if (splits > 1 && mine && tile + 2 * ncl < tiles) {
+      // The slots may be rewritten -- if the CTA has another tile (nobody waits otherwise).
+      if (splits > 1 && mine && tile + ncl < tiles) {
         for (uint32_t d = 0; d < static_cast<uint32_t>(splits); ++d)
           if (d != crank) mbar_arrive_release_cluster(cluster_map(&red_empty[par], d));
       }
@@ -511,7 +511,8 @@ int max_clusters(int s, int sms) {
 
 // Chooses the cluster size s in {1, 2, 4, 8} over which K is split.  Cost model (cycles, measured):
 // a block of 256 channels costs the main loop BLOCK_CYCLES; the exchange through shared memory
-// adds SPLIT_CYCLES once; tiles beyond the clusters the device holds at once take further waves.
+// adds SPLIT_CYCLES per tile (the cluster's CTAs meet at every tile); tiles beyond the clusters
+// the device holds at once take further waves.
 template <int NT>
 int choose_splits(int tiles, int blocks, int sms) {
   constexpr double BLOCK_CYCLES = NT == 64 ? 1100.0 : (NT == 32 ? 900.0 : 700.0);
@@ -523,7 +524,7 @@ int choose_splits(int tiles, int blocks, int sms) {
     const int ncl = max_clusters<NT>(s, sms);
     if (ncl <= 0) continue;
     const int waves = (tiles + ncl - 1) / ncl;
-    const double cost = static_cast<double>(waves) * ((blocks + s - 1) / s) * BLOCK_CYCLES + (s > 1 ? SPLIT_CYCLES : 0.0);
+    const double cost = static_cast<double>(waves) * (((blocks + s - 1) / s) * BLOCK_CYCLES + (s > 1 ? SPLIT_CYCLES : 0.0));
     if (s == 1 || cost < best_cost * 0.97) {
       best_cost = cost;
       best = s;
