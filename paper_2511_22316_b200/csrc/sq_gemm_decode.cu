@@ -47,7 +47,8 @@ enum DecSite : uint32_t {
 
 template <int NT>
 struct DecSmem {
-  static constexpr int S_ST = NT == 64 ? 5 : 6;      // staging stages (256 channels each)
+  static constexpr int S_ST = NT == 64 ? 5 : 6;      // staging stages (256 channels each); deeper rings measured no faster
+  static_assert(NT == 16 || NT == 32 || NT == 64, "token-count classes");
   static constexpr int W_ST = 128 * 128;             // packed weight rows, two k-blocks
   static constexpr int X_ST = NT * 128;              // packed token rows, two k-blocks
   static constexpr int X_OP = 2 * NT * 128;          // int8 token rows, two k-block tiles
@@ -63,6 +64,7 @@ struct DecSmem {
   static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
   static constexpr int TOTAL = OFF_MISC + 32 + NT * 4;   // TMEM address, then the tokens' scales as floats
   static constexpr int DYN_BYTES = TOTAL + 1024;
+  static_assert(DYN_BYTES <= 227 * 1024, "shared memory of one SM");
 };
 
 // Widens the 128 staged bytes of NT token rows into two int8 k-block tiles (NT x 128 B each,
