@@ -148,6 +148,9 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     // ------------------------------ MMA issuer (leader CTA) -------------------------------------
     if (rank == 0 && elect_one()) {
       constexpr uint32_t idesc = umma_idesc(/*c=s32*/ 2, /*a=s8*/ 1, /*b=s8*/ 1, P_TILE_M, P_TILE_N);
+      // The issuing thread pays several cycles per instruction: descriptors are formed once and
+      // differ from block to block by constants in the start-address field (no carry out of it).
+      const uint64_t b_desc0 = umma_desc_sw128(smem_u32(smem + L::OFF_B_OP));
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int tile = pair; tile < num_tiles && ok; tile += npairs, ++tcount) {
@@ -159,14 +162,21 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
           ok = mbar_wait(&full[s], (it / S_OP) & 1, PSITE_FULL, limit);
           if (!ok) break;
           tc_fence_after_sync();
+          // K = 32 int8 per MMA: 8 TMEM columns, 32 shared-memory bytes (2 in the descriptor's
+          // 16-byte units; the second k-block tile lies 128 * 128 bytes further on).
           const uint32_t a_tmem = tmem_base + P_A_COL0 + s * P_A_COLS_PER_STAGE;
-          const uint32_t b_base = smem_u32(smem + L::OFF_B_OP + s * L::B_OP);
-          const int nk = (2 * sb + 1 < num_kb) ? 8 : 4;  // K = 32 int8 each: 8 TMEM columns / 32 smem bytes
-#pragma unroll 4
-          for (int k = 0; k < nk; ++k)
-            umma_i8_ts_pair(tmem_base, a_tmem + k * 8,
-                            umma_desc_sw128(b_base + (k >> 2) * (128 * 128) + (k & 3) * 32), idesc,
-                            (sb | k) != 0 ? 1u : 0u);
+          const uint64_t bd = b_desc0 + static_cast<uint64_t>(s * (L::B_OP >> 4));
+          constexpr uint32_t KB1 = (128 * 128) >> 4;
+          umma_i8_ts_pair(tmem_base, a_tmem, bd, idesc, sb != 0 ? 1u : 0u);
+          umma_i8_ts_pair(tmem_base, a_tmem + 8, bd + 2, idesc, 1u);
+          umma_i8_ts_pair(tmem_base, a_tmem + 16, bd + 4, idesc, 1u);
+          umma_i8_ts_pair(tmem_base, a_tmem + 24, bd + 6, idesc, 1u);
+          if (2 * sb + 1 < num_kb) {
+            umma_i8_ts_pair(tmem_base, a_tmem + 32, bd + KB1, idesc, 1u);
+            umma_i8_ts_pair(tmem_base, a_tmem + 40, bd + (KB1 + 2), idesc, 1u);
+            umma_i8_ts_pair(tmem_base, a_tmem + 48, bd + (KB1 + 4), idesc, 1u);
+            umma_i8_ts_pair(tmem_base, a_tmem + 56, bd + (KB1 + 6), idesc, 1u);
+          }
           umma_commit_pair_mc(&empty[s], 3);            // frees ring stage s in both CTAs
         }
         umma_commit_pair_mc(tmem_full, 3);              // accumulator complete (or abandoned)
