@@ -130,14 +130,15 @@ __device__ __forceinline__ float absmax32(const uint32_t (&r)[32]) {
 // an SM (each with its own producer and MMA issuer); with 512 a CTA has the SM to itself.
 template <int N2, int S>
 __global__ void __launch_bounds__((2 + 4 * S) * 32, (S * 2 * N2 <= 256) ? 2 : 1)
-rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigned char* __restrict__ a1_img,
-                       const unsigned char* __restrict__ b2_img, int n1, long long rows,
-                       uint8_t* __restrict__ Xq, __half* __restrict__ scales, float* __restrict__ Zdbg) {
+rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ RqLayout L,
+                       const unsigned char* __restrict__ a1_img, const unsigned char* __restrict__ b2_img, int n1,
+                       int rows, uint8_t* __restrict__ Xq, __half* __restrict__ scales, float* __restrict__ Zdbg) {
   constexpr int TM_COLS = S * 2 * N2;             // 256 or 512
   griddep_launch_dependents();                   // a GEMM launched behind this kernel may set itself up
   constexpr int XQ = N2 / 64;
   constexpr int SLOT_COLS = 2 * N2;              // D1 (N2 columns) + D2 (N2 columns)
-  const RqLayout L = rq_layout(n1, N2, TM_COLS == 512 ? kMaxDynSmem : kHalfDynSmem);
+  // The layout comes from the host (the same rq_layout call that sized the shared memory); group
+  // counts are 32-bit: the set-up is on the critical path of a decode step.
   const int n = n1 * N2;
   const int G = L.G, LS = L.LS;
 
@@ -158,42 +159,45 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
   float* amax_x = reinterpret_cast<float*>(bars + 26);      // [S groups][2 parities][4 warps]
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-  const long long ngroups = (rows + G - 1) / G;
-  const long long my_groups = (ngroups > blockIdx.x) ? (ngroups - blockIdx.x + gridDim.x - 1) / gridDim.x : 0;
+  const int ngroups = (rows + G - 1) / G;
+  const int my_groups = (ngroups > static_cast<int>(blockIdx.x))
+                            ? (ngroups - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x)
+                            : 0;
   const uint32_t limit = wait_limit();
 
   // One X tile set per token group: G tokens, XQ 64-column blocks each.
-  auto load_group = [&](long long i) {
-    const long long g = blockIdx.x + i * gridDim.x;
-    const int s = static_cast<int>(i % L.XS);
+  auto load_group = [&](int i) {
+    const int g = static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x);
+    const int s = i % L.XS;
     mbar_arrive_expect_tx(&x_full[s], static_cast<uint32_t>(L.x_bytes));
     for (int tk = 0; tk < G; ++tk)
       for (int a = 0; a < XQ; ++a)
         tma_load_3d(xs + s * L.x_bytes + tk * L.x_token + a * L.x_tile, &tmap_x, &x_full[s], a * 64, 0,
-                    static_cast<int32_t>(g * G + tk));
+                    g * G + tk);
   };
-  const long long preload = my_groups < L.XS ? my_groups : L.XS;
+  const int preload = my_groups < L.XS ? my_groups : L.XS;
 
   if (threadIdx.x == 0) {
-    tma_prefetch_desc(&tmap_x);
+    // The first loads go out before anything else is set up: the whole X ring, then the factor
+    // images.  Only the barriers they complete on exist at that point; nobody else touches a
+    // barrier before the __syncthreads below.
+    for (int b = 0; b < 4; ++b) mbar_init(&x_full[b], 1);
+    mbar_init(img_full, 1);
+    mbar_fence_init();
+    for (int i = 0; i < preload; ++i) load_group(i);
+    mbar_arrive_expect_tx(img_full, static_cast<uint32_t>(L.a1_bytes + L.b2_bytes));
+    for (int o = 0; o < L.a1_bytes; o += 16384)
+      bulk_load_1d(a1s + o, a1_img + o, static_cast<uint32_t>(min(16384, L.a1_bytes - o)), img_full);
+    for (int o = 0; o < L.b2_bytes; o += 16384)
+      bulk_load_1d(b2s + o, b2_img + o, static_cast<uint32_t>(min(16384, L.b2_bytes - o)), img_full);
     for (int b = 0; b < 4; ++b) {
-      mbar_init(&x_full[b], 1);
       mbar_init(&x_empty[b], 1);
       mbar_init(&d1_full[b], 1);
       mbar_init(&a2_ready[b], 4);
       mbar_init(&d2_full[b], 1);
       mbar_init(&d_free[b], 4);
     }
-    mbar_init(img_full, 1);
     mbar_fence_init();
-    // The first loads go out before the rest of the CTA has finished setting up: the whole X ring,
-    // then the factor images.
-    for (long long i = 0; i < preload; ++i) load_group(i);
-    mbar_arrive_expect_tx(img_full, static_cast<uint32_t>(L.a1_bytes + L.b2_bytes));
-    for (int o = 0; o < L.a1_bytes; o += 16384)
-      bulk_load_1d(a1s + o, a1_img + o, static_cast<uint32_t>(min(16384, L.a1_bytes - o)), img_full);
-    for (int o = 0; o < L.b2_bytes; o += 16384)
-      bulk_load_1d(b2s + o, b2_img + o, static_cast<uint32_t>(min(16384, L.b2_bytes - o)), img_full);
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, TM_COLS);
@@ -207,7 +211,7 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
   if (warp == 0) {
     // ------------------------------ producer: keeps the X ring full -------------------------------------
     if (lane == 0) {
-      for (long long i = preload; i < my_groups; ++i) {
+      for (int i = preload; i < my_groups; ++i) {
         if (!mbar_wait(&x_empty[i % L.XS], ((i / L.XS) & 1) ^ 1, RQ_X_EMPTY, limit)) break;
         load_group(i);
       }
@@ -222,8 +226,8 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
       const uint64_t x_desc0 = umma_desc_sw128_mn(smem_u32(xs), static_cast<uint32_t>(L.x_tile));
       const int ksteps1 = L.N1 / 16;                 // K = p, 16 per MMA
       bool ok = mbar_wait(img_full, 0, RQ_IMG, limit);
-      auto stage1 = [&](long long i) {
-        const int slot = static_cast<int>(i % S), xs_i = static_cast<int>(i % L.XS);
+      auto stage1 = [&](int i) {
+        const int slot = i % S, xs_i = i % L.XS;
         tc_fence_after_sync();
         const uint32_t d1 = tmem_base + slot * SLOT_COLS;
         uint32_t acc = 0;
@@ -241,8 +245,8 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
         umma_commit(&x_empty[xs_i]);
         umma_commit(&d1_full[slot]);
       };
-      auto stage2 = [&](long long i) {
-        const int slot = static_cast<int>(i % S);
+      auto stage2 = [&](int i) {
+        const int slot = i % S;
         tc_fence_after_sync();
         const uint32_t d1 = tmem_base + slot * SLOT_COLS, d2 = d1 + N2;
 #pragma unroll
@@ -256,7 +260,7 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
       };
       // Whichever is ready goes: stage 1 of the next group whose X tile has landed and whose slot has
       // been drained, and stage 2 of the oldest group whose operand has been converted.
-      long long i1 = 0, i2 = 0;
+      int i1 = 0, i2 = 0;
       uint32_t idle = 0;
       while (ok && i2 < my_groups) {
         bool did = false;
@@ -289,9 +293,9 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigne
     const int wpt = LS / 32;                       // warps that share a token
     const int q0 = (quarter / wpt) * wpt;
     bool ok = true;
-    for (long long i = w; i < my_groups && ok; i += S) {
-      const long long g = blockIdx.x + i * gridDim.x;
-      const long long token = g * G + tk;
+    for (int i = w; i < my_groups && ok; i += S) {
+      const int g = static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x);
+      const long long token = static_cast<long long>(g) * G + tk;
       const uint32_t ph = (i / S) & 1;
 
       // ---- D1 -> fp16 hi/lo in place, with a per-lane power-of-two scale --------------------------
@@ -470,6 +474,7 @@ bool rotate_quant_tc_prepare(sq_rotation* h) {
 sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
                                    float* Zdbg, cudaStream_t s) {
   const int n1 = h->n1, n2 = h->n2;
+  if (rows > 0x7FFFFFFF) return SQ_ERR_UNSUPPORTED;   // the kernel counts token groups in 32 bits
   // n2 = 64 with images small enough: two CTAs per SM, two accumulator slots each.
   const RqLayout Lh = rq_layout(n1, n2, kHalfDynSmem);
   const bool dual = (n2 == 64) && Lh.XS >= 2;
@@ -498,7 +503,7 @@ sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t 
       smem_set = smem;
     }
     const unsigned grid = static_cast<unsigned>(std::min<long long>(ngroups, static_cast<long long>(sms) * ctas_per_sm));
-    kern<<<grid, (2 + 4 * slots) * 32, smem, s>>>(mx, a1, b2, n1, rows, static_cast<uint8_t*>(Xq),
+    kern<<<grid, (2 + 4 * slots) * 32, smem, s>>>(mx, L, a1, b2, n1, static_cast<int>(rows), static_cast<uint8_t*>(Xq),
                                                   static_cast<__half*>(scales), Zdbg);
     return true;
   };
