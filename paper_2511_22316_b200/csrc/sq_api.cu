@@ -1,6 +1,7 @@
 // C ABI entry points: argument validation on the host, then the kernel launchers.
 #include <cmath>
 #include <cstring>
+#include <mutex>
 #include <new>
 
 #include "sq_internal.h"
@@ -257,6 +258,41 @@ size_t sq_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K) {
          sq_linear_workspace_bytes(M, N, K);
 }
 
+namespace {
+// Copy streams and events of sq_linear_host, made once per device and kept until exit.
+constexpr int kHostChunks = 8;
+struct HostPipe {
+  bool ready = false;
+  cudaStream_t h2d = nullptr, d2h = nullptr;
+  cudaEvent_t start = nullptr, landed[kHostChunks] = {}, done[kHostChunks] = {};
+};
+HostPipe* host_pipe() {
+  static HostPipe pipes[64];
+  static std::mutex mu;
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= 64) return nullptr;
+  std::lock_guard<std::mutex> lock(mu);
+  HostPipe& p = pipes[dev];
+  if (!p.ready) {
+    bool ok = cudaStreamCreateWithFlags(&p.h2d, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaStreamCreateWithFlags(&p.d2h, cudaStreamNonBlocking) == cudaSuccess &&
+              cudaEventCreateWithFlags(&p.start, cudaEventDisableTiming) == cudaSuccess;
+    for (int c = 0; c < kHostChunks && ok; ++c)
+      ok = cudaEventCreateWithFlags(&p.landed[c], cudaEventDisableTiming) == cudaSuccess &&
+           cudaEventCreateWithFlags(&p.done[c], cudaEventDisableTiming) == cudaSuccess;
+    if (!ok) {
+      cudaGetLastError();
+      return nullptr;
+    }
+    p.ready = true;
+  }
+  return &p;
+}
+}  // namespace
+
+// Large batches are cut into up to eight row chunks: chunk c + 1 travels to the device while chunk c
+// is computed and chunk c - 1 travels back (the two copy directions use separate streams, the link
+// is full duplex), so the call takes about one direction's copy time instead of the sum of both.
 sq_status_t sq_linear_host(const sq_rotation_t* rot, const void* X_host, int64_t M, const void* Wq, const void* sw,
                            int64_t N, int64_t K, void* workspace, size_t workspace_bytes, void* Y_host,
                            void* stream) {
@@ -268,15 +304,49 @@ sq_status_t sq_linear_host(const sq_rotation_t* rot, const void* X_host, int64_t
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   const size_t xb = static_cast<size_t>(M) * K * 2, yb = static_cast<size_t>(M) * N * 2;
-  void* dX = ws;
-  void* dY = ws + align_up(xb, 256);
-  void* lws = static_cast<unsigned char*>(dY) + align_up(yb, 256);
-  if (cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return SQ_ERR_CUDA;
-  sq_status_t st = sq_linear(rot, dX, M, Wq, sw, N, K, lws, sq_linear_workspace_bytes(M, N, K), dY, stream);
+  unsigned char* dX = ws;
+  unsigned char* dY = ws + align_up(xb, 256);
+  void* lws = dY + align_up(yb, 256);
+  const size_t lws_bytes = sq_linear_workspace_bytes(M, N, K);
+  // Chunks of at least 256 rows (a full tile of the prefill GEMM), a multiple of 256 rows each.
+  int64_t chunk_rows = M;
+  if (M >= 512) chunk_rows = ((M + kHostChunks - 1) / kHostChunks + 255) / 256 * 256;
+  const int chunks = static_cast<int>((M + chunk_rows - 1) / chunk_rows);
+  HostPipe* p = chunks > 1 ? host_pipe() : nullptr;
+  if (chunks == 1 || p == nullptr) {
+    if (cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return SQ_ERR_CUDA;
+    sq_status_t st = sq_linear(rot, dX, M, Wq, sw, N, K, lws, lws_bytes, dY, stream);
+    if (st != SQ_OK) return st;
+    if (cudaMemcpyAsync(Y_host, dY, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SQ_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess) return SQ_ERR_CUDA;
+    return SQ_OK;
+  }
+  // Everything follows what is already queued on the caller's stream.
+  if (cudaEventRecord(p->start, s) != cudaSuccess || cudaStreamWaitEvent(p->h2d, p->start, 0) != cudaSuccess ||
+      cudaStreamWaitEvent(p->d2h, p->start, 0) != cudaSuccess)
+    return SQ_ERR_CUDA;
+  sq_status_t st = SQ_OK;
+  for (int c = 0; c < chunks && st == SQ_OK; ++c) {
+    const int64_t r0 = c * chunk_rows, r = (M - r0 < chunk_rows) ? M - r0 : chunk_rows;
+    const size_t xo = static_cast<size_t>(r0) * K * 2, yo = static_cast<size_t>(r0) * N * 2;
+    if (cudaMemcpyAsync(dX + xo, static_cast<const unsigned char*>(X_host) + xo, static_cast<size_t>(r) * K * 2,
+                        cudaMemcpyHostToDevice, p->h2d) != cudaSuccess ||
+        cudaEventRecord(p->landed[c], p->h2d) != cudaSuccess || cudaStreamWaitEvent(s, p->landed[c], 0) != cudaSuccess) {
+      st = SQ_ERR_CUDA;
+      break;
+    }
+    st = sq_linear(rot, dX + xo, r, Wq, sw, N, K, lws, lws_bytes, dY + yo, stream);
+    if (st != SQ_OK) break;
+    if (cudaEventRecord(p->done[c], s) != cudaSuccess || cudaStreamWaitEvent(p->d2h, p->done[c], 0) != cudaSuccess ||
+        cudaMemcpyAsync(static_cast<unsigned char*>(Y_host) + yo, dY + yo, static_cast<size_t>(r) * N * 2,
+                        cudaMemcpyDeviceToHost, p->d2h) != cudaSuccess)
+      st = SQ_ERR_CUDA;
+  }
+  // Wait for all three streams whatever happened, so that no copy outlives the call.
+  const bool synced = cudaStreamSynchronize(p->h2d) == cudaSuccess && cudaStreamSynchronize(s) == cudaSuccess &&
+                      cudaStreamSynchronize(p->d2h) == cudaSuccess;
   if (st != SQ_OK) return st;
-  if (cudaMemcpyAsync(Y_host, dY, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SQ_ERR_CUDA;
-  if (cudaStreamSynchronize(s) != cudaSuccess) return SQ_ERR_CUDA;
-  return SQ_OK;
+  return synced ? SQ_OK : SQ_ERR_CUDA;
 }
 
 sq_status_t sq_last_device_status(void* stream) {

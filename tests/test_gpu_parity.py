@@ -430,6 +430,24 @@ def test_linear_prefill_config_sampled(sq):
     assert np.linalg.norm(Yg - Yo) <= 1e-2 * np.linalg.norm(Yo)
 
 
+def test_linear_host_chunked_equals_device_path(sq):
+    """sq_linear_host cuts batches of 512 rows or more into row chunks whose copies and computation
+    overlap.  Every row is treated on its own, so the outputs must equal those of one sq_linear call
+    on the whole batch bit for bit -- here with a ragged last chunk (1100 = 4 x 256 + 76 rows) that
+    takes a different GEMM kernel than the full chunks -- and twice in a row (the copy streams and
+    events are reused)."""
+    w = wl.small("host_chunks", 1100, 64, 64, 264, 77)
+    X, W = wl.make_layer(w)
+    R1, R2 = ora.build_rotation(X.astype(np.float32), w.n1, w.n2)
+    Yd = run_linear(sq, w, X, W, R1, R2, host=False)
+    for _ in range(2):
+        Yh = run_linear(sq, w, X, W, R1, R2, host=True)
+        assert np.array_equal(Yh.view(np.uint16), Yd.view(np.uint16))
+    rows = np.array([0, 255, 256, 1023, 1024, 1099])
+    Yo = ora.linear(X[rows], W, R1, R2).astype(np.float64)
+    assert np.linalg.norm(Yd[rows].astype(np.float64) - Yo) <= 1e-2 * np.linalg.norm(Yo)
+
+
 def test_empty_inputs_are_no_ops(sq):
     w = wl.TINY
     X = wl.make_activations(w)
