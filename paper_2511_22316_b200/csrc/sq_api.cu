@@ -2,6 +2,7 @@
 #include <cmath>
 #include <cstring>
 #include <mutex>
+#include <vector>
 #include <new>
 
 #include "sq_internal.h"
@@ -10,6 +11,26 @@
 namespace sq {
 std::atomic<uint64_t> g_launches{0};
 thread_local bool g_pdl_next = false;
+
+bool ensure_dyn_smem(const void* kern, int bytes) {
+  struct Entry { int dev; const void* kern; int bytes; };
+  static std::mutex mu;
+  static std::vector<Entry> set;
+  if (bytes <= 48 * 1024) return true;                 // within every kernel's default limit
+  int dev = 0;
+  if (cudaGetDevice(&dev) != cudaSuccess) return false;
+  std::lock_guard<std::mutex> lock(mu);
+  for (Entry& e : set)
+    if (e.dev == dev && e.kern == kern) {
+      if (e.bytes >= bytes) return true;
+      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+      e.bytes = bytes;
+      return true;
+    }
+  if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes) != cudaSuccess) return false;
+  set.push_back({dev, kern, bytes});
+  return true;
+}
 
 int sm_count() {
   static std::atomic<int> cache[64];

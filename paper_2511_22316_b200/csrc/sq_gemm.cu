@@ -356,12 +356,7 @@ sq_status_t launch_tc(const void* Xq, const void* sx, const void* Wq, const void
   CUtensorMap mx, mw;
   if (!make_packed_map(&mx, Xq, M, K / 2, BM) || !make_packed_map(&mw, Wq, N, K / 2, BN)) return SQ_ERR_CUDA;
   auto kern = w4a4_gemm_tc_kernel<BN, S_OP, S_ST>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
-      return SQ_ERR_CUDA;
-    attr_set = true;
-  }
+  if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), L::DYN_BYTES)) return SQ_ERR_CUDA;
   const int sms = sm_count();
   if (sms <= 0) return SQ_ERR_CUDA;
   const int tiles = ((N + BN - 1) / BN) * ((M + BM - 1) / BM);

@@ -542,12 +542,7 @@ sq_status_t launch_decode(const void* Xq, const void* sx, const void* Wq, const 
   const int sms = sm_count();
   if (sms <= 0) return SQ_ERR_CUDA;
   auto kern = w4a4_gemm_decode_kernel<NT>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
-      return SQ_ERR_CUDA;
-    attr_set = true;
-  }
+  if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), L::DYN_BYTES)) return SQ_ERR_CUDA;
   const int tiles = (N + 127) / 128, blocks = (K / 128 + 1) / 2;
   const int splits = choose_splits<NT>(tiles, blocks, sms);
   const int ncl_max = max_clusters<NT>(splits, sms);

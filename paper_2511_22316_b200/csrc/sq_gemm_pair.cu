@@ -338,12 +338,7 @@ sq_status_t launch_w4a4_gemm_pair(const void* Xq, const void* sx, const void* Wq
       !make_out_map(&my, Y, M, N))
     return SQ_ERR_CUDA;
   auto kern = w4a4_gemm_pair_kernel<S_OP, S_ST>;
-  static bool attr_set = false;
-  if (!attr_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, L::DYN_BYTES) != cudaSuccess)
-      return SQ_ERR_CUDA;
-    attr_set = true;
-  }
+  if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), L::DYN_BYTES)) return SQ_ERR_CUDA;
   const int sms = sm_count();
   if (sms <= 0) return SQ_ERR_CUDA;
   const int tiles = ((N + P_TILE_N - 1) / P_TILE_N) * ((M + P_TILE_M - 1) / P_TILE_M);

@@ -163,11 +163,7 @@ sq_status_t launch_gemv(const void* Xq, const void* sx, const void* Wq, const vo
   const int warps = gemv_warps(ntask, sms);
   const int smem = MT * K;                               // 2 * MT * (K / 8) words
   auto kern = w4a4_gemv_kernel<MT>;
-  static int smem_set = 48 * 1024;
-  if (smem > smem_set) {
-    if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SQ_ERR_CUDA;
-    smem_set = smem;
-  }
+  if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return SQ_ERR_CUDA;
   const unsigned grid = static_cast<unsigned>(std::min<long long>(sms, (ntask + warps - 1) / warps));
   const cudaError_t err = launch_maybe_pdl(kern, dim3(grid), dim3(warps * 32), static_cast<size_t>(smem), s,
                                            static_cast<const uint8_t*>(Xq), static_cast<const __half*>(sx),

@@ -69,6 +69,10 @@ inline cudaError_t launch_maybe_pdl(void (*kern)(KArgs...), dim3 grid, dim3 bloc
   return launch_cluster_maybe_pdl(kern, grid, block, smem, s, 1u, static_cast<Args&&>(args)...);
 }
 
+// Raises a kernel's dynamic shared-memory limit to `bytes` if it is lower.  Function attributes
+// belong to a device: the sizes already set are remembered per (device, kernel).
+bool ensure_dyn_smem(const void* kern, int bytes);
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Host-side construction of the factors in float64 (sq_rotation_host.cu).

@@ -423,20 +423,12 @@ sq_status_t launch_rotate_quant_pair(const sq_rotation* h, const void* X, int64_
   const unsigned char* b2 = static_cast<const unsigned char*>(h->dB2img);
   if (n2 == 64) {
     auto kern = rotate_quant_pair_kernel<64>;
-    static int smem_set = 0;
-    if (smem > smem_set) {
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SQ_ERR_CUDA;
-      smem_set = smem;
-    }
+    if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return SQ_ERR_CUDA;
     kern<<<grid, (2 + 4 * 4) * 32, smem, s>>>(mx, a1, b2, n1, rows, static_cast<uint8_t*>(Xq),
                                               static_cast<__half*>(scales), Zdbg);
   } else {
     auto kern = rotate_quant_pair_kernel<128>;
-    static int smem_set = 0;
-    if (smem > smem_set) {
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return SQ_ERR_CUDA;
-      smem_set = smem;
-    }
+    if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return SQ_ERR_CUDA;
     kern<<<grid, (2 + 4 * 2) * 32, smem, s>>>(mx, a1, b2, n1, rows, static_cast<uint8_t*>(Xq),
                                               static_cast<__half*>(scales), Zdbg);
   }

@@ -495,23 +495,19 @@ sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t 
   const long long ngroups = (rows + L.G - 1) / L.G;
   const unsigned char* a1 = static_cast<const unsigned char*>(h->dA1img);
   const unsigned char* b2 = static_cast<const unsigned char*>(h->dB2img);
-  auto launch = [&](auto kern, int slots, int ctas_per_sm, int& smem_set) -> bool {
+  auto launch = [&](auto kern, int slots, int ctas_per_sm) -> bool {
     // A CTA that wants all of TMEM asks for more than half of the shared memory, so that it is alone.
     const int smem = ctas_per_sm == 1 ? std::max(L.total + 1024, 120 * 1024) : L.total + 1024;
-    if (smem > smem_set) {
-      if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, smem) != cudaSuccess) return false;
-      smem_set = smem;
-    }
+    if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return false;
     const unsigned grid = static_cast<unsigned>(std::min<long long>(ngroups, static_cast<long long>(sms) * ctas_per_sm));
     kern<<<grid, (2 + 4 * slots) * 32, smem, s>>>(mx, L, a1, b2, n1, static_cast<int>(rows), static_cast<uint8_t*>(Xq),
                                                   static_cast<__half*>(scales), Zdbg);
     return true;
   };
-  static int set_64_2 = 0, set_64_4 = 0, set_128_2 = 0;     // largest shared-memory size set per kernel
   bool ok;
-  if (n2 == 64 && dual) ok = launch(rotate_quant_tc_kernel<64, 2>, 2, 2, set_64_2);
-  else if (n2 == 64) ok = launch(rotate_quant_tc_kernel<64, 4>, 4, 1, set_64_4);
-  else ok = launch(rotate_quant_tc_kernel<128, 2>, 2, 1, set_128_2);
+  if (n2 == 64 && dual) ok = launch(rotate_quant_tc_kernel<64, 2>, 2, 2);
+  else if (n2 == 64) ok = launch(rotate_quant_tc_kernel<64, 4>, 4, 1);
+  else ok = launch(rotate_quant_tc_kernel<128, 2>, 2, 1);
   if (!ok) return SQ_ERR_CUDA;
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;

@@ -362,9 +362,12 @@ def test_gemm_decode_needs_no_workspace(sq):
     assert np.array_equal(y.numpy(np.float16, (M, N)).view(np.uint16), Y1.view(np.uint16))
 
 
-def test_gemm_is_deterministic(sq):
+@pytest.mark.parametrize("M,N,K", [(200, 384, 1024), (40, 136, 8192), (16, 5120, 14336), (2, 264, 4096)])
+def test_gemm_is_deterministic(sq, M, N, K):
+    """Two calls give the same bits: the pair kernel, the decode kernel with K split over clusters
+    (one tile per cluster, and several tiles per cluster with the reduce buffer reused), the
+    dot-product kernel."""
     rng = np.random.default_rng(5)
-    M, N, K = 200, 384, 1024
     Xc, Wc = random_codes(rng, M, K), random_codes(rng, N, K)
     sx = rng.uniform(0.01, 2.0, size=M).astype(np.float16)
     sw = rng.uniform(0.001, 0.1, size=N).astype(np.float16)
