@@ -131,9 +131,12 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     if (elect_one()) {
       uint32_t it = 0;
       bool ok = true;
+      // Tile order: token tiles innermost.  The pairs that run at the same time then share a few weight
+      // tiles and all of X, which stays in L2; with the channel tiles innermost every token tile
+      // streamed the whole weight matrix from HBM again once it no longer fitted L2.
       for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
-        const int m0 = (tile / tiles_n) * P_TILE_M + static_cast<int>(rank) * 128;
-        const int n0 = (tile % tiles_n) * P_TILE_N + static_cast<int>(rank) * 128;
+        const int m0 = (tile % tiles_m) * P_TILE_M + static_cast<int>(rank) * 128;
+        const int n0 = (tile / tiles_m) * P_TILE_N + static_cast<int>(rank) * 128;
         for (int sb = 0; sb < num_sb; ++sb, ++it) {
           const int ss = it % S_ST;
           ok = mbar_wait(&st_empty[ss], ((it / S_ST) & 1) ^ 1, PSITE_ST_EMPTY, limit);
@@ -258,8 +261,8 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     uint32_t tcount = 0, nstore = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += npairs, ++tcount) {
-      const int m0 = (tile / tiles_n) * P_TILE_M + static_cast<int>(rank) * 128;
-      const int n0 = (tile % tiles_n) * P_TILE_N;
+      const int m0 = (tile % tiles_m) * P_TILE_M + static_cast<int>(rank) * 128;
+      const int n0 = (tile / tiles_m) * P_TILE_N;
       // Fetched while the MMAs still run: this row's token step, and the channel steps of the warp's
       // 128 columns, four per lane (handed round by shuffles when a chunk needs them).
       const int row0 = m0 + q * 32, row = row0 + lane;
