@@ -98,6 +98,7 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   const int tiles_n = (N + P_TILE_N - 1) / P_TILE_N, tiles_m = (M + P_TILE_M - 1) / P_TILE_M;
   const int num_tiles = tiles_n * tiles_m;
   const uint32_t limit = wait_limit();
+  const int pre_sb = num_sb < S_ST ? num_sb : S_ST;    // blocks whose weights are requested during set-up
 
   if (threadIdx.x == 0) {
     tma_prefetch_desc(&tmap_x);
@@ -114,6 +115,15 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     mbar_init(tmem_full, 1);
     mbar_init(tmem_empty, 2 * P_EPI_WARPS);
     mbar_fence_init();
+    // The weights of the first tile's first blocks do not depend on the kernel launched before this
+    // one: they are requested now (local barriers only), the activations after the wait below.
+    if (pair < num_tiles) {
+      const int n0 = (pair / tiles_m) * P_TILE_N + static_cast<int>(rank) * 128;
+      for (int sb = 0; sb < pre_sb; ++sb) {
+        mbar_arrive_expect_tx(&st_full[sb], L::A_ST + L::B_ST);
+        tma_load_2d(smem + L::OFF_B_ST + sb * L::B_ST, &tmap_w, &st_full[sb], sb * 128, n0);
+      }
+    }
   }
   if (warp == 1) {
     tmem_alloc_pair(tmem_slot, 512);
@@ -139,6 +149,10 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         const int n0 = (tile / tiles_m) * P_TILE_N + static_cast<int>(rank) * 128;
         for (int sb = 0; sb < num_sb; ++sb, ++it) {
           const int ss = it % S_ST;
+          if (it < static_cast<uint32_t>(pre_sb)) {     // armed and half loaded during set-up
+            tma_load_2d(smem + L::OFF_A_ST + ss * L::A_ST, &tmap_x, &st_full[ss], sb * 128, m0);
+            continue;
+          }
           ok = mbar_wait(&st_empty[ss], ((it / S_ST) & 1) ^ 1, PSITE_ST_EMPTY, limit);
           if (!ok) break;
           mbar_arrive_expect_tx(&st_full[ss], L::A_ST + L::B_ST);
