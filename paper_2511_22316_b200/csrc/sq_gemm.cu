@@ -391,6 +391,31 @@ sq_status_t launch_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, con
   const bool tc_ok = (K % BK == 0) && (N % 8 == 0) && K >= BK;
   if (gemm_pair_supported(M, N, K))
     return launch_w4a4_gemm_pair(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
+  if (M > 64 && M <= 128 && gemm_decode_supported(64, N, K)) {
+    // 65 to 128 tokens: the CTA-pair kernel with its tile half empty, or the decode kernel twice
+    // (64 tokens, then the rest; the weights are read twice).  Estimates in microseconds from
+    // measured rates: a 256-channel block costs a pair 0.54 and a decode CTA 0.46; fixed costs 6
+    // and 8 per launch.  The pair kernel wins when its 256-channel tiles fill the 74 pairs or K is
+    // short; the decode kernel wins on long K with few output channels (it splits K).
+    const int sms = sm_count();
+    if (sms <= 0) return SQ_ERR_CUDA;
+    const int num_sb = static_cast<int>((K / 128 + 1) / 2);
+    const int pair_tiles = static_cast<int>((N + 255) / 256), pairs = sms / 2 > 0 ? sms / 2 : 1;
+    const double pair_us = 6.0 + 0.54 * num_sb * ((pair_tiles + pairs - 1) / pairs);
+    const int dec_tiles = static_cast<int>((N + 127) / 128);
+    int split = 1;
+    while (split < 8 && dec_tiles * split * 2 <= sms && num_sb / (split * 2) >= 2) split *= 2;
+    const int clusters = sms / split > 0 ? sms / split : 1;
+    const double dec_us = 2.0 * (8.0 + 0.46 * ((num_sb + split - 1) / split) * ((dec_tiles + clusters - 1) / clusters));
+    if (pair_us <= dec_us) return launch_w4a4_gemm_pair(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
+    const sq_status_t st = launch_w4a4_gemm_decode(Xq, sx, Wq, sw, 64, (int)N, (int)K, Y, accdbg, nullptr, 0, s);
+    if (st != SQ_OK) return st;
+    const size_t half = 64;
+    return launch_w4a4_gemm_decode(static_cast<const unsigned char*>(Xq) + half * (K / 2),
+                                   static_cast<const __half*>(sx) + half, Wq, sw, (int)(M - 64), (int)N, (int)K,
+                                   static_cast<__half*>(Y) + half * N, accdbg ? accdbg + half * N : nullptr, nullptr, 0,
+                                   s);
+  }
   if (tc_ok) {
     if (N >= 256 && M > 64)
       return launch_tc<256, 2, 2>(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);

@@ -269,6 +269,9 @@ GEMM_SHAPES = [
     # tiles per pair and more k-blocks than the operand ring holds
     (129, 128, 128), (256, 256, 128), (200, 136, 384), (384, 520, 1664), (1000, 1288, 896),
     (513, 2304, 2176),
+    # 65..128 tokens: the pair kernel with a half-empty tile (many channel tiles or short K) or the
+    # decode kernel twice (few channels, long K), with one and with 63 rows in the second launch
+    (100, 9608, 512), (96, 520, 8192), (65, 256, 6144), (127, 264, 4096),
     # decode kernel (M <= 64, weights as the A operand, K split over a cluster): all three
     # token-count classes, ragged channel tile, odd k-block count, the two decode layer shapes;
     # clusters of 2, 4 and 8, and more tiles than the device holds clusters (slots reused)
