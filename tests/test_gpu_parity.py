@@ -299,6 +299,29 @@ def test_gemm_accumulators_bit_exact(sq, M, N, K):
     assert _fp16_ulps_apart(Y, Yo.astype(np.float16)).max() <= 1
 
 
+def test_gemm_random_shapes_bit_exact(sq):
+    """Seeded random shapes across every kernel's range (token counts from each dispatch class, ragged
+    channel counts, K a multiple of 128 or merely even): accumulators equal the oracle's bit for bit."""
+    rng = np.random.default_rng(20251122)
+    done = 0
+    while done < 60:
+        cls = done % 6
+        M = int([rng.integers(1, 5), rng.integers(3, 17), rng.integers(17, 65), rng.integers(65, 129),
+                 rng.integers(129, 300), rng.integers(1, 300)][cls])
+        N = int(rng.integers(1, 200)) * 8 if rng.random() < 0.85 else int(rng.integers(1, 1500))
+        K = int(rng.integers(1, 60)) * 128 if rng.random() < 0.85 else int(rng.integers(1, 2000)) * 2
+        if M * N * K > 1.0e8:
+            continue
+        Xc, Wc = random_codes(rng, M, K), random_codes(rng, N, K)
+        sx = rng.uniform(0.01, 2.0, size=M).astype(np.float16)
+        sw = rng.uniform(0.001, 0.1, size=N).astype(np.float16)
+        Y, acc = run_gemm(sq, Xc, Wc, sx, sw)
+        acc_o = ora.gemm_i32(Xc, Wc)
+        assert np.array_equal(acc, acc_o), (M, N, K)
+        assert _fp16_ulps_apart(Y, ora.dequant(acc_o, sx, sw)).max() <= 1, (M, N, K)
+        done += 1
+
+
 def test_gemm_extreme_codes_do_not_overflow(sq):
     M, N, K = 4, 8, 28672
     Xc = np.full((M, K), -8, np.int8)
