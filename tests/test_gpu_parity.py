@@ -434,7 +434,9 @@ def run_linear(sq, w, X, W, R1, R2, host=False):
 
 
 @pytest.mark.parametrize("w", [wl.TINY, wl.small("lin1", 70, 64, 64, 264, 51), wl.small("lin2", 9, 12, 8, 24, 52),
-                               wl.small("lin3", 5, 172, 64, 136, 53), wl.decode_up(4)])
+                               wl.small("lin3", 5, 172, 64, 136, 53), wl.decode_up(4),
+                               wl.small("lin_decode_split", 16, 112, 128, 512, 54),
+                               wl.small("lin_mid_batch", 100, 64, 64, 520, 55)])
 @pytest.mark.parametrize("host", [False, True])
 def test_linear_matches_oracle(sq, w, host):
     X, W = wl.make_layer(w)
