@@ -10,12 +10,13 @@
 // Pipeline per CTA (block = 256 channels = 128 packed bytes per row = two k-blocks of 128):
 //   warp 0        TMA: packed A rows and packed B rows, one block per staging stage
 //   warps 2..5    A: staging -> registers -> widen -> TMEM ring stage        } arrive on the
-//   warps 6..13   B: staging -> registers -> widen -> swizzled operand ring  } leader's full[s]
+//   warps 6..9    B: staging -> registers -> widen -> swizzled operand ring  } leader's full[s]
 //   warp 1        (leader CTA only) 8 MMAs of K = 32 per block; commit frees the ring stage in
 //                 both CTAs; the last commit of a tile publishes the accumulator to both CTAs
-//   warps 14..21  epilogue: TMEM -> dequantise -> fp16 tile in shared memory -> TMA store (which
-//                 also clips the ragged edges); two warps per TMEM lane quarter, four 32-column
-//                 chunks each; the accumulator is handed back as soon as it has been read
+//   warps 10..25  epilogue: TMEM -> dequantise -> fp16 tile in shared memory -> TMA store (which
+//                 also clips the ragged edges); four warps per TMEM lane quarter, two 32-column
+//                 chunks each, so that the single accumulator is handed back after one chunk's
+//                 worth of work and the next tile's MMAs wait as briefly as possible
 // Every hand-over costs each warp a few hundred cycles of barrier and fence latency whatever the
 // amount of data, which is why a ring stage holds two k-blocks.
 // The widening and the operand byte order are those of the single-CTA kernel (sq_gemm.cu).
@@ -29,8 +30,8 @@ namespace sq {
 namespace {
 
 constexpr int P_A_WARPS = 4;
-constexpr int P_B_WARPS = 8;
-constexpr int P_EPI_WARPS = 8;
+constexpr int P_B_WARPS = 4;             // one weight row of the CTA's 128 per thread
+constexpr int P_EPI_WARPS = 16;          // four per TMEM lane quarter, two 32-column chunks each
 constexpr int P_THREADS = (2 + P_A_WARPS + P_B_WARPS + P_EPI_WARPS) * 32;
 constexpr int P_TILE_M = 256;            // tokens per pair tile (128 per CTA)
 constexpr int P_TILE_N = 256;            // output channels per pair tile (128 staged per CTA)
@@ -53,7 +54,7 @@ struct PairSmem {
   static constexpr int OFF_B_ST = OFF_A_ST + S_ST * A_ST;
   static constexpr int OUT_BUF = 32 * 64;            // fp16 [32 rows x 32 columns], 64-byte swizzle
   static constexpr int OFF_OUT = OFF_B_ST + S_ST * B_ST;
-  static constexpr int OFF_BAR = OFF_OUT + P_EPI_WARPS * 2 * OUT_BUF;
+  static constexpr int OFF_BAR = OFF_OUT + P_EPI_WARPS * OUT_BUF;     // one staging tile per epilogue warp
   static constexpr int NUM_BARS = 2 * S_OP + 2 * S_ST + 2;
   static constexpr int OFF_TMEM = OFF_BAR + NUM_BARS * 8;
   static constexpr int TOTAL = OFF_TMEM + 16;
@@ -245,19 +246,40 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     }
   } else if (warp < 2 + P_A_WARPS + P_B_WARPS) {
     // ------------------------------ B unpackers: staging -> registers -> operand ring -----------
-    const int t = threadIdx.x - (2 + P_A_WARPS) * 32;   // 0 .. 255
+    // Thread t widens row t of the CTA's 128 weight rows: eight 16-byte loads (both k-blocks) first,
+    // then the sixteen stores.  Consecutive lanes take consecutive rows, whose swizzled chunks fall
+    // into different bank groups.
+    const int br = threadIdx.x - (2 + P_A_WARPS) * 32;  // 0 .. 127
+    const int bsw = br & 7;
     uint32_t it = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
       for (int sb = 0; sb < num_sb && ok; ++sb, ++it) {
         const int ss = it % S_ST, s = it % S_OP;
-        ok = mbar_wait(&st_full[ss], (it / S_ST) & 1, PSITE_ST_FULL_B, limit) &&
-             mbar_wait(&empty[s], ((it / S_OP) & 1) ^ 1, PSITE_EMPTY_B, limit);
+        ok = mbar_wait(&st_full[ss], (it / S_ST) & 1, PSITE_ST_FULL_B, limit);
         if (!ok) break;
-        const unsigned char* st = smem + L::OFF_B_ST + ss * L::B_ST;
-        unsigned char* op = smem + L::OFF_B_OP + s * L::B_OP;
-        unpack_tile<128>(st, op, t, 0);
-        if (2 * sb + 1 < num_kb) unpack_tile<128>(st, op + 128 * 128, t, 1);
+        const int nh = (2 * sb + 1 < num_kb) ? 2 : 1;
+        const unsigned char* row = smem + L::OFF_B_ST + ss * L::B_ST + br * 128;
+        uint4 w[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+          if (c < 4 * nh) w[c] = *reinterpret_cast<const uint4*>(row + ((c ^ bsw) << 4));
+        ok = mbar_wait(&empty[s], ((it / S_OP) & 1) ^ 1, PSITE_EMPTY_B, limit);
+        if (!ok) break;
+#pragma unroll
+        for (int c = 0; c < 8; ++c) {
+          if (c < 4 * nh) {
+            const int h = c >> 2, j = c & 3;
+            uint4 lo, hi;
+            lo.x = (w[c].x << 4) & 0xF0F0F0F0u; hi.x = w[c].x & 0xF0F0F0F0u;
+            lo.y = (w[c].y << 4) & 0xF0F0F0F0u; hi.y = w[c].y & 0xF0F0F0F0u;
+            lo.z = (w[c].z << 4) & 0xF0F0F0F0u; hi.z = w[c].z & 0xF0F0F0F0u;
+            lo.w = (w[c].w << 4) & 0xF0F0F0F0u; hi.w = w[c].w & 0xF0F0F0F0u;
+            unsigned char* orow = smem + L::OFF_B_OP + s * L::B_OP + h * (128 * 128) + br * 128;
+            *reinterpret_cast<uint4*>(orow + ((j ^ bsw) << 4)) = lo;
+            *reinterpret_cast<uint4*>(orow + (((4 + j) ^ bsw) << 4)) = hi;
+          }
+        }
         fence_proxy_async_smem();                       // generic-proxy stores -> visible to the MMA
         __syncwarp();
         if (lane == 0) {
@@ -268,10 +290,10 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     }
   } else {
     // ------------------------------ epilogue ----------------------------------------------------
-    const int e = warp - (2 + P_A_WARPS + P_B_WARPS);   // 0 .. 7
+    const int e = warp - (2 + P_A_WARPS + P_B_WARPS);   // 0 .. 15
     const int q = warp & 3;                             // TMEM lane quarter this warp may read
-    const int c_first = (e >> 2) * 4;                   // this warp's four 32-column chunks
-    unsigned char* obuf = smem + L::OFF_OUT + e * 2 * L::OUT_BUF;
+    const int c_first = (e >> 2) * 2;                   // this warp's two 32-column chunks
+    unsigned char* obuf = smem + L::OFF_OUT + e * L::OUT_BUF;
     uint32_t tcount = 0, nstore = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += npairs, ++tcount) {
@@ -288,20 +310,20 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
       tc_fence_after_sync();
       const uint32_t tmem_d = tmem_base + (static_cast<uint32_t>(q * 32) << 16);
 #pragma unroll 1
-      for (int j = 0; j < 4; ++j, ++nstore) {
+      for (int j = 0; j < 2; ++j, ++nstore) {
         const int c = c_first + j;
         uint32_t r[32];
         tmem_ld_32x32b_x32(tmem_d + c * 32, r);
         tmem_wait_ld();
-        if (j == 3) {                                   // last read of this warp: hand the accumulator back
+        if (j == 1) {                                   // last read of this warp: hand the accumulator back
           tc_fence_before_sync();
           __syncwarp();
           if (lane == 0) mbar_arrive_cluster(tmem_empty, 0);
         }
         const int col0 = n0 + c * 32;
-        unsigned char* buf = obuf + (nstore & 1) * L::OUT_BUF;
-        if (nstore >= 2) {                              // the store issued two chunks ago has read `buf`
-          if (lane == 0) tma_store_wait_read_1();
+        unsigned char* buf = obuf;
+        if (nstore >= 1) {                              // the previous chunk's store has read `buf`
+          if (lane == 0) tma_store_wait_read_0();
           __syncwarp();
         }
 #pragma unroll
