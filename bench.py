@@ -122,9 +122,11 @@ class ClockSampler:
 
     def _read(self):
         for line in self.proc.stdout:
-            self.lines.append(line.strip())
+            self.lines.append((time.perf_counter(), line.strip()))
 
-    def stop(self):
+    def stop(self, t_begin=None, t_end=None):
+        """Median SM clock and throttle reasons over the samples that arrived inside [t_begin, t_end]
+        (the timed region); if fewer than three did, over every sample of the run, and says so."""
         if self.proc is None:
             return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         self.proc.terminate()
@@ -134,7 +136,9 @@ class ClockSampler:
             self.proc.kill()
         sm, smax, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
+        inside = [ln for (t, ln) in self.lines if t_begin is not None and t_begin <= t <= t_end]
+        scope = "timed region" if len(inside) >= 3 else "whole run (timed region shorter than three samples)"
+        for ln in (inside if len(inside) >= 3 else [ln for (_, ln) in self.lines]):
             f = [x.strip() for x in ln.split(",")]
             if len(f) < 9:
                 continue
@@ -148,7 +152,7 @@ class ClockSampler:
                     reasons.add(name)
         return {"sm_mhz": statistics.median(sm) if sm else None,
                 "sm_max_mhz": max(smax) if smax else None,
-                "samples": len(sm), "reasons": sorted(reasons)}
+                "samples": len(sm), "scope": scope, "reasons": sorted(reasons)}
 
 
 # ----------------------------------------------------------------------------------------------
@@ -308,11 +312,13 @@ def run_ours(args, w):
     launches0 = sq.sq_kernel_launch_count()
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     sync_all()
+    t_region0 = time.perf_counter()
     e0.record()
     for i in range(args.steps):
         step(i)
     e1.record()
     sync_all()
+    t_region1 = time.perf_counter()
     ms_total = e0.elapsed_time(e1)
     launches = sq.sq_kernel_launch_count() - launches0
 
@@ -392,7 +398,7 @@ def run_ours(args, w):
     e2e_ms = h0.elapsed_time(h1) / e2e_steps
     status = sq.sq_last_device_status()
 
-    clocks = sampler.stop() if rank == 0 else None
+    clocks = sampler.stop(t_region0, t_region1) if rank == 0 else None
 
     # ---- max over ranks ---------------------------------------------------------------------
     t = torch.tensor([ms_total, e2e_ms, rq_ms, gemm_ms, graph_ms if graph_ms is not None else -1.0],
@@ -472,13 +478,17 @@ def run_ours(args, w):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=1000)
+    ap.add_argument("--steps", type=int, default=None,
+                    help="timed steps (default: 20000, about a second of config 2, so that several clock samples "
+                         "fall inside the timed region; 20 passes for --impl reference)")
     ap.add_argument("--warmup", type=int, default=5)
     ap.add_argument("--workload", default=DEFAULT_WORKLOAD)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true",
                     help="skip the timed CPU oracle leg (for profiler runs)")
     args = ap.parse_args()
+    if args.steps is None:
+        args.steps = 20 if args.impl == "reference" else 20000
     w = wl.by_name(args.workload)
     if args.impl == "reference":
         return run_reference(args, w)
