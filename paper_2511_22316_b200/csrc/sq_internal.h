@@ -109,7 +109,9 @@ bool gemm_pair_supported(int64_t M, int64_t N, int64_t K);
 sq_status_t launch_w4a4_gemm_pair(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N,
                                   int K, void* Y, int32_t* accdbg, cudaStream_t s);
 
-// Step 3 for decode-sized problems (sq_gemm_decode.cu): weights as the A operand, split K.
+// Step 3 for decode-sized problems (sq_gemm_decode.cu): weights as the A operand, K split over a
+// thread-block cluster with the partial tiles exchanged on chip (the workspace arguments are unused
+// and the size is 0; they remain for a kernel that wants scratch).
 bool gemm_decode_supported(int64_t M, int64_t N, int64_t K);
 size_t gemm_decode_workspace_bytes(int64_t M, int64_t N, int64_t K);
 sq_status_t launch_w4a4_gemm_decode(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N, int K,
