@@ -209,7 +209,7 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
         if (i1 < my_tokens && i1 < i2 + S &&
             mbar_test_wait(&x_full[i1 % L.XS], (i1 / L.XS) & 1) &&
             mbar_test_wait(&xp_full[i1 % L.XS], (i1 / L.XS) & 1) &&
-            mbar_test_wait(&d_free[i1 % S], ((i1 / S) & 1) ^ 1)) {
+            mbar_test_wait(&d2_full[i1 % S], ((i1 / S) & 1) ^ 1)) {   // D1 free: the slot's previous stage 2 is done
           stage1(i1++);
           did = true;
         }

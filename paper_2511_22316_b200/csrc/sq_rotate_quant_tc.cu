@@ -258,15 +258,19 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         }
         umma_commit(&d2_full[slot]);
       };
-      // Whichever is ready goes: stage 1 of the next group whose X tile has landed and whose slot has
-      // been drained, and stage 2 of the oldest group whose operand has been converted.
+      // Whichever is ready goes: stage 1 of the next group whose X tile has landed and whose slot's D1
+      // columns are free, and stage 2 of the oldest group whose operand has been converted.  D1 is free
+      // as soon as stage 2 of the slot's previous group has completed (it was that stage's A operand),
+      // so stage 1 of the next group runs while the previous one is still being quantised out of the D2
+      // columns; D2 is not written again before the group's warps have finished reading it, because
+      // they convert the next group (which is what lets its stage 2 go) only after that.
       int i1 = 0, i2 = 0;
       uint32_t idle = 0;
       while (ok && i2 < my_groups) {
         bool did = false;
         if (i1 < my_groups && i1 < i2 + S &&
             mbar_test_wait(&x_full[i1 % L.XS], (i1 / L.XS) & 1) &&
-            mbar_test_wait(&d_free[i1 % S], ((i1 / S) & 1) ^ 1)) {
+            mbar_test_wait(&d2_full[i1 % S], ((i1 / S) & 1) ^ 1)) {
           stage1(i1++);
           did = true;
         }
