@@ -93,7 +93,6 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
   uint64_t* d1_full = bars + 12;       // [4] each CTA's own copy
   uint64_t* a2_ready = bars + 16;      // [4] 8 warps of the pair (leader's copy is used)
   uint64_t* d2_full = bars + 20;       // [4] each CTA's own copy
-  uint64_t* d_free = bars + 24;        // [4] 8 warps of the pair (leader's copy is used)
   uint64_t* amax_bar = bars + 28;      // [4] the partner group's absmax has arrived (local)
   uint64_t* img_full = bars + 32;      // this CTA's factor images (local)
   uint64_t* peer_img = bars + 33;      // the partner's factor images (leader's copy is used)
@@ -124,7 +123,6 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
       mbar_init(&d1_full[b], 1);
       mbar_init(&a2_ready[b], 8);
       mbar_init(&d2_full[b], 1);
-      mbar_init(&d_free[b], 8);
       mbar_init(&amax_bar[b], 1);
     }
     mbar_init(img_full, 1);
@@ -315,11 +313,6 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
         uint32_t r[32];
         tmem_ld_32x32b_x32(d2 + 32 * c, r);
         tmem_wait_ld();
-        if (c == N2 / 32 - 1) {                      // last read of the slot
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive_cluster(&d_free[w], 0);
-        }
         float t[32];
 #pragma unroll
         for (int e = 0; e < 32; ++e) {

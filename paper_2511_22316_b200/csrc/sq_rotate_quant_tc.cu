@@ -153,7 +153,6 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
   uint64_t* d1_full = bars + 8;        // [4]
   uint64_t* a2_ready = bars + 12;      // [4]
   uint64_t* d2_full = bars + 16;       // [4]
-  uint64_t* d_free = bars + 20;        // [4]
   uint64_t* img_full = bars + 24;
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(bars + 25);
   float* amax_x = reinterpret_cast<float*>(bars + 26);      // [S groups][2 parities][4 warps]
@@ -195,7 +194,6 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
       mbar_init(&d1_full[b], 1);
       mbar_init(&a2_ready[b], 4);
       mbar_init(&d2_full[b], 1);
-      mbar_init(&d_free[b], 4);
     }
     mbar_fence_init();
   }
@@ -379,11 +377,6 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         uint32_t r[32];
         tmem_ld_32x32b_x32(d2 + 32 * c, r);
         tmem_wait_ld();
-        if (c == N2 / 32 - 1) {                      // last read of the slot: stage 1 may reuse it
-          tc_fence_before_sync();
-          __syncwarp();
-          if (lane == 0) mbar_arrive(&d_free[w]);
-        }
         float t[32];
 #pragma unroll
         for (int e = 0; e < 32; ++e) {
