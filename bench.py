@@ -39,11 +39,11 @@ INT8_OVER_BF16 = 2.0      # nominal dense ratio (4.5 POPS int8 : 2.25 PFLOP/s bf
 # profiles/ (bytes; None until a capture exists for that kernel and workload).
 NCU_TRAFFIC = {
     ("gemm", "llama2_7b_qkvo_prefill"): 12632320,           # w4a4_gemm_pair_kernel: reads (Y stays in L2)
-    ("rotate_quant", "llama2_7b_qkvo_prefill"): 16888320,   # rotate_quant_tc_kernel
+    ("rotate_quant", "llama2_7b_qkvo_prefill"): 16888064,   # rotate_quant_tc_kernel
     ("gemm", "llama3_8b_up_decode_m16"): 29457152,          # w4a4_gemm_decode_kernel, K not split
     ("gemm", "llama3_8b_down_decode_m16"): 29518848,        # w4a4_gemm_decode_kernel, K over clusters of 4
     ("gemm", "llama3_8b_up_decode_m1"): 29409280,           # w4a4_gemv_kernel
-    ("rotate_quant", "llama2_7b_down_prefill"): 45398528,   # rotate_quant_pair_kernel
+    ("rotate_quant", "llama2_7b_down_prefill"): 45403904,   # rotate_quant_pair_kernel
 }
 
 
