@@ -268,7 +268,7 @@ def run_ours(args, w):
     l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
     per_set = M * K * 2 + M * K // 2 + M * N * 2 + N * K // 2
     nsets = max(2, int(np.ceil(1.5 * l2 / per_set)) + 1)
-    ws_bytes = sq.sq_linear_workspace_bytes(M, N, K)
+    ws_bytes = sq.sq_linear_workspace_bytes(M, K)
     Xh = torch.from_numpy(X).pin_memory()
     sets = []
     for i in range(nsets):

@@ -13,7 +13,8 @@
  *
  * General conventions
  *   - Pointers marked HOST are ordinary host memory; pointers marked DEVICE are CUDA device
- *     memory of the device that was current when the rotation handle was created.  The
+ *     memory of the device that was current when the rotation handle was created.  A call that
+ *     takes a handle while another device is current returns SQ_ERR_INVALID_ARG.  The
  *     caller owns every buffer; the library allocates only the sq_rotation_t handle (and the
  *     device copies of R1, R2 inside it), freed by sq_rotation_destroy.
  *   - All matrices are dense row-major.  X is [M x n] (one token per row, ld = n), W is
@@ -96,7 +97,8 @@ void sq_rotation_destroy(sq_rotation_t* rot);
 
 /* Steps 1+2, fused: Z_t = R1^T X~_t R2 in fp32 on chip, Delta_t = fp16(max|Z_t|/7),
  * code = clamp(floor(fl(fl(z * fl(1/Delta)) + 0.5)), -8, 7) in fp32 arithmetic, packed.
- *   rot           handle; n = n1*n2 of the handle.  Supported: n even, n <= 32768.
+ *   rot           handle; n = n1*n2 of the handle.  Supported: n2 even (SQ_ERR_SHAPE otherwise),
+ *                 n <= 32768.
  *   X             DEVICE fp16 [M x n]
  *   Xq            DEVICE uint8 [M x n/2]   (out)
  *   sx            DEVICE fp16 [M]          (out; Delta_t; 0 for an all-zero row)
@@ -118,22 +120,19 @@ sq_status_t sq_pack_weight(const sq_rotation_t* rot_or_null, const void* W, int6
  *   Wq  DEVICE uint8 [N x K/2]     sw  DEVICE fp16 [N]
  *   Y   DEVICE fp16  [M x N] (out)
  *   accdbg_or_null  DEVICE int32 [M x N] (out, optional: the raw accumulators)
- *   workspace       DEVICE scratch of at least sq_w4a4_gemm_workspace_bytes(M,N,K) bytes, or
- *                   NULL.  Every kernel of this version keeps its intermediates on chip (split-K
- *                   partial tiles are exchanged through cluster shared memory), so the size is 0
- *                   for all shapes and the argument is not read; it stays in the signature so
- *                   that callers need not change if a later kernel wants scratch.
+ * No scratch memory: every kernel keeps its intermediates on chip (split-K partial tiles are
+ * exchanged through cluster shared memory).
  * Supported: K even, K <= 65536 (so that the 256x-scaled int32 accumulator cannot overflow).
  * The tensor-core path needs K % 128 == 0 and N % 8 == 0; other shapes run a plain integer
  * kernel with the same results. */
-size_t sq_w4a4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
 sq_status_t sq_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw,
                          int64_t M, int64_t N, int64_t K, void* Y, void* accdbg_or_null,
-                         void* workspace, size_t workspace_bytes, void* stream);
+                         void* stream);
 
 /* The whole layer on one stream: steps 1+2 into the workspace (Xq, sx), then step 3.
- *   workspace  DEVICE, at least sq_linear_workspace_bytes(M, N, K) bytes, 256-byte aligned */
-size_t sq_linear_workspace_bytes(int64_t M, int64_t N, int64_t K);
+ *   workspace  DEVICE, at least sq_linear_workspace_bytes(M, K) bytes, 256-byte aligned
+ * Every argument of both halves is validated before the first kernel is queued. */
+size_t sq_linear_workspace_bytes(int64_t M, int64_t K);
 sq_status_t sq_linear(const sq_rotation_t* rot, const void* X, int64_t M,
                       const void* Wq, const void* sw, int64_t N, int64_t K,
                       void* workspace, size_t workspace_bytes, void* Y, void* stream);
@@ -149,7 +148,7 @@ sq_status_t sq_linear(const sq_rotation_t* rot, const void* X, int64_t M,
  * image; every GPU that loads the library holds it until the process exits.
  *   - Arguments as sq_linear, minus the workspace.  All pointers DEVICE; the caller owns X, Wq,
  *     sw and Y.
- *   - Limit: sq_linear_workspace_bytes(M, N, K) <= SQ_LINEAR_STATIC_SCRATCH_BYTES, i.e. roughly
+ *   - Limit: sq_linear_workspace_bytes(M, K) <= SQ_LINEAR_STATIC_SCRATCH_BYTES, i.e. roughly
  *     M * K / 2 + 2 * M bytes (LLaMA-2-7B prefill, 2048 x 4096, needs 4.2 MB).  Larger problems
  *     return SQ_ERR_UNSUPPORTED before anything is launched: split M, or use sq_linear.
  *   - The first call on each device looks up the scratch's device address (a CUDA runtime query,
@@ -180,6 +179,14 @@ sq_status_t sq_linear_host(const sq_rotation_t* rot, const void* X_host, int64_t
 /* Synchronises `stream`, then returns and clears the device status word: SQ_OK, or
  * SQ_ERR_TIMEOUT if any kernel since the last call gave up a bounded wait, or SQ_ERR_CUDA. */
 sq_status_t sq_last_device_status(void* stream);
+
+/* Diagnostic (the paper has no counterpart): enqueues a one-thread kernel that waits, with the
+ * same bounded-wait routine the production kernels use, on a hardware barrier that nothing ever
+ * completes, for `polls` polls (1 .. 1000000), and then gives up.  Nothing else is in flight in
+ * that kernel.  A following sq_last_device_status(stream) therefore returns SQ_ERR_TIMEOUT once
+ * and SQ_OK afterwards, and the context stays usable: this is how the time-out reporting path is
+ * checked without hanging or faulting anything. */
+sq_status_t sq_debug_bounded_wait(uint32_t polls, void* stream);
 
 /* Number of kernels this library has launched in the calling process (monotonic counter). */
 uint64_t sq_kernel_launch_count(void);

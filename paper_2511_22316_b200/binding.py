@@ -25,9 +25,9 @@ SQ_ROT_ART, SQ_ROT_URT, SQ_ROT_HADAMARD, SQ_ROT_DEFAULT = 1, 2, 4, 7
 EXPORTS = (
     "sq_factorize", "sq_build_rotation", "sq_rotation_from_factors", "sq_rotation_get_factors",
     "sq_rotation_dims", "sq_rotation_destroy", "sq_rotate_quant_act", "sq_pack_weight",
-    "sq_w4a4_gemm_workspace_bytes", "sq_w4a4_gemm", "sq_linear_workspace_bytes", "sq_linear",
+    "sq_w4a4_gemm", "sq_linear_workspace_bytes", "sq_linear",
     "sq_linear_static", "sq_linear_host_workspace_bytes", "sq_linear_host", "sq_last_device_status",
-    "sq_kernel_launch_count", "sq_status_string",
+    "sq_debug_bounded_wait", "sq_kernel_launch_count", "sq_status_string",
 )
 
 
@@ -59,11 +59,9 @@ def load() -> ctypes.CDLL:
     lib.sq_rotation_destroy.restype = None
     lib.sq_rotate_quant_act.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
     lib.sq_pack_weight.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_void_p, c_void_p, c_void_p]
-    lib.sq_w4a4_gemm_workspace_bytes.argtypes = [c_int64, c_int64, c_int64]
-    lib.sq_w4a4_gemm_workspace_bytes.restype = c_size_t
     lib.sq_w4a4_gemm.argtypes = [c_void_p, c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64,
-                                 c_void_p, c_void_p, c_void_p, c_size_t, c_void_p]
-    lib.sq_linear_workspace_bytes.argtypes = [c_int64, c_int64, c_int64]
+                                 c_void_p, c_void_p, c_void_p]
+    lib.sq_linear_workspace_bytes.argtypes = [c_int64, c_int64]
     lib.sq_linear_workspace_bytes.restype = c_size_t
     lib.sq_linear.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_int64,
                               c_void_p, c_size_t, c_void_p, c_void_p]
@@ -74,6 +72,7 @@ def load() -> ctypes.CDLL:
     lib.sq_linear_host.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_int64,
                                    c_void_p, c_size_t, c_void_p, c_void_p]
     lib.sq_last_device_status.argtypes = [c_void_p]
+    lib.sq_debug_bounded_wait.argtypes = [c_uint32, c_void_p]
     lib.sq_kernel_launch_count.argtypes = []
     lib.sq_kernel_launch_count.restype = c_uint64
     lib.sq_status_string.argtypes = [ctypes.c_int]
@@ -200,18 +199,13 @@ def sq_pack_weight(rot: Optional[Rotation], W, N: int, K: int, Wq, sw, stream=No
                                  _stream(stream)), "sq_pack_weight")
 
 
-def sq_w4a4_gemm_workspace_bytes(M: int, N: int, K: int) -> int:
-    return int(load().sq_w4a4_gemm_workspace_bytes(M, N, K))
-
-
-def sq_w4a4_gemm(Xq, sx, Wq, sw, M: int, N: int, K: int, Y, accdbg=None, workspace=None, workspace_bytes: int = 0,
-                 stream=None) -> None:
+def sq_w4a4_gemm(Xq, sx, Wq, sw, M: int, N: int, K: int, Y, accdbg=None, stream=None) -> None:
     _check(load().sq_w4a4_gemm(_ptr(Xq), _ptr(sx), _ptr(Wq), _ptr(sw), M, N, K, _ptr(Y), _ptr(accdbg),
-                               _ptr(workspace), workspace_bytes, _stream(stream)), "sq_w4a4_gemm")
+                               _stream(stream)), "sq_w4a4_gemm")
 
 
-def sq_linear_workspace_bytes(M: int, N: int, K: int) -> int:
-    return int(load().sq_linear_workspace_bytes(M, N, K))
+def sq_linear_workspace_bytes(M: int, K: int) -> int:
+    return int(load().sq_linear_workspace_bytes(M, K))
 
 
 def sq_linear(rot: Rotation, X, M: int, Wq, sw, N: int, K: int, workspace, workspace_bytes: int, Y,
@@ -243,6 +237,11 @@ def sq_linear_host(rot: Rotation, X_host, M: int, Wq, sw, N: int, K: int, worksp
 
 def sq_last_device_status(stream=None) -> int:
     return int(load().sq_last_device_status(_stream(stream)))
+
+
+def sq_debug_bounded_wait(polls: int, stream=None) -> None:
+    """Enqueues the diagnostic kernel whose only wait runs out after `polls` polls (see the header)."""
+    _check(load().sq_debug_bounded_wait(int(polls), _stream(stream)), "sq_debug_bounded_wait")
 
 
 def sq_kernel_launch_count() -> int:

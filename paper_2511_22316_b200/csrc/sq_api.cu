@@ -62,11 +62,22 @@ sq_status_t read_and_clear_device_status(cudaStream_t s) {
 extern "C" void sq_rotation_destroy(sq_rotation_t* rot);
 
 namespace sq {
+// One thread, one barrier that nobody arrives at, the library's own bounded wait: it gives up after
+// `polls` polls, records its site in the status word and returns.  No copy, MMA or TMEM allocation
+// is in flight when it does.
+__global__ void bounded_wait_probe_kernel(uint32_t polls) {
+  __shared__ uint64_t bar;
+  mbar_init(&bar, 1);
+  mbar_fence_init();
+  mbar_wait(&bar, 0, /*site=*/255u, polls);
+}
+}  // namespace sq
+
+namespace sq {
 sq_status_t rotate_quant_dispatch(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
                                   float* Zdbg, cudaStream_t s) {
-  static const bool force_generic = getenv("SQ_ROTATE_GENERIC") != nullptr;
-  if (h->tc_ready && !force_generic) return launch_rotate_quant_tc(h, X, rows, Xq, scales, Zdbg, s);
-  if (h->tc_pair && !force_generic) return launch_rotate_quant_pair(h, X, rows, Xq, scales, Zdbg, s);
+  if (h->tc_ready) return launch_rotate_quant_tc(h, X, rows, Xq, scales, Zdbg, s);
+  if (h->tc_pair) return launch_rotate_quant_pair(h, X, rows, Xq, scales, Zdbg, s);
   return launch_rotate_quant(h->dR1, h->dR2, h->n1, h->n2, X, rows, Xq, scales, Zdbg, s);
 }
 }  // namespace sq
@@ -136,18 +147,31 @@ sq_status_t check_gemm_args(const void* Xq, const void* sx, const void* Wq, cons
   return SQ_OK;
 }
 
+// A handle's factors live on the device that was current when it was made; a call with another
+// device current would hand that GPU's kernels pointers into this one's memory.
+sq_status_t check_handle_device(const sq_rotation* rot) {
+  int dev = -1;
+  if (cudaGetDevice(&dev) != cudaSuccess) return SQ_ERR_CUDA;
+  return dev == rot->device ? SQ_OK : SQ_ERR_INVALID_ARG;
+}
+
 }  // namespace
 
 extern "C" {
 
 sq_status_t sq_factorize(int64_t n, int32_t* n1, int32_t* n2) {
   if (!n1 || !n2 || n < 1 || n > (1ll << 40)) return SQ_ERR_INVALID_ARG;
-  const double root = std::sqrt(static_cast<double>(n));
-  int64_t best = 1;
-  for (int64_t a = 1; a <= n; a *= 2) {
-    if (n % a != 0) continue;
-    if (std::fabs(static_cast<double>(a) - root) < std::fabs(static_cast<double>(best) - root)) best = a;
-  }
+  // The powers of two that divide n are 2^0 .. 2^v, v = number of trailing zero bits of n.  The one
+  // nearest to sqrt(n) is one of the two powers of two that bracket sqrt(n), each clipped to 2^v:
+  // lo = 2^e with 4^e <= n < 4^(e+1), hi = 2 lo.  "lo is at least as near as hi" is
+  // sqrt(n) - lo <= hi - sqrt(n), i.e. 4 n <= 9 lo^2 in exact integer arithmetic; the smaller power
+  // wins a tie (Algorithm 1 keeps the first candidate it meets, and it meets them in rising order).
+  const int v = __builtin_ctzll(static_cast<unsigned long long>(n));
+  int e = 0;
+  while ((4ll << (2 * e)) <= n) ++e;                       // largest e with 4^e <= n
+  int64_t lo = 1ll << (e < v ? e : v);
+  int64_t hi = 1ll << (e + 1 < v ? e + 1 : v);
+  const int64_t best = (hi == lo || 4 * n <= 9 * lo * lo) ? lo : hi;
   if (n / best > INT32_MAX) return SQ_ERR_UNSUPPORTED;
   *n1 = static_cast<int32_t>(n / best);
   *n2 = static_cast<int32_t>(best);
@@ -208,6 +232,7 @@ sq_status_t sq_rotate_quant_act(const sq_rotation_t* rot, const void* X, int64_t
   if (rot->n2 & 1) return SQ_ERR_SHAPE;
   sq_status_t st = check_rows_args(X, Xq, sx, Zdbg_or_null, M, n);
   if (st != SQ_OK || M == 0) return st;
+  if ((st = check_handle_device(rot)) != SQ_OK) return st;
   return sq::rotate_quant_dispatch(rot, X, M, Xq, sx, static_cast<float*>(Zdbg_or_null),
                                    static_cast<cudaStream_t>(stream));
 }
@@ -220,54 +245,52 @@ sq_status_t sq_pack_weight(const sq_rotation_t* rot_or_null, const void* W, int6
   }
   sq_status_t st = check_rows_args(W, Wq, sw, nullptr, N, K);
   if (st != SQ_OK || N == 0) return st;
+  if (rot_or_null && (st = check_handle_device(rot_or_null)) != SQ_OK) return st;
   if (rot_or_null)
     return sq::rotate_quant_dispatch(rot_or_null, W, N, Wq, sw, nullptr, static_cast<cudaStream_t>(stream));
   return sq::launch_rotate_quant(nullptr, nullptr, 1, static_cast<int>(K), W, N, Wq, sw, nullptr,
                                  static_cast<cudaStream_t>(stream));
 }
 
-size_t sq_w4a4_gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
-  if (M <= 0 || N <= 0 || K <= 0) return 0;
-  return sq::gemm_workspace_bytes(M, N, K);
-}
-
 sq_status_t sq_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw, int64_t M, int64_t N,
-                         int64_t K, void* Y, void* accdbg_or_null, void* workspace, size_t workspace_bytes,
-                         void* stream) {
+                         int64_t K, void* Y, void* accdbg_or_null, void* stream) {
   sq_status_t st = check_gemm_args(Xq, sx, Wq, sw, M, N, K, Y, accdbg_or_null);
   if (st != SQ_OK || M == 0 || N == 0) return st;
-  if (workspace && !sq::aligned16(workspace)) return SQ_ERR_ALIGN;
-  return sq::launch_w4a4_gemm(Xq, sx, Wq, sw, M, N, K, Y, static_cast<int32_t*>(accdbg_or_null), workspace,
-                              workspace ? workspace_bytes : 0, static_cast<cudaStream_t>(stream));
+  return sq::launch_w4a4_gemm(Xq, sx, Wq, sw, M, N, K, Y, static_cast<int32_t*>(accdbg_or_null),
+                              static_cast<cudaStream_t>(stream));
 }
 
-// Workspace layout of sq_linear: [Xq: M*K/2][sx: 2*M][GEMM scratch], each 256-byte aligned.
-size_t sq_linear_workspace_bytes(int64_t M, int64_t N, int64_t K) {
-  if (M <= 0 || N <= 0 || K <= 0) return 0;
-  return align_up(static_cast<size_t>(M) * (K / 2), 256) + align_up(static_cast<size_t>(M) * 2, 256) +
-         align_up(sq::gemm_workspace_bytes(M, N, K), 256);
+// Workspace layout of sq_linear: [Xq: M*K/2][sx: 2*M], each 256-byte aligned.
+size_t sq_linear_workspace_bytes(int64_t M, int64_t K) {
+  if (M <= 0 || K <= 0) return 0;
+  return align_up(static_cast<size_t>(M) * (K / 2), 256) + align_up(static_cast<size_t>(M) * 2, 256);
 }
 
 sq_status_t sq_linear(const sq_rotation_t* rot, const void* X, int64_t M, const void* Wq, const void* sw,
                       int64_t N, int64_t K, void* workspace, size_t workspace_bytes, void* Y, void* stream) {
   if (!rot) return SQ_ERR_INVALID_ARG;
   if (static_cast<int64_t>(rot->n1) * rot->n2 != K) return SQ_ERR_SHAPE;
+  if (rot->n2 & 1) return SQ_ERR_SHAPE;
   if (M < 0 || N < 0) return SQ_ERR_INVALID_ARG;
   if (M == 0 || N == 0) return SQ_OK;
   if (!workspace) return SQ_ERR_INVALID_ARG;
   if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQ_ERR_ALIGN;
-  if (workspace_bytes < sq_linear_workspace_bytes(M, N, K)) return SQ_ERR_NOMEM;
+  if (workspace_bytes < sq_linear_workspace_bytes(M, K)) return SQ_ERR_NOMEM;
   unsigned char* ws = static_cast<unsigned char*>(workspace);
   void* Xq = ws;
   void* sx = ws + align_up(static_cast<size_t>(M) * (K / 2), 256);
-  void* gws = static_cast<unsigned char*>(sx) + align_up(static_cast<size_t>(M) * 2, 256);
-  const size_t gws_bytes = sq::gemm_workspace_bytes(M, N, K);
-  sq_status_t st = sq_rotate_quant_act(rot, X, M, Xq, sx, nullptr, stream);
+  // Both halves are validated before anything is queued.
+  sq_status_t st = check_rows_args(X, Xq, sx, nullptr, M, K);
+  if (st != SQ_OK) return st;
+  if ((st = check_gemm_args(Xq, sx, Wq, sw, M, N, K, Y, nullptr)) != SQ_OK) return st;
+  if ((st = check_handle_device(rot)) != SQ_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = sq::rotate_quant_dispatch(rot, X, M, Xq, sx, nullptr, s);
   if (st != SQ_OK) return st;
   // Every tensor-core GEMM kernel and the dot-product kernel start their set-up (and their weight
   // loads) while the rotate kernel drains; they wait for it before they read Xq or sx.
   sq::g_pdl_next = true;
-  st = sq_w4a4_gemm(Xq, sx, Wq, sw, M, N, K, Y, nullptr, gws_bytes ? gws : nullptr, gws_bytes, stream);
+  st = sq::launch_w4a4_gemm(Xq, sx, Wq, sw, M, N, K, Y, nullptr, s);
   sq::g_pdl_next = false;
   return st;
 }
@@ -276,7 +299,7 @@ sq_status_t sq_linear(const sq_rotation_t* rot, const void* X, int64_t M, const 
 size_t sq_linear_host_workspace_bytes(int64_t M, int64_t N, int64_t K) {
   if (M <= 0 || N <= 0 || K <= 0) return 0;
   return align_up(static_cast<size_t>(M) * K * 2, 256) + align_up(static_cast<size_t>(M) * N * 2, 256) +
-         sq_linear_workspace_bytes(M, N, K);
+         sq_linear_workspace_bytes(M, K);
 }
 
 namespace {
@@ -328,19 +351,30 @@ sq_status_t sq_linear_host(const sq_rotation_t* rot, const void* X_host, int64_t
   unsigned char* dX = ws;
   unsigned char* dY = ws + align_up(xb, 256);
   void* lws = dY + align_up(yb, 256);
-  const size_t lws_bytes = sq_linear_workspace_bytes(M, N, K);
+  const size_t lws_bytes = sq_linear_workspace_bytes(M, K);
+  // Everything sq_linear would refuse is refused here, before the first copy is queued.
+  if (static_cast<int64_t>(rot->n1) * rot->n2 != K || (rot->n2 & 1)) return SQ_ERR_SHAPE;
+  {
+    unsigned char* lw = static_cast<unsigned char*>(lws);
+    sq_status_t pre = check_rows_args(dX, lw, lw + align_up(static_cast<size_t>(M) * (K / 2), 256), nullptr, M, K);
+    if (pre == SQ_OK) pre = check_gemm_args(lw, lw, Wq, sw, M, N, K, dY, nullptr);
+    if (pre == SQ_OK) pre = check_handle_device(rot);
+    if (pre != SQ_OK) return pre;
+  }
   // Chunks of at least 256 rows (a full tile of the prefill GEMM), a multiple of 256 rows each.
   int64_t chunk_rows = M;
   if (M >= 512) chunk_rows = ((M + kHostChunks - 1) / kHostChunks + 255) / 256 * 256;
   const int chunks = static_cast<int>((M + chunk_rows - 1) / chunk_rows);
   HostPipe* p = chunks > 1 ? host_pipe() : nullptr;
   if (chunks == 1 || p == nullptr) {
+    // Whatever fails after the first copy is queued, the stream is drained before returning: no
+    // copy from or to the caller's host buffers outlives the call.
+    sq_status_t st = SQ_OK;
     if (cudaMemcpyAsync(dX, X_host, xb, cudaMemcpyHostToDevice, s) != cudaSuccess) return SQ_ERR_CUDA;
-    sq_status_t st = sq_linear(rot, dX, M, Wq, sw, N, K, lws, lws_bytes, dY, stream);
-    if (st != SQ_OK) return st;
-    if (cudaMemcpyAsync(Y_host, dY, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) return SQ_ERR_CUDA;
-    if (cudaStreamSynchronize(s) != cudaSuccess) return SQ_ERR_CUDA;
-    return SQ_OK;
+    st = sq_linear(rot, dX, M, Wq, sw, N, K, lws, lws_bytes, dY, stream);
+    if (st == SQ_OK && cudaMemcpyAsync(Y_host, dY, yb, cudaMemcpyDeviceToHost, s) != cudaSuccess) st = SQ_ERR_CUDA;
+    if (cudaStreamSynchronize(s) != cudaSuccess && st == SQ_OK) st = SQ_ERR_CUDA;
+    return st;
   }
   // Everything follows what is already queued on the caller's stream.
   if (cudaEventRecord(p->start, s) != cudaSuccess || cudaStreamWaitEvent(p->h2d, p->start, 0) != cudaSuccess ||
@@ -372,6 +406,13 @@ sq_status_t sq_linear_host(const sq_rotation_t* rot, const void* X_host, int64_t
 
 sq_status_t sq_last_device_status(void* stream) {
   return sq::read_and_clear_device_status(static_cast<cudaStream_t>(stream));
+}
+
+sq_status_t sq_debug_bounded_wait(uint32_t polls, void* stream) {
+  if (polls < 1 || polls > 1000000u) return SQ_ERR_INVALID_ARG;
+  sq::bounded_wait_probe_kernel<<<1, 1, 0, static_cast<cudaStream_t>(stream)>>>(polls);
+  sq::count_launch();
+  return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
 }
 
 uint64_t sq_kernel_launch_count(void) { return sq::g_launches.load(std::memory_order_relaxed); }

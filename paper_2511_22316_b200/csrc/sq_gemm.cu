@@ -293,25 +293,28 @@ w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
 }
 
 // Plain integer kernel for shapes the tensor-core path does not take (K % 128 != 0, N % 8 != 0):
-// one thread per output, byte-wise.  Same results, bit for bit.
+// one thread per output, byte-wise; gridDim.y strides over the token rows (a grid's y extent stops
+// at 65535).  Same results, bit for bit.
 __global__ void w4a4_gemm_simple_kernel(const uint8_t* __restrict__ Xq, const __half* __restrict__ sx,
                                         const uint8_t* __restrict__ Wq, const __half* __restrict__ sw,
                                         int M, int N, int K, __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
   const int c = blockIdx.x * blockDim.x + threadIdx.x;
-  const int t = blockIdx.y;
-  if (c >= N || t >= M) return;
-  const uint8_t* a = Xq + static_cast<size_t>(t) * (K / 2);
+  if (c >= N) return;
   const uint8_t* b = Wq + static_cast<size_t>(c) * (K / 2);
-  int32_t acc = 0;
-  for (int j = 0; j < K / 2; ++j) {
-    const int av = a[j], bv = b[j];
-    const int a0 = (av << 28) >> 28, a1 = (av << 24) >> 28;      // sign-extended nibbles
-    const int b0 = (bv << 28) >> 28, b1 = (bv << 24) >> 28;
-    acc += a0 * b0 + a1 * b1;
+  const float swv = __half2float(sw[c]);
+  for (int t = blockIdx.y; t < M; t += gridDim.y) {
+    const uint8_t* a = Xq + static_cast<size_t>(t) * (K / 2);
+    int32_t acc = 0;
+    for (int j = 0; j < K / 2; ++j) {
+      const int av = a[j], bv = b[j];
+      const int a0 = (av << 28) >> 28, a1 = (av << 24) >> 28;      // sign-extended nibbles
+      const int b0 = (bv << 28) >> 28, b1 = (bv << 24) >> 28;
+      acc += a0 * b0 + a1 * b1;
+    }
+    const float s = __half2float(sx[t]) * swv;
+    Y[static_cast<size_t>(t) * N + c] = __float2half_rn(static_cast<float>(acc) * s);
+    if (accdbg) accdbg[static_cast<size_t>(t) * N + c] = acc;
   }
-  const float s = __half2float(sx[t]) * __half2float(sw[c]);
-  Y[static_cast<size_t>(t) * N + c] = __float2half_rn(static_cast<float>(acc) * s);
-  if (accdbg) accdbg[static_cast<size_t>(t) * N + c] = acc;
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -377,17 +380,12 @@ static bool use_gemv(int64_t M, int64_t N, int64_t K) {
   return gemv_supported(M, N, K) && (M <= 2 || !gemm_decode_supported(M, N, K));
 }
 
-size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K) {
-  return use_gemv(M, N, K) ? 0 : gemm_decode_workspace_bytes(M, N, K);
-}
-
 sq_status_t launch_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw, int64_t M, int64_t N,
-                             int64_t K, void* Y, int32_t* accdbg, void* workspace, size_t workspace_bytes,
-                             cudaStream_t s) {
+                             int64_t K, void* Y, int32_t* accdbg, cudaStream_t s) {
   if (M == 0 || N == 0) return SQ_OK;
   if (use_gemv(M, N, K)) return launch_w4a4_gemv(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
   if (gemm_decode_supported(M, N, K))
-    return launch_w4a4_gemm_decode(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, workspace, workspace_bytes, s);
+    return launch_w4a4_gemm_decode(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
   const bool tc_ok = (K % BK == 0) && (N % 8 == 0) && K >= BK;
   if (gemm_pair_supported(M, N, K))
     return launch_w4a4_gemm_pair(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
@@ -408,20 +406,19 @@ sq_status_t launch_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, con
     const int clusters = sms / split > 0 ? sms / split : 1;
     const double dec_us = 2.0 * (8.0 + 0.46 * ((num_sb + split - 1) / split) * ((dec_tiles + clusters - 1) / clusters));
     if (pair_us <= dec_us) return launch_w4a4_gemm_pair(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
-    const sq_status_t st = launch_w4a4_gemm_decode(Xq, sx, Wq, sw, 64, (int)N, (int)K, Y, accdbg, nullptr, 0, s);
+    const sq_status_t st = launch_w4a4_gemm_decode(Xq, sx, Wq, sw, 64, (int)N, (int)K, Y, accdbg, s);
     if (st != SQ_OK) return st;
     const size_t half = 64;
     return launch_w4a4_gemm_decode(static_cast<const unsigned char*>(Xq) + half * (K / 2),
                                    static_cast<const __half*>(sx) + half, Wq, sw, (int)(M - 64), (int)N, (int)K,
-                                   static_cast<__half*>(Y) + half * N, accdbg ? accdbg + half * N : nullptr, nullptr, 0,
-                                   s);
+                                   static_cast<__half*>(Y) + half * N, accdbg ? accdbg + half * N : nullptr, s);
   }
   if (tc_ok) {
     if (N >= 256 && M > 64)
       return launch_tc<256, 2, 2>(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
     return launch_tc<128, 3, 3>(Xq, sx, Wq, sw, (int)M, (int)N, (int)K, Y, accdbg, s);
   }
-  dim3 block(128), grid((unsigned)((N + 127) / 128), (unsigned)M);
+  dim3 block(128), grid((unsigned)((N + 127) / 128), (unsigned)(M < 65535 ? M : 65535));
   w4a4_gemm_simple_kernel<<<grid, block, 0, s>>>(static_cast<const uint8_t*>(Xq), static_cast<const __half*>(sx),
                                                  static_cast<const uint8_t*>(Wq), static_cast<const __half*>(sw),
                                                  (int)M, (int)N, (int)K, static_cast<__half*>(Y), accdbg);

@@ -13,7 +13,7 @@
 // receives, from each of the others, the 128 / s rows it finishes (one slot per source, written
 // with st.shared::cluster and handed over with a cluster-scope release/acquire barrier), adds
 // them to its own rows, dequantises and writes fp16.  Integer addition makes the result
-// independent of any order; no partial tile, counter or workspace exists in global memory.
+// independent of any order; no partial tile, counter or scratch exists in global memory.
 //
 // Warp roles: warp 0 = TMA producer, warp 1 = MMA issuer, warps 2..9 = two groups of weight
 // converters and warps 10..13 = two groups of token unpackers (a group takes every other block:
@@ -564,11 +564,8 @@ bool gemm_decode_supported(int64_t M, int64_t N, int64_t K) {
   return M >= 1 && M <= 64 && N >= 128 && (K % 128 == 0) && K >= 256 && (N % 8 == 0);
 }
 
-// The split-K exchange lives in shared memory: no workspace.
-size_t gemm_decode_workspace_bytes(int64_t, int64_t, int64_t) { return 0; }
-
 sq_status_t launch_w4a4_gemm_decode(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N, int K,
-                                    void* Y, int32_t* accdbg, void*, size_t, cudaStream_t s) {
+                                    void* Y, int32_t* accdbg, cudaStream_t s) {
   if (M <= 16) return launch_decode<16>(Xq, sx, Wq, sw, M, N, K, Y, accdbg, s);
   if (M <= 32) return launch_decode<32>(Xq, sx, Wq, sw, M, N, K, Y, accdbg, s);
   return launch_decode<64>(Xq, sx, Wq, sw, M, N, K, Y, accdbg, s);

@@ -99,10 +99,8 @@ sq_status_t rotate_quant_dispatch(const sq_rotation* h, const void* X, int64_t r
                                   float* Zdbg, cudaStream_t s);
 
 // Step 3 (sq_gemm.cu).
-size_t gemm_workspace_bytes(int64_t M, int64_t N, int64_t K);
 sq_status_t launch_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw,
-                             int64_t M, int64_t N, int64_t K, void* Y, int32_t* accdbg,
-                             void* workspace, size_t workspace_bytes, cudaStream_t s);
+                             int64_t M, int64_t N, int64_t K, void* Y, int32_t* accdbg, cudaStream_t s);
 
 // Step 3 on CTA pairs (sq_gemm_pair.cu): prefill-sized problems.
 bool gemm_pair_supported(int64_t M, int64_t N, int64_t K);
@@ -110,12 +108,10 @@ sq_status_t launch_w4a4_gemm_pair(const void* Xq, const void* sx, const void* Wq
                                   int K, void* Y, int32_t* accdbg, cudaStream_t s);
 
 // Step 3 for decode-sized problems (sq_gemm_decode.cu): weights as the A operand, K split over a
-// thread-block cluster with the partial tiles exchanged on chip (the workspace arguments are unused
-// and the size is 0; they remain for a kernel that wants scratch).
+// thread-block cluster with the partial tiles exchanged on chip (no scratch in global memory).
 bool gemm_decode_supported(int64_t M, int64_t N, int64_t K);
-size_t gemm_decode_workspace_bytes(int64_t M, int64_t N, int64_t K);
 sq_status_t launch_w4a4_gemm_decode(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N, int K,
-                                    void* Y, int32_t* accdbg, void* workspace, size_t workspace_bytes, cudaStream_t s);
+                                    void* Y, int32_t* accdbg, cudaStream_t s);
 
 // Step 3 for one to four tokens (sq_gemv.cu): dot products on the CUDA cores.
 bool gemv_supported(int64_t M, int64_t N, int64_t K);

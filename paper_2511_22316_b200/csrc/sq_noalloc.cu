@@ -42,7 +42,7 @@ extern "C" sq_status_t sq_linear_static(const sq_rotation_t* rot, const void* X,
                                         const void* sw, int64_t N, int64_t K, void* Y, void* stream) {
   if (!rot || M < 0 || N < 0 || K < 2) return SQ_ERR_INVALID_ARG;
   if (M == 0 || N == 0) return SQ_OK;
-  const size_t need = sq_linear_workspace_bytes(M, N, K);
+  const size_t need = sq_linear_workspace_bytes(M, K);
   if (need > static_cast<size_t>(SQ_LINEAR_STATIC_SCRATCH_BYTES)) return SQ_ERR_UNSUPPORTED;
   void* scratch = static_scratch_ptr();
   if (scratch == nullptr) return SQ_ERR_CUDA;

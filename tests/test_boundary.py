@@ -53,6 +53,33 @@ def test_factorize_matches_hand_traces(lib):
     assert lib.sq_factorize(16, None, ctypes.byref(b)) == sq.SQ_ERR_INVALID_ARG
 
 
+def test_factorize_is_the_nearest_power_of_two_divisor(lib):
+    """Algorithm 1 by its definition, in exact integer arithmetic: among the powers of two a that
+    divide n, the one minimising |a - sqrt(n)|, the smaller one on a tie.  |a - r| < |b - r| for
+    a < b (r = sqrt(n)) is decided without square roots: a wins iff a + b >= 2r iff (a + b)^2 >= 4n
+    when both lie on different sides, and the nearer to r otherwise."""
+    def nearest(n):
+        cands = [1 << k for k in range(n.bit_length()) if n % (1 << k) == 0]
+        best = cands[0]
+        for a in cands[1:]:
+            # is a strictly closer to sqrt(n) than best (best < a)?
+            if a * a <= n:                      # both at or below the root: the larger is closer
+                best = a
+            elif best * best >= n:              # both at or above: the smaller stays
+                pass
+            elif (a + best) ** 2 < 4 * n:       # opposite sides: a closer iff a - r < r - best
+                best = a
+        return n // best, best
+    for n in list(range(1, 3000)) + [4096, 5120, 8192, 11008, 14336, 28672, 2 ** 20, 2 ** 21, 9 * 2 ** 18, 2 ** 31 - 1,
+                                     3 * 2 ** 30, 2 ** 40]:
+        assert sq.sq_factorize(n) == nearest(n), n
+
+
+def test_debug_bounded_wait_rejects_bad_poll_counts(lib):
+    assert lib.sq_debug_bounded_wait(0, None) == sq.SQ_ERR_INVALID_ARG
+    assert lib.sq_debug_bounded_wait(2000000, None) == sq.SQ_ERR_INVALID_ARG
+
+
 def test_status_strings(lib):
     seen = set()
     for code in range(8):
@@ -79,15 +106,15 @@ def test_build_rotation_rejects_bad_shapes(lib):
 def test_gemm_rejects_bad_arguments_before_launch(lib):
     g = lib.sq_w4a4_gemm
     p = 0x1000          # never dereferenced: every case below fails validation first
-    assert g(p, p, p, p, 4, 8, 7, p, None, None, 0, None) == sq.SQ_ERR_SHAPE          # odd K
-    assert g(p, p, p, p, 4, 8, 0, p, None, None, 0, None) == sq.SQ_ERR_SHAPE
-    assert g(p, p, p, p, 4, 8, 1 << 20, p, None, None, 0, None) == sq.SQ_ERR_UNSUPPORTED
-    assert g(p, p, p, p, -1, 8, 128, p, None, None, 0, None) == sq.SQ_ERR_INVALID_ARG
-    assert g(None, p, p, p, 4, 8, 128, p, None, None, 0, None) == sq.SQ_ERR_INVALID_ARG
-    assert g(p + 4, p, p, p, 4, 8, 128, p, None, None, 0, None) == sq.SQ_ERR_ALIGN
-    assert g(p, p, p, p, 4, 8, 128, p, p + 8, None, 0, None) == sq.SQ_ERR_ALIGN
-    assert g(p, p, p, p, 0, 8, 128, p, None, None, 0, None) == sq.SQ_OK                # M = 0: no-op
-    assert g(None, None, None, None, 0, 0, 128, None, None, None, 0, None) == sq.SQ_OK
+    assert g(p, p, p, p, 4, 8, 7, p, None, None) == sq.SQ_ERR_SHAPE          # odd K
+    assert g(p, p, p, p, 4, 8, 0, p, None, None) == sq.SQ_ERR_SHAPE
+    assert g(p, p, p, p, 4, 8, 1 << 20, p, None, None) == sq.SQ_ERR_UNSUPPORTED
+    assert g(p, p, p, p, -1, 8, 128, p, None, None) == sq.SQ_ERR_INVALID_ARG
+    assert g(None, p, p, p, 4, 8, 128, p, None, None) == sq.SQ_ERR_INVALID_ARG
+    assert g(p + 4, p, p, p, 4, 8, 128, p, None, None) == sq.SQ_ERR_ALIGN
+    assert g(p, p, p, p, 4, 8, 128, p, p + 8, None) == sq.SQ_ERR_ALIGN
+    assert g(p, p, p, p, 0, 8, 128, p, None, None) == sq.SQ_OK                # M = 0: no-op
+    assert g(None, None, None, None, 0, 0, 128, None, None, None) == sq.SQ_OK
 
 
 def test_rows_calls_reject_null_handle_and_bad_sizes(lib):
@@ -104,8 +131,8 @@ def test_rows_calls_reject_null_handle_and_bad_sizes(lib):
 
 
 def test_workspace_sizes(lib):
-    assert sq.sq_linear_workspace_bytes(0, 8, 128) == 0
-    w = sq.sq_linear_workspace_bytes(2048, 4096, 4096)
+    assert sq.sq_linear_workspace_bytes(0, 128) == 0
+    w = sq.sq_linear_workspace_bytes(2048, 4096)
     assert w >= 2048 * 2048 + 2 * 2048 and w % 256 == 0
     h = sq.sq_linear_host_workspace_bytes(2048, 4096, 4096)
     assert h >= w + 2 * 2048 * 4096 * 2

@@ -215,6 +215,32 @@ def test_urt_degenerate():
     assert np.allclose(V @ RU, ora.uniform_target(V), atol=1e-12)
 
 
+@pytest.mark.parametrize("scale", [1.0, 1e6, 1e-6])
+def test_near_ties_in_outlier_minimum_and_rank(scale):
+    """Magnitudes within a RELATIVE 1e-9 count as tied and the lowest index wins (ART's outlier and
+    minimum; URT's rank order keeps the index order); magnitudes 1e-6 apart do not tie.  Expected
+    indices and targets are written out by hand; scaling the vector by 1e6 or 1e-6 must change
+    nothing (an absolute tolerance would flip the first case at 1e6 and the second at 1e-6)."""
+    e12, e6 = 1e-12, 1e-6
+    # |c_1| = 5 and |c_2| = 5(1 + 1e-12) tie for the outlier -> i = 1;
+    # |c_0| = 0.5(1 + 1e-12) and |c_3| = 0.5 tie for the minimum -> j = 0
+    c = scale * np.array([0.5 * (1 + e12), -5.0, 5.0 * (1 + e12), 0.5, 2.0])
+    assert ora.art_indices(c) == (1, 0)
+    # 1e-6 apart: the larger one is the outlier (i = 2), the smaller one the minimum (j = 3)
+    c = scale * np.array([0.5 * (1 + e6), -5.0, 5.0 * (1 + e6), 0.5, 2.0])
+    assert ora.art_indices(c) == (2, 3)
+    # URT target for n = 4: q = (-3, -1, 1, 3)/4, ||q||^2 = 5/4.
+    # V = (1 + 1e-12, 3, 1, -2): entries 0 and 2 tie, so the ascending order is 3, 0, 2, 1 (index order
+    # inside the tie) and U = ||V||/||q|| * (-1/4, 3/4, 1/4, -3/4) with ||V||^2 = 15 (+ 2e-12).
+    V = scale * np.array([1.0 * (1 + e12), 3.0, 1.0, -2.0])
+    s = scale * math.sqrt(15.0 / 1.25)
+    assert np.allclose(ora.uniform_target(V), s * np.array([-0.25, 0.75, 0.25, -0.75]), rtol=1e-11, atol=0)
+    # 1e-6 apart: entry 2 (1.0) now ranks below entry 0 -> order 3, 2, 0, 1
+    V = scale * np.array([1.0 * (1 + e6), 3.0, 1.0, -2.0])
+    s = scale * math.sqrt((15.0 + 2e-6 + 1e-12) / 1.25)
+    assert np.allclose(ora.uniform_target(V), s * np.array([0.25, 0.75, -0.25, -0.75]), rtol=1e-11, atol=0)
+
+
 # ---------------------------------------------------------------- Hadamard (P7)
 @pytest.mark.parametrize("n", [1, 2, 4, 32, 128])
 def test_hadamard(n):

@@ -42,7 +42,7 @@ def test_static_scratch_matches_workspace_path_twice_in_a_row(sq):
         X, W, R1, R2, rot, wq, sw = _layer(sq, w)
         M, N, K = w.M, w.N, w.n
         dX = dev(X)
-        nbytes = sq.sq_linear_workspace_bytes(M, N, K)
+        nbytes = sq.sq_linear_workspace_bytes(M, K)
         assert nbytes <= sq.SQ_LINEAR_STATIC_SCRATCH_BYTES
         ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
         off = (-ws.data_ptr()) % 256
