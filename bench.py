@@ -5,6 +5,10 @@ One step = one pass of the whole path (sq_linear) over one batch of synthetic ac
 the named workload.  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
+                  [--structured-r2] [--no-sweep] [--no-cpu-baseline]
+
+After the headline workload the default run also times every other benchmark workload briefly and
+reports them under "per_workload" of the same line (skipped with --no-sweep or N > 1).
 
 N > 1: launched under torchrun, one process per GPU; the path shards over tokens with no
 collective (each rank owns its own batch and a replica of the packed weights), so scaling is
@@ -87,7 +91,9 @@ def gemm_kernel_name(w):
     return "w4a4_gemm_tc_kernel" if fast else "w4a4_gemm_simple_kernel"
 
 
-def rotate_kernel_name(w):
+def rotate_kernel_name(w, structured=False):
+    if structured:
+        return "rotate_quant_st_kernel"
     if w.n2 in (64, 128) and w.n1 <= 128:
         return "rotate_quant_tc_kernel"
     if w.n2 in (64, 128) and w.n1 <= 256:
@@ -103,11 +109,21 @@ class ClockSampler:
              "clocks_event_reasons.hw_slowdown,clocks_event_reasons.hw_thermal_slowdown,"
              "clocks_event_reasons.sw_thermal_slowdown,clocks_event_reasons.sw_power_cap")
 
-    def __init__(self, gpu_index: int):
-        self.gpu = gpu_index
+    def __init__(self, gpu_id: str):
+        self.gpu = gpu_id          # a UUID ("GPU-...") when it could be resolved, else an nvidia-smi index
         self.proc = None
         self.lines = []
         self.thread = None
+
+    @staticmethod
+    def resolve(torch, device_index: int) -> str:
+        """The nvidia-smi id of the torch device: its UUID (CUDA_VISIBLE_DEVICES may renumber the
+        devices, so the torch index is not nvidia-smi's)."""
+        try:
+            uuid = str(torch.cuda.get_device_properties(device_index).uuid)
+            return uuid if uuid.startswith("GPU-") else "GPU-" + uuid
+        except Exception:
+            return str(device_index)
 
     def start(self):
         try:
@@ -124,16 +140,20 @@ class ClockSampler:
         for line in self.proc.stdout:
             self.lines.append((time.perf_counter(), line.strip()))
 
-    def stop(self, t_begin=None, t_end=None):
-        """Median SM clock and throttle reasons over the samples that arrived inside [t_begin, t_end]
-        (the timed region); if fewer than three did, over every sample of the run, and says so."""
+    def stop(self):
         if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+            return
         self.proc.terminate()
         try:
             self.proc.wait(timeout=5)
         except Exception:
             self.proc.kill()
+
+    def window(self, t_begin=None, t_end=None):
+        """Median SM clock and throttle reasons over the samples that arrived inside [t_begin, t_end]
+        (a timed region); if fewer than three did, over every sample so far, and says so."""
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
         sm, smax, reasons = [], [], set()
         names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
         inside = [ln for (t, ln) in self.lines if t_begin is not None and t_begin <= t <= t_end]
@@ -228,117 +248,71 @@ def run_reference(args, w):
 # ----------------------------------------------------------------------------------------------
 # CUDA arm
 # ----------------------------------------------------------------------------------------------
-def run_ours(args, w):
-    import torch
-    from paper_2511_22316_b200 import binding as sq
-    from paper_2511_22316_b200 import build as sqbuild
+class Layer:
+    """One workload resident on the device: rotation handle, packed weights, and a ring of buffer sets
+    larger than L2 so that no step finds its inputs cached."""
 
-    rank = int(os.environ.get("RANK", "0"))
-    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
-    world = int(os.environ.get("WORLD_SIZE", "1"))
-    if not torch.cuda.is_available():
-        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
-    torch.cuda.set_device(local_rank)
-    if rank == 0 or world == 1:
-        sqbuild.build()
-    dist = None
-    if world > 1:
-        import torch.distributed as dist_mod
-        dist = dist_mod
-        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
-        dist.barrier()
-    sq.load()
-
-    M, N, K = w.M, w.N, w.K
-    # every rank draws its own batch (weak scaling over tokens); the weights are replicated
-    import dataclasses
-    w_rank = dataclasses.replace(w, seed=w.seed + 7919 * rank) if rank else w
-    X = wl.make_activations(w_rank)
-    W = wl.make_weights(w)
-    rot = sq.sq_build_rotation(X.astype(np.float32), w.n1, w.n2, seed=0)
-
-    dW = torch.from_numpy(W).cuda()
-    Wq = torch.empty((N, K // 2), dtype=torch.uint8, device="cuda")
-    sw = torch.empty((N,), dtype=torch.float16, device="cuda")
-    sq.sq_pack_weight(rot, dW, N, K, Wq, sw)
-    torch.cuda.synchronize()
-    del dW
-
-    # ring of buffer sets larger than L2 so that no step finds its inputs cached
-    l2 = torch.cuda.get_device_properties(local_rank).L2_cache_size
-    per_set = M * K * 2 + M * K // 2 + M * N * 2 + N * K // 2
-    nsets = max(2, int(np.ceil(1.5 * l2 / per_set)) + 1)
-    ws_bytes = sq.sq_linear_workspace_bytes(M, K)
-    Xh = torch.from_numpy(X).pin_memory()
-    sets = []
-    for i in range(nsets):
-        ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
-        off = (-ws.data_ptr()) % 256
-        sets.append({
-            "X": Xh.cuda(non_blocking=False).clone(),
-            "Wq": Wq.clone(), "sw": sw.clone(),
-            "Y": torch.empty((M, N), dtype=torch.float16, device="cuda"),
-            "ws": ws, "ws_ptr": ws.data_ptr() + off,
-            "Xq": torch.empty((M, K // 2), dtype=torch.uint8, device="cuda"),
-            "sx": torch.empty((M,), dtype=torch.float16, device="cuda"),
-        })
-
-    # device pointers resolved once: the timed loop passes plain integers through the C ABI
-    for s_ in sets:
-        s_["ptrs"] = (s_["X"].data_ptr(), s_["Wq"].data_ptr(), s_["sw"].data_ptr(), s_["ws_ptr"], s_["Y"].data_ptr())
-
-    def step(i):
-        x_, wq_, sw_, ws_, y_ = sets[i % nsets]["ptrs"]
-        sq.sq_linear(rot, x_, M, wq_, sw_, N, K, ws_, ws_bytes, y_)
-
-    def sync_all():
+    def __init__(self, sq, torch, w, device_index, rank=0, structured_r2=False, keep_host=False):
+        import dataclasses
+        self.sq, self.torch, self.w = sq, torch, w
+        M, N, K = w.M, w.N, w.K
+        w_rank = dataclasses.replace(w, seed=w.seed + 7919 * rank) if rank else w
+        X = wl.make_activations(w_rank)
+        W = wl.make_weights(w)
+        flags = sq.SQ_ROT_DEFAULT | (sq.SQ_ROT_APPLY_STRUCTURED if structured_r2 else 0)
+        self.rot = sq.sq_build_rotation(X.astype(np.float32), w.n1, w.n2, flags=flags, seed=0)
+        dW = torch.from_numpy(W).cuda()
+        Wq = torch.empty((N, K // 2), dtype=torch.uint8, device="cuda")
+        sw = torch.empty((N,), dtype=torch.float16, device="cuda")
+        sq.sq_pack_weight(self.rot, dW, N, K, Wq, sw)
         torch.cuda.synchronize()
-        if dist is not None:
-            dist.barrier()
-            torch.cuda.synchronize()
+        del dW
+        self.l2 = torch.cuda.get_device_properties(device_index).L2_cache_size
+        self.per_set = M * K * 2 + M * K // 2 + M * N * 2 + N * K // 2
+        self.nsets = max(2, int(np.ceil(1.5 * self.l2 / self.per_set)) + 1)
+        self.ws_bytes = sq.sq_linear_workspace_bytes(M, K)
+        self.Xh = torch.from_numpy(X).pin_memory()
+        self.sets = []
+        for _ in range(self.nsets):
+            ws = torch.empty(self.ws_bytes + 256, dtype=torch.uint8, device="cuda")
+            off = (-ws.data_ptr()) % 256
+            st = {"X": self.Xh.cuda(non_blocking=False).clone(), "Wq": Wq.clone(), "sw": sw.clone(),
+                  "Y": torch.empty((M, N), dtype=torch.float16, device="cuda"), "ws": ws, "ws_ptr": ws.data_ptr() + off,
+                  "Xq": torch.empty((M, K // 2), dtype=torch.uint8, device="cuda"),
+                  "sx": torch.empty((M,), dtype=torch.float16, device="cuda")}
+            # device pointers resolved once: the timed loop passes plain integers through the C ABI
+            st["ptrs"] = (st["X"].data_ptr(), st["Wq"].data_ptr(), st["sw"].data_ptr(), st["ws_ptr"], st["Y"].data_ptr())
+            self.sets.append(st)
+        self.X, self.W = (X, W) if keep_host else (None, None)
 
-    for i in range(max(args.warmup, 3)):
-        step(i)
-    sync_all()
+    def step(self, i):
+        w = self.w
+        x_, wq_, sw_, ws_, y_ = self.sets[i % self.nsets]["ptrs"]
+        self.sq.sq_linear(self.rot, x_, w.M, wq_, sw_, w.N, w.K, ws_, self.ws_bytes, y_)
 
-    sampler = ClockSampler(local_rank)
-    if rank == 0:
-        sampler.start()
-        time.sleep(0.3)
+    def rotate_quant(self, i):
+        s, w = self.sets[i % self.nsets], self.w
+        self.sq.sq_rotate_quant_act(self.rot, s["X"], w.M, s["Xq"], s["sx"])
 
-    # ---- timed region: exactly K steps of sq_linear ------------------------------------------
-    launches0 = sq.sq_kernel_launch_count()
-    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-    sync_all()
-    t_region0 = time.perf_counter()
-    e0.record()
-    for i in range(args.steps):
-        step(i)
-    e1.record()
-    sync_all()
-    t_region1 = time.perf_counter()
-    ms_total = e0.elapsed_time(e1)
-    launches = sq.sq_kernel_launch_count() - launches0
+    def gemm(self, i):
+        s, w = self.sets[i % self.nsets], self.w
+        self.sq.sq_w4a4_gemm(s["Xq"], s["sx"], s["Wq"], s["sw"], w.M, w.N, w.K, s["Y"], None)
 
-    # ---- attribution: the same two kernels, launched through their own entry points, each
-    # bracketed by events on the launching stream (same ring, same stream, right after) -------
-    attr_steps = min(args.steps, 200)
-    ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(attr_steps)]
-    for i in range(attr_steps):
-        s = sets[i % nsets]
-        ev[i][0].record()
-        sq.sq_rotate_quant_act(rot, s["X"], M, s["Xq"], s["sx"])
-        ev[i][1].record()
-        sq.sq_w4a4_gemm(s["Xq"], s["sx"], s["Wq"], s["sw"], M, N, K, s["Y"], None)
-        ev[i][2].record()
-    torch.cuda.synchronize()
-    rq_ms = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
-    gemm_ms = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+    def timed_steps(self, steps):
+        """CUDA events on the launching stream around `steps` calls of sq_linear, launched one by one."""
+        torch = self.torch
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(steps):
+            self.step(i)
+        e1.record()
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1)
 
-    # ---- the same calls replayed from CUDA graphs: launch overhead taken out.  Short kernels
-    # (decode shapes) are launch-bound when issued one by one, so the per-kernel figures below
-    # come from graphs of back-to-back launches when capture works, else from the events above.
-    def graph_time(fn, count):
+    def graph_time(self, fn, count):
+        """Milliseconds per call of `fn` replayed from a CUDA graph of `count` back-to-back calls (launch
+        overhead taken out); None when capture is not possible."""
+        torch = self.torch
         try:
             gstream = torch.cuda.Stream()
             gstream.wait_stream(torch.cuda.current_stream())
@@ -364,16 +338,197 @@ def run_ours(args, w):
             torch.cuda.synchronize()
             return None
 
-    gsteps = min(args.steps, 4 * nsets)
-    graph_ms = graph_time(step, gsteps)
-    rq_graph = graph_time(lambda i: sq.sq_rotate_quant_act(rot, sets[i % nsets]["X"], M, sets[i % nsets]["Xq"],
-                                                           sets[i % nsets]["sx"]), gsteps)
-    gemm_graph = graph_time(lambda i: sq.sq_w4a4_gemm(sets[i % nsets]["Xq"], sets[i % nsets]["sx"], sets[i % nsets]["Wq"],
-                                                      sets[i % nsets]["sw"], M, N, K, sets[i % nsets]["Y"], None), gsteps)
-    kernel_timing = "cuda events around single launches"
-    if rq_graph is not None and gemm_graph is not None:
-        rq_ms, gemm_ms = rq_graph, gemm_graph
-        kernel_timing = "cuda events around graph replays of back-to-back launches"
+    def kernel_times(self, count):
+        """(rotate+quant ms, GEMM ms, whole step from a graph ms, how): per-entry-point times from graph
+        replays of back-to-back launches on the ring, else from events around single launches."""
+        torch = self.torch
+        graph_ms = self.graph_time(self.step, count)
+        rq = self.graph_time(self.rotate_quant, count)
+        ge = self.graph_time(self.gemm, count)
+        how = "cuda events around graph replays of back-to-back launches"
+        if rq is None or ge is None:
+            ev = [[torch.cuda.Event(enable_timing=True) for _ in range(3)] for _ in range(count)]
+            for i in range(count):
+                ev[i][0].record()
+                self.rotate_quant(i)
+                ev[i][1].record()
+                self.gemm(i)
+                ev[i][2].record()
+            torch.cuda.synchronize()
+            rq = statistics.mean(e[0].elapsed_time(e[1]) for e in ev)
+            ge = statistics.mean(e[1].elapsed_time(e[2]) for e in ev)
+            how = "cuda events around single launches"
+        return rq, ge, graph_ms, how
+
+    def close(self):
+        self.rot.close()
+        self.sets = []
+        self.torch.cuda.empty_cache()
+
+
+def int8_yardstick(torch, w, l2_bytes):
+    """A library int8 GEMM (torch._int_mm: int8 x int8 -> int32) of the workload's shape, timed in the same
+    run on buffers rotated through more than L2: what "the dense INT8 tensor peak" amounts to on this machine
+    at this size.  None where the library does not take the shape."""
+    try:
+        M, N, K = w.M, w.N, w.K
+        if M <= 16 or K % 8 or N % 8:
+            return None
+        per = M * K + K * N + 4 * M * N
+        nsets = max(2, int(np.ceil(1.5 * l2_bytes / per)) + 1)
+        A = [torch.randint(-8, 8, (M, K), dtype=torch.int8, device="cuda") for _ in range(nsets)]
+        B = [torch.randint(-8, 8, (K, N), dtype=torch.int8, device="cuda") for _ in range(nsets)]
+        for i in range(3):
+            torch._int_mm(A[i % nsets], B[i % nsets])
+        torch.cuda.synchronize()
+        iters = 20
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for i in range(iters):
+            torch._int_mm(A[i % nsets], B[i % nsets])
+        e1.record()
+        torch.cuda.synchronize()
+        ms = e0.elapsed_time(e1) / iters
+        return {"name": "torch._int_mm (int8 x int8 -> int32, library GEMM)", "ms": ms,
+                "tops": 2.0 * M * N * K / (ms * 1e-3) / 1e12}
+    except Exception as exc:
+        sys.stderr.write(f"int8 yardstick skipped: {exc}\n")
+        return None
+
+
+def link_yardstick(torch, in_bytes, out_bytes, iters=10):
+    """Milliseconds for one pinned host->device copy of `in_bytes` and one device->host copy of `out_bytes`
+    running concurrently on two streams, no computation: the floor of an end-to-end step on this link."""
+    try:
+        hin = torch.empty(in_bytes, dtype=torch.uint8).pin_memory()
+        hout = torch.empty(out_bytes, dtype=torch.uint8).pin_memory()
+        din = torch.empty(in_bytes, dtype=torch.uint8, device="cuda")
+        dout = torch.empty(out_bytes, dtype=torch.uint8, device="cuda")
+        s1, s2 = torch.cuda.Stream(), torch.cuda.Stream()
+        torch.cuda.synchronize()
+        best = None
+        for rep in range(2):
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            s1.wait_event(e0)
+            s2.wait_event(e0)
+            for _ in range(iters):
+                with torch.cuda.stream(s1):
+                    din.copy_(hin, non_blocking=True)
+                with torch.cuda.stream(s2):
+                    hout.copy_(dout, non_blocking=True)
+            torch.cuda.current_stream().wait_stream(s1)
+            torch.cuda.current_stream().wait_stream(s2)
+            e1.record()
+            torch.cuda.synchronize()
+            ms = e0.elapsed_time(e1) / iters
+            best = ms if best is None else min(best, ms)
+        return best
+    except Exception as exc:
+        sys.stderr.write(f"link yardstick skipped: {exc}\n")
+        return None
+
+
+def rooflines(w, rq_ms, gemm_ms, pk, structured, yard=None):
+    """The two kernels' roofline entries: (GEMM, rotate+quant)."""
+    gemm_tops = ops_per_step(w) / (gemm_ms * 1e-3) / 1e12
+    rq_gbs = rotate_quant_bytes(w) / (rq_ms * 1e-3) / 1e9
+    int8_peak = pk["bf16_tflops"] * INT8_OVER_BF16
+    if w.M <= 64:       # decode: bound by reading the packed weights once
+        gemm_gbs = gemm_bytes(w) / (gemm_ms * 1e-3) / 1e9
+        roof_gemm = {"kernel": gemm_kernel_name(w), "bound": "hbm", "achieved": gemm_gbs, "peak": pk["hbm_gbs"],
+                     "unit": "GB/s", "frac": gemm_gbs / pk["hbm_gbs"],
+                     "traffic": NCU_TRAFFIC.get(("gemm", w.name)),
+                     "peak_source": f"{pk['source']} copy bandwidth", "ms_per_launch": gemm_ms,
+                     "algorithmic_bytes": gemm_bytes(w), "frac_of_spec_8000": gemm_gbs / 8000.0}
+    else:
+        roof_gemm = {"kernel": gemm_kernel_name(w), "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak,
+                     "unit": "TOP/s", "frac": gemm_tops / int8_peak,
+                     "traffic": NCU_TRAFFIC.get(("gemm", w.name)),
+                     "peak_source": f"{pk['source']} bf16 burst x{INT8_OVER_BF16:g} (nominal int8:bf16 ratio)",
+                     "ms_per_launch": gemm_ms, "algorithmic_ops": ops_per_step(w),
+                     "frac_of_spec_4500": gemm_tops / 4500.0}
+        if yard is not None:
+            roof_gemm["yardstick"] = dict(yard, frac=gemm_tops / yard["tops"])
+    roof_rq = {"kernel": rotate_kernel_name(w, structured), "bound": "hbm", "achieved": rq_gbs, "peak": pk["hbm_gbs"],
+               "unit": "GB/s", "frac": rq_gbs / pk["hbm_gbs"],
+               "traffic": NCU_TRAFFIC.get(("rotate_quant", w.name)) if not structured else None,
+               "peak_source": f"{pk['source']} copy bandwidth", "ms_per_launch": rq_ms,
+               "algorithmic_bytes": rotate_quant_bytes(w), "frac_of_spec_8000": rq_gbs / 8000.0}
+    return roof_gemm, roof_rq
+
+
+def run_ours(args, w):
+    import torch
+    from paper_2511_22316_b200 import binding as sq
+    from paper_2511_22316_b200 import build as sqbuild
+
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(local_rank)
+    if rank == 0 or world == 1:
+        sqbuild.build()
+    dist = None
+    if world > 1:
+        import torch.distributed as dist_mod
+        dist = dist_mod
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+        dist.barrier()
+    sq.load()
+
+    M, N, K = w.M, w.N, w.K
+    # every rank draws its own batch (weak scaling over tokens); the weights are replicated
+    layer = Layer(sq, torch, w, local_rank, rank=rank, structured_r2=args.structured_r2, keep_host=True)
+    nsets, per_set, l2 = layer.nsets, layer.per_set, layer.l2
+    structured = layer.rot.structured
+
+    def sync_all():
+        torch.cuda.synchronize()
+        if dist is not None:
+            dist.barrier()
+            torch.cuda.synchronize()
+
+    warm = max(args.warmup, 3)
+    for i in range(warm):
+        layer.step(i)
+    sync_all()
+
+    sampler = ClockSampler(ClockSampler.resolve(torch, local_rank))
+    if rank == 0:
+        sampler.start()
+        time.sleep(0.3)
+
+    # ---- timed region: exactly K steps of sq_linear ------------------------------------------
+    launches0 = sq.sq_kernel_launch_count()
+    sync_all()
+    t_region0 = time.perf_counter()
+    ms_total = layer.timed_steps(args.steps)
+    sync_all()
+    t_region1 = time.perf_counter()
+    launches = sq.sq_kernel_launch_count() - launches0
+    clocks = sampler.window(t_region0, t_region1) if rank == 0 else None
+
+    # ---- the same step for at least half a second, so that several clock samples fall inside it:
+    # the step time and the clocks it ran at (time x median SM MHz lets a reader normalise) -----------
+    sustained = None
+    if rank == 0 and world == 1:
+        n_sus = max(args.steps, int(np.ceil(600.0 / max(ms_total / args.steps, 1e-3))))
+        n_sus = min(n_sus, 400000)
+        t0 = time.perf_counter()
+        ms_sus = layer.timed_steps(n_sus)
+        t1 = time.perf_counter()
+        sustained = {"steps": n_sus, "ms_per_step": ms_sus / n_sus,
+                     "value": ops_per_step(w) / (ms_sus / n_sus * 1e-3) / 1e12, "unit": UNIT,
+                     "clocks": sampler.window(t0, t1)}
+        if sustained["clocks"].get("sm_mhz"):
+            sustained["us_x_mhz"] = ms_sus / n_sus * 1e3 * sustained["clocks"]["sm_mhz"]
+
+    # ---- attribution: the two entry points and the whole step replayed from CUDA graphs -------
+    gsteps = min(max(args.steps, 8), 4 * nsets)
+    rq_ms, gemm_ms, graph_ms, kernel_timing = layer.kernel_times(gsteps)
 
     # ---- end to end: host activations in, host outputs out, through sq_linear_host ------------
     hws_bytes = sq.sq_linear_host_workspace_bytes(M, N, K)
@@ -381,20 +536,21 @@ def run_ours(args, w):
     hoff = (-hws.data_ptr()) % 256
     Yh = torch.empty((M, N), dtype=torch.float16).pin_memory()
     e2e_steps = max(3, min(args.steps, 20))
+    sets = layer.sets
     for _ in range(2):
-        sq.sq_linear_host(rot, Xh, M, sets[0]["Wq"], sets[0]["sw"], N, K, hws.data_ptr() + hoff, hws_bytes, Yh)
+        sq.sq_linear_host(layer.rot, layer.Xh, M, sets[0]["Wq"], sets[0]["sw"], N, K, hws.data_ptr() + hoff, hws_bytes, Yh)
     sync_all()
     h0, h1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
     h0.record()
     for i in range(e2e_steps):
         s = sets[i % nsets]
-        sq.sq_linear_host(rot, Xh, M, s["Wq"], s["sw"], N, K, hws.data_ptr() + hoff, hws_bytes, Yh)
+        sq.sq_linear_host(layer.rot, layer.Xh, M, s["Wq"], s["sw"], N, K, hws.data_ptr() + hoff, hws_bytes, Yh)
     h1.record()
     sync_all()
     e2e_ms = h0.elapsed_time(h1) / e2e_steps
     status = sq.sq_last_device_status()
-
-    clocks = sampler.stop(t_region0, t_region1) if rank == 0 else None
+    link_ms = link_yardstick(torch, M * K * 2, M * N * 2) if (rank == 0 and world == 1) else None
+    del hws
 
     # ---- max over ranks ---------------------------------------------------------------------
     t = torch.tensor([ms_total, e2e_ms, rq_ms, gemm_ms, graph_ms if graph_ms is not None else -1.0],
@@ -409,33 +565,13 @@ def run_ours(args, w):
         pk = peaks()
         value = world * ops_per_step(w) / (ms_per_step * 1e-3) / 1e12
         e2e_value = world * ops_per_step(w) / (e2e_ms * 1e-3) / 1e12
-        gemm_tops = ops_per_step(w) / (gemm_ms * 1e-3) / 1e12
-        rq_gbs = rotate_quant_bytes(w) / (rq_ms * 1e-3) / 1e9
-        int8_peak = pk["bf16_tflops"] * INT8_OVER_BF16
-        if w.M <= 64:       # decode: bound by reading the packed weights once
-            gemm_gbs = gemm_bytes(w) / (gemm_ms * 1e-3) / 1e9
-            roof_gemm = {"kernel": gemm_kernel_name(w), "bound": "hbm", "achieved": gemm_gbs, "peak": pk["hbm_gbs"],
-                         "unit": "GB/s", "frac": gemm_gbs / pk["hbm_gbs"],
-                         "traffic": NCU_TRAFFIC.get(("gemm", w.name)),
-                         "peak_source": f"{pk['source']} copy bandwidth", "ms_per_launch": gemm_ms,
-                         "algorithmic_bytes": gemm_bytes(w), "frac_of_spec_8000": gemm_gbs / 8000.0}
-        else:
-            roof_gemm = {"kernel": gemm_kernel_name(w), "bound": "tensor", "achieved": gemm_tops, "peak": int8_peak,
-                         "unit": "TOP/s", "frac": gemm_tops / int8_peak,
-                         "traffic": NCU_TRAFFIC.get(("gemm", w.name)),
-                         "peak_source": f"{pk['source']} bf16 burst x{INT8_OVER_BF16:g} (nominal int8:bf16 ratio)",
-                         "ms_per_launch": gemm_ms, "algorithmic_ops": ops_per_step(w),
-                         "frac_of_spec_4500": gemm_tops / 4500.0}
-        roof_rq = {"kernel": rotate_kernel_name(w), "bound": "hbm", "achieved": rq_gbs, "peak": pk["hbm_gbs"],
-                   "unit": "GB/s", "frac": rq_gbs / pk["hbm_gbs"],
-                   "traffic": NCU_TRAFFIC.get(("rotate_quant", w.name)),
-                   "peak_source": f"{pk['source']} copy bandwidth", "ms_per_launch": rq_ms,
-                   "algorithmic_bytes": rotate_quant_bytes(w), "frac_of_spec_8000": rq_gbs / 8000.0}
+        yard = int8_yardstick(torch, w, l2) if world == 1 else None
+        roof_gemm, roof_rq = rooflines(w, rq_ms, gemm_ms, pk, structured, yard)
         dominant, other = (roof_gemm, roof_rq) if gemm_ms >= rq_ms else (roof_rq, roof_gemm)
 
         cpu = None
         if world == 1 and not args.no_cpu_baseline:
-            arm = OracleArm(w, rows=256, X=X, W=W)
+            arm = OracleArm(w, rows=256, X=layer.X, W=layer.W)
             arm.one_pass()
             times, t_start = [], time.perf_counter()
             while time.perf_counter() - t_start < 10.0 or not times:
@@ -443,12 +579,56 @@ def run_ours(args, w):
             cpu = {"value": arm.tops(statistics.mean(times)), "unit": UNIT, "cores": arm.threads(),
                    "kind": "oracle", "sample": f"{arm.sample}; {len(times)} passes, "
                                                f"{statistics.mean(times):.3f} s per pass"}
+            del arm
+        layer.X = layer.W = None
+
+        # ---- every other benchmark workload, briefly: step (launched and from a graph), the two
+        # kernels, both roofline fractions and the clocks sampled while it ran ------------------
+        per_workload = None
+        if world == 1 and not args.no_sweep:
+            per_workload = {w.name: {"M": M, "N": N, "K": K, "n1": w.n1, "n2": w.n2, "steps": args.steps,
+                                     "ms_per_step": ms_per_step, "step_graph_replay_ms": graph_ms,
+                                     "value": value, "unit": UNIT, "rotate_quant": roof_rq, "gemm": roof_gemm,
+                                     "clocks": clocks}}
+            layer.close()
+            for ow in wl.ALL_WORKLOADS:
+                if ow.name == w.name:
+                    continue
+                try:
+                    ol = Layer(sq, torch, ow, local_rank, structured_r2=args.structured_r2)
+                    for i in range(5):
+                        ol.step(i)
+                    torch.cuda.synchronize()
+                    ostep = 100
+                    t0 = time.perf_counter()
+                    oms = ol.timed_steps(ostep) / ostep
+                    # keep the clocks' window at least 0.35 s long
+                    extra = int(np.ceil(max(0.0, 0.35 - (time.perf_counter() - t0)) / max(oms * 1e-3, 1e-6)))
+                    if extra > 0:
+                        ol.timed_steps(min(extra, 200000))
+                    t1 = time.perf_counter()
+                    orq, oge, ogr, _ = ol.kernel_times(min(ostep, 4 * ol.nsets))
+                    og, orr = rooflines(ow, orq, oge, pk, ol.rot.structured,
+                                        int8_yardstick(torch, ow, l2))
+                    per_workload[ow.name] = {
+                        "M": ow.M, "N": ow.N, "K": ow.K, "n1": ow.n1, "n2": ow.n2, "steps": ostep,
+                        "ms_per_step": oms, "step_graph_replay_ms": ogr,
+                        "value": ops_per_step(ow) / (oms * 1e-3) / 1e12, "unit": UNIT,
+                        "rotate_quant": orr, "gemm": og, "clocks": sampler.window(t0, t1),
+                        "device_status": sq.sq_last_device_status()}
+                    ol.close()
+                    del ol
+                except Exception as exc:
+                    per_workload[ow.name] = {"error": str(exc)}
+        sampler.stop()
+
         line = {
             "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": args.steps,
-            "warmup": max(args.warmup, 3), "ms_per_step": ms_per_step, "higher_is_better": True,
+            "warmup": warm, "ms_per_step": ms_per_step, "higher_is_better": True,
             "scaling": "weak", "vs_baseline": None, "dtype": "int8",
             "data": "synthetic",
             "config": {"workload": w.name, "M_per_gpu": M, "N": N, "K": K, "n1": w.n1, "n2": w.n2,
+                       "r2_application": "structured (butterflies + rotation chains)" if structured else "dense",
                        "parallelism": f"token-sharded x{world}, no collective",
                        "l2": f"ring of {nsets} buffer sets ({nsets * per_set / 1e6:.0f} MB > L2 "
                              f"{l2 / 1e6:.0f} MB)"},
@@ -457,13 +637,19 @@ def run_ours(args, w):
             "kernel_ms": {"rotate_quant": rq_ms, "w4a4_gemm": gemm_ms, "sum": rq_ms + gemm_ms,
                           "step": ms_per_step, "step_graph_replay": graph_ms, "how": kernel_timing},
             "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": e2e_ms, "h2d_bytes_per_step": M * K * 2,
-                    "d2h_bytes_per_step": M * N * 2, "api": "sq_linear_host (pinned host X -> host Y)"},
+                    "d2h_bytes_per_step": M * N * 2, "api": "sq_linear_host (pinned host X -> host Y)",
+                    "link_yardstick_ms": link_ms,
+                    "frac_of_link": (link_ms / e2e_ms) if link_ms else None},
             "gpu_launches": int(launches),
             "clocks": clocks,
             "device_status": status,
         }
+        if sustained is not None:
+            line["sustained"] = sustained
         if cpu is not None:
             line["cpu_baseline"] = cpu
+        if per_workload is not None:
+            line["per_workload"] = per_workload
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()
@@ -482,6 +668,11 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true",
                     help="skip the timed CPU oracle leg (for profiler runs)")
+    ap.add_argument("--no-sweep", action="store_true",
+                    help="time the named workload only (skip the per_workload table)")
+    ap.add_argument("--structured-r2", action="store_true",
+                    help="build the rotation with SQ_ROT_APPLY_STRUCTURED: R2 = H R2^U applied piece by piece "
+                         "in registers instead of as a dense matrix on the tensor cores")
     args = ap.parse_args()
     if args.steps is None:
         args.steps = 20 if args.impl == "reference" else 20000

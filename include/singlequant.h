@@ -62,6 +62,14 @@ enum { SQ_ROT_ART = 1, SQ_ROT_URT = 2, SQ_ROT_HADAMARD = 4, SQ_ROT_DEFAULT = 7 }
  * in the plane (outlier, minimum) of the column as rotated so far.  The paper finds one step
  * sufficient; the default is one. */
 #define SQ_ROT_ART_STEPS(k) ((uint32_t)((k) - 1) << 8)
+/* A handle made by sq_build_rotation knows how R2 = H R2^U was composed.  With this bit in `flags`
+ * (and n2 = 64 or 128, n1 <= 128) the kernel of steps 1+2 applies R2 piece by piece in fp32 registers
+ * -- Hadamard butterflies, then the two chains of plane rotations of URT in closed form -- instead of
+ * as a dense matrix on the tensor cores: the same operator with about a tenth of the multiply-adds.
+ * Without the bit (the default, and always for handles made by sq_rotation_from_factors) R2 is applied
+ * as the dense matrix, which measures as fast or faster on a B200 at every benchmark shape (the
+ * structured form trades idle tensor cores for busy arithmetic pipes). */
+#define SQ_ROT_APPLY_STRUCTURED (1u << 20)
 
 /* Algorithm 1 (Kronecker Dimension Factorization).  Host only.  n2 = the power of two dividing
  * n closest to sqrt(n), the first found winning ties; n1 = n / n2.  n >= 1. */
@@ -93,6 +101,9 @@ sq_status_t sq_rotation_from_factors(const float* R1, const float* R2, int32_t n
 /* Copies the fp32 factors back to HOST buffers of n1*n1 and n2*n2 floats. */
 sq_status_t sq_rotation_get_factors(const sq_rotation_t* rot, float* R1, float* R2);
 sq_status_t sq_rotation_dims(const sq_rotation_t* rot, int32_t* n1, int32_t* n2);
+/* 1 when steps 1+2 with this handle apply R2 through its composition (see SQ_ROT_APPLY_STRUCTURED), 0 when
+ * they apply it as a dense matrix (also for a NULL handle). */
+int32_t sq_rotation_is_structured(const sq_rotation_t* rot);
 void sq_rotation_destroy(sq_rotation_t* rot);
 
 /* Steps 1+2, fused: Z_t = R1^T X~_t R2 in fp32 on chip, Delta_t = fp16(max|Z_t|/7),

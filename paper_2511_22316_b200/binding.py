@@ -21,10 +21,11 @@ SQ_OK = 0
 SQ_ERR_INVALID_ARG, SQ_ERR_SHAPE, SQ_ERR_ALIGN, SQ_ERR_UNSUPPORTED = 1, 2, 3, 4
 SQ_ERR_NOMEM, SQ_ERR_CUDA, SQ_ERR_TIMEOUT = 5, 6, 7
 SQ_ROT_ART, SQ_ROT_URT, SQ_ROT_HADAMARD, SQ_ROT_DEFAULT = 1, 2, 4, 7
+SQ_ROT_APPLY_STRUCTURED = 1 << 20
 
 EXPORTS = (
     "sq_factorize", "sq_build_rotation", "sq_rotation_from_factors", "sq_rotation_get_factors",
-    "sq_rotation_dims", "sq_rotation_destroy", "sq_rotate_quant_act", "sq_pack_weight",
+    "sq_rotation_dims", "sq_rotation_is_structured", "sq_rotation_destroy", "sq_rotate_quant_act", "sq_pack_weight",
     "sq_w4a4_gemm", "sq_linear_workspace_bytes", "sq_linear",
     "sq_linear_static", "sq_linear_host_workspace_bytes", "sq_linear_host", "sq_last_device_status",
     "sq_debug_bounded_wait", "sq_kernel_launch_count", "sq_status_string",
@@ -55,6 +56,8 @@ def load() -> ctypes.CDLL:
     lib.sq_rotation_from_factors.argtypes = [c_void_p, c_void_p, c_int32, c_int32, POINTER(c_void_p)]
     lib.sq_rotation_get_factors.argtypes = [c_void_p, c_void_p, c_void_p]
     lib.sq_rotation_dims.argtypes = [c_void_p, POINTER(c_int32), POINTER(c_int32)]
+    lib.sq_rotation_is_structured.argtypes = [c_void_p]
+    lib.sq_rotation_is_structured.restype = c_int32
     lib.sq_rotation_destroy.argtypes = [c_void_p]
     lib.sq_rotation_destroy.restype = None
     lib.sq_rotate_quant_act.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_void_p, c_void_p]
@@ -137,6 +140,10 @@ class Rotation:
     def factors(self) -> Tuple[np.ndarray, np.ndarray]:
         return sq_rotation_get_factors(self)
 
+    @property
+    def structured(self) -> bool:
+        return sq_rotation_is_structured(self)
+
     def close(self) -> None:
         if self._h:
             load().sq_rotation_destroy(self._h)
@@ -187,6 +194,10 @@ def sq_rotation_get_factors(rot: Rotation) -> Tuple[np.ndarray, np.ndarray]:
     R2 = np.empty((n2, n2), np.float32)
     _check(load().sq_rotation_get_factors(rot.handle, R1.ctypes.data, R2.ctypes.data), "sq_rotation_get_factors")
     return R1, R2
+
+
+def sq_rotation_is_structured(rot: Rotation) -> bool:
+    return bool(load().sq_rotation_is_structured(rot.handle))
 
 
 def sq_rotate_quant_act(rot: Rotation, X, M: int, Xq, sx, Zdbg=None, stream=None) -> None:

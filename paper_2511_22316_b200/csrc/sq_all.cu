@@ -6,6 +6,7 @@
 #include "sq_gemv.cu"
 #include "sq_rotate_quant.cu"
 #include "sq_rotate_quant_tc.cu"
+#include "sq_rotate_quant_st.cu"
 #include "sq_rotate_quant_pair.cu"
 #include "sq_rotation_host.cu"
 #include "sq_api.cu"

@@ -76,6 +76,7 @@ __global__ void bounded_wait_probe_kernel(uint32_t polls) {
 namespace sq {
 sq_status_t rotate_quant_dispatch(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
                                   float* Zdbg, cudaStream_t s) {
+  if (h->st_ready) return launch_rotate_quant_st(h, X, rows, Xq, scales, Zdbg, s);
   if (h->tc_ready) return launch_rotate_quant_tc(h, X, rows, Xq, scales, Zdbg, s);
   if (h->tc_pair) return launch_rotate_quant_pair(h, X, rows, Xq, scales, Zdbg, s);
   return launch_rotate_quant(h->dR1, h->dR2, h->n1, h->n2, X, rows, Xq, scales, Zdbg, s);
@@ -91,11 +92,12 @@ constexpr int64_t kMaxRows = (1ll << 31) - 1;
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 sq_status_t make_handle(std::vector<float>&& R1, std::vector<float>&& R2, int32_t n1, int32_t n2,
-                        sq_rotation_t** out) {
+                        const R2Structure* s2, sq_rotation_t** out) {
   sq_rotation* h = new (std::nothrow) sq_rotation();
   if (!h) return SQ_ERR_NOMEM;
   h->n1 = n1;
   h->n2 = n2;
+  if (s2) h->s2 = *s2;
   h->R1 = std::move(R1);
   h->R2 = std::move(R2);
   if (cudaGetDevice(&h->device) != cudaSuccess) {
@@ -112,9 +114,10 @@ sq_status_t make_handle(std::vector<float>&& R1, std::vector<float>&& R2, int32_
     delete h;
     return SQ_ERR_CUDA;
   }
-  const bool prepared = sq::rotate_quant_tc_supported(n1, n2)     ? sq::rotate_quant_tc_prepare(h)
-                        : sq::rotate_quant_pair_supported(n1, n2) ? sq::rotate_quant_pair_prepare(h)
-                                                                  : true;
+  const bool prepared = (sq::rotate_quant_tc_supported(n1, n2)     ? sq::rotate_quant_tc_prepare(h)
+                         : sq::rotate_quant_pair_supported(n1, n2) ? sq::rotate_quant_pair_prepare(h)
+                                                                   : true) &&
+                        sq::rotate_quant_st_prepare(h);
   if (!prepared) {
     sq_rotation_destroy(h);
     return SQ_ERR_CUDA;
@@ -182,14 +185,16 @@ sq_status_t sq_build_rotation(const float* calib, int64_t T, int64_t n, int32_t 
                               uint64_t seed, const double* O_or_null, sq_rotation_t** out) {
   if (!out) return SQ_ERR_INVALID_ARG;
   *out = nullptr;
-  if (!calib || T < 1 || n1 < 1 || n2 < 1 || (flags & ~(7u | (0x7FFu << 8)))) return SQ_ERR_INVALID_ARG;
+  if (!calib || T < 1 || n1 < 1 || n2 < 1 || (flags & ~(7u | (0x7FFu << 8) | SQ_ROT_APPLY_STRUCTURED)))
+    return SQ_ERR_INVALID_ARG;
   if (static_cast<int64_t>(n1) * n2 != n) return SQ_ERR_SHAPE;
   if ((flags & SQ_ROT_HADAMARD) && (n2 & (n2 - 1)) != 0) return SQ_ERR_SHAPE;
   if (n1 > 4096 || n2 > 4096) return SQ_ERR_UNSUPPORTED;
   std::vector<float> R1, R2;
-  sq_status_t st = sq::build_factors_host(calib, T, n, n1, n2, flags, seed, O_or_null, R1, R2);
+  R2Structure s2;
+  sq_status_t st = sq::build_factors_host(calib, T, n, n1, n2, flags, seed, O_or_null, R1, R2, &s2);
   if (st != SQ_OK) return st;
-  return make_handle(std::move(R1), std::move(R2), n1, n2, out);
+  return make_handle(std::move(R1), std::move(R2), n1, n2, (flags & SQ_ROT_APPLY_STRUCTURED) ? &s2 : nullptr, out);
 }
 
 sq_status_t sq_rotation_from_factors(const float* R1, const float* R2, int32_t n1, int32_t n2,
@@ -199,7 +204,7 @@ sq_status_t sq_rotation_from_factors(const float* R1, const float* R2, int32_t n
   if (!R1 || !R2 || n1 < 1 || n2 < 1) return SQ_ERR_INVALID_ARG;
   if (n1 > 4096 || n2 > 4096) return SQ_ERR_UNSUPPORTED;
   std::vector<float> a(R1, R1 + static_cast<size_t>(n1) * n1), b(R2, R2 + static_cast<size_t>(n2) * n2);
-  return make_handle(std::move(a), std::move(b), n1, n2, out);
+  return make_handle(std::move(a), std::move(b), n1, n2, nullptr, out);
 }
 
 sq_status_t sq_rotation_get_factors(const sq_rotation_t* rot, float* R1, float* R2) {
@@ -215,6 +220,8 @@ sq_status_t sq_rotation_dims(const sq_rotation_t* rot, int32_t* n1, int32_t* n2)
   *n2 = rot->n2;
   return SQ_OK;
 }
+
+int32_t sq_rotation_is_structured(const sq_rotation_t* rot) { return (rot && rot->st_ready) ? 1 : 0; }
 
 void sq_rotation_destroy(sq_rotation_t* rot) {
   if (!rot) return;

@@ -9,6 +9,17 @@
 
 #include "../../include/singlequant.h"
 
+// How R2 = H R2^U was composed (paragraphs "Uniformity Rotation Transformation", "The Overall
+// SingleQuant Method"): R2^U = R_map R'_map^T, R_map the chain of plane rotations on adjacent
+// coordinates with v R_map = ||v|| e_1, R'_map the same for the target u.  Known for handles made
+// by sq_build_rotation, unknown for factors injected by the caller.
+struct R2Structure {
+  bool known = false;
+  bool hadamard = false;        // H is the Sylvester Hadamard matrix / sqrt(n2) (else the identity)
+  bool urt = false;             // R2^U is present (else the identity)
+  std::vector<double> v, u;     // URT's source vector and its target, length n2 (when urt)
+};
+
 struct sq_rotation {
   int32_t n1 = 0, n2 = 0;
   int device = -1;
@@ -21,6 +32,10 @@ struct sq_rotation {
   void* dB2img = nullptr;
   bool tc_ready = false;   // images for the single-CTA kernel (n1 <= 128)
   bool tc_pair = false;    // images for the CTA-pair kernel (128 < n1 <= 256)
+  // structured application of R2 (sq_rotate_quant_st.cu): composition and kernel coefficients
+  R2Structure s2;
+  bool st_ready = false;
+  std::vector<float> st_coef;   // the kernel's coefficient block (host copy, passed by value)
 };
 
 namespace sq {
@@ -78,7 +93,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // Host-side construction of the factors in float64 (sq_rotation_host.cu).
 sq_status_t build_factors_host(const float* calib, int64_t T, int64_t n, int32_t n1, int32_t n2,
                                uint32_t flags, uint64_t seed, const double* O,
-                               std::vector<float>& R1, std::vector<float>& R2);
+                               std::vector<float>& R1, std::vector<float>& R2, R2Structure* s2);
 
 // Steps 1+2 (sq_rotate_quant.cu).  R1/R2 device fp32 or both nullptr for the identity.
 sq_status_t launch_rotate_quant(const float* dR1, const float* dR2, int n1, int n2, const void* X,
@@ -94,6 +109,11 @@ bool rotate_quant_pair_supported(int n1, int n2);
 bool rotate_quant_pair_prepare(sq_rotation* h);
 sq_status_t launch_rotate_quant_pair(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
                                      float* Zdbg, cudaStream_t s);
+// Steps 1+2 with R2 applied through its structure (sq_rotate_quant_st.cu): R1^T on the tensor cores,
+// then the Hadamard butterflies and the two rotation chains of URT in registers.
+bool rotate_quant_st_prepare(sq_rotation* h);
+sq_status_t launch_rotate_quant_st(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
+                                   float* Zdbg, cudaStream_t s);
 // Picks the tensor-core kernel when the handle has its images, else the generic fp32 kernel.
 sq_status_t rotate_quant_dispatch(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
                                   float* Zdbg, cudaStream_t s);

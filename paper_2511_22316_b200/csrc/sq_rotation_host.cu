@@ -68,12 +68,14 @@ Mat chain_to_e1(std::vector<double> v) {
   return R;
 }
 
-// URT: R^U with v R^U = u, u the rank-preserving evenly spaced target of the same norm.
-Mat urt(const std::vector<double>& v) {
+// The target of URT: the evenly spaced template q_k = (2k - n - 1)/n, assigned by the rank order of v
+// and scaled to the norm of v.  Returns false for the degenerate inputs (n < 2, v = 0) whose URT
+// is the identity.
+bool uniform_target(const std::vector<double>& v, std::vector<double>& u) {
   const int n = static_cast<int>(v.size());
   bool any = false;
   for (double x : v) any = any || (x != 0.0);
-  if (n < 2 || !any) return identity(n);
+  if (n < 2 || !any) return false;
   std::vector<int> order(n);
   std::iota(order.begin(), order.end(), 0);
   // entries closer than 1e-9 max|v| count as equal and keep their index order
@@ -90,10 +92,19 @@ Mat urt(const std::vector<double>& v) {
     qnorm2 += q[k - 1] * q[k - 1];
   }
   const double scale = std::sqrt(vnorm2) / std::sqrt(qnorm2);
-  std::vector<double> u(n, 0.0);
+  u.assign(n, 0.0);
   for (int k = 0; k < n; ++k) u[order[k]] = scale * q[k];
+  return true;
+}
+
+// URT: R^U with v R^U = u, u the rank-preserving evenly spaced target of the same norm.
+Mat urt(const std::vector<double>& v, std::vector<double>* u_out = nullptr) {
+  const int n = static_cast<int>(v.size());
+  std::vector<double> u;
+  if (!uniform_target(v, u)) return identity(n);
   Mat Rv = chain_to_e1(v);
   Mat Ru = chain_to_e1(u);
+  if (u_out) *u_out = u;
   return matmul(Rv, transpose(Ru, n), n);
 }
 
@@ -219,7 +230,7 @@ namespace sq {
 
 sq_status_t build_factors_host(const float* calib, int64_t T, int64_t n, int32_t n1, int32_t n2,
                                uint32_t flags, uint64_t seed, const double* O,
-                               std::vector<float>& R1out, std::vector<float>& R2out) {
+                               std::vector<float>& R1out, std::vector<float>& R2out, R2Structure* s2) {
   // 1. the calibration token with the largest |entry|, and where that entry sits
   int64_t t_star = 0, pos = 0;
   float best = -1.0f;
@@ -287,8 +298,18 @@ sq_status_t build_factors_host(const float* calib, int64_t T, int64_t n, int32_t
   std::vector<double> v(n2, 0.0);
   for (int q = 0; q < n2; ++q)
     for (int k = 0; k < n2; ++k) v[q] += LA[static_cast<size_t>(row) * n2 + k] * H[static_cast<size_t>(k) * n2 + q];
-  Mat RU2 = (flags & SQ_ROT_URT) ? urt(v) : identity(n2);
+  std::vector<double> u;
+  Mat RU2 = (flags & SQ_ROT_URT) ? urt(v, &u) : identity(n2);
   Mat R2 = matmul(H, RU2, n2);
+  if (s2 != nullptr) {
+    // How R2 was put together, for kernels that apply its pieces one after the other instead of
+    // the dense product: x R2 = ((x H) R_map) R'_map^T with the two chains given by v and u.
+    s2->known = true;
+    s2->hadamard = (flags & SQ_ROT_HADAMARD) != 0 && n2 > 1;
+    s2->urt = !u.empty();
+    s2->v = s2->urt ? v : std::vector<double>();
+    s2->u = u;
+  }
 
   R1out.resize(R1.size());
   R2out.resize(R2.size());

@@ -47,9 +47,10 @@ def run_rotate_quant(sq, rot, X, want_z=True):
             z.numpy(np.float32, (M, n)) if z is not None else None)
 
 
-def check_rotate_quant(sq, X, R1, R2, rows=None):
-    """Compares the fused kernel with the oracle on the rows `rows` (default: all)."""
-    rot = sq.sq_rotation_from_factors(R1, R2)
+def check_rotate_quant(sq, X, R1, R2, rows=None, rot=None):
+    """Compares the fused kernel with the oracle on the rows `rows` (default: all).  `rot`: the handle
+    to run with (default: one made from the oracle's factors R1, R2)."""
+    rot = sq.sq_rotation_from_factors(R1, R2) if rot is None else rot
     Xq, sx, Z = run_rotate_quant(sq, rot, X)
     sel = np.arange(X.shape[0]) if rows is None else np.asarray(rows)
     Zo = ora.rotate(X[sel], R1, R2)
@@ -234,6 +235,82 @@ def test_rotate_quant_is_deterministic(sq):
     for x, y in zip(a, b):
         assert np.array_equal(x.view(np.uint8), y.view(np.uint8))
     rot.close()
+
+
+# ------------------------------------------------------------------ steps 1+2, R2 applied through its structure
+ST_SHAPES = [(64, 64, 37), (64, 64, 301), (8, 64, 9), (24, 64, 7), (48, 64, 11), (128, 64, 5), (100, 64, 3),
+             (32, 128, 5), (100, 128, 3), (112, 128, 4), (64, 128, 6), (128, 128, 3), (16, 128, 13)]
+
+
+def _structured_pair(sq, X, n1, n2, flags, seed=3):
+    """The oracle's factors and the library's handle for the same calibration batch and the same random
+    block O; the handle applies R2 = H R2^U piece by piece, the oracle as the dense product."""
+    O = ora.haar_orthogonal(n1 - 2, np.random.default_rng(seed)) if n1 > 2 else None
+    R1, R2 = ora.build_rotation(X.astype(np.float32), n1, n2, flags=flags, O=O)
+    rot = sq.sq_build_rotation(X.astype(np.float32), n1, n2, flags=flags | sq.SQ_ROT_APPLY_STRUCTURED, O=O)
+    return R1, R2, rot
+
+
+@pytest.mark.parametrize("n1,n2,M", ST_SHAPES)
+def test_structured_rotation_matches_oracle(sq, n1, n2, M):
+    w = wl.small(f"st{n1}x{n2}", M, n1, n2, 8, seed=n1 * 5 + n2)
+    X = wl.make_activations(w)
+    R1, R2, rot = _structured_pair(sq, X, n1, n2, ora.ROT_DEFAULT)
+    assert rot.structured
+    check_rotate_quant(sq, X, R1, R2, rot=rot)
+
+
+@pytest.mark.parametrize("flags", [0, 1, 2, 3, 4, 5, 6])
+@pytest.mark.parametrize("n1,n2,M", [(64, 64, 21), (112, 128, 5)])
+def test_structured_rotation_with_components_switched_off(sq, n1, n2, M, flags):
+    """Every subset of ART / URT / Hadamard: R2 is H R2^U, H alone, R2^U alone or the identity."""
+    w = wl.small(f"stf{n1}x{n2}", M, n1, n2, 8, seed=n1 + n2 + flags)
+    X = wl.make_activations(w)
+    R1, R2, rot = _structured_pair(sq, X, n1, n2, flags)
+    assert rot.structured
+    check_rotate_quant(sq, X, R1, R2, rot=rot)
+
+
+def test_structured_and_dense_application_agree(sq):
+    """The same handle built without SQ_ROT_APPLY_STRUCTURED holds the same factors and rotates through
+    the dense kernel; both are within the tolerance of the oracle, and their rotated rows within 2e-5
+    of each other."""
+    w = wl.small("stvsd", 70, 64, 64, 8, 91)
+    X = wl.make_activations(w)
+    R1, R2, rot = _structured_pair(sq, X, 64, 64, ora.ROT_DEFAULT)
+    O = ora.haar_orthogonal(62, np.random.default_rng(3))
+    dense = sq.sq_build_rotation(X.astype(np.float32), 64, 64, flags=sq.SQ_ROT_DEFAULT, O=O)
+    assert rot.structured and not dense.structured
+    for a, b in zip(rot.factors(), dense.factors()):
+        assert np.array_equal(a, b)
+    _, _, Zs = run_rotate_quant(sq, rot, X)
+    _, _, Zd = run_rotate_quant(sq, dense, X)
+    assert np.linalg.norm(Zs.astype(np.float64) - Zd) <= 2e-5 * np.linalg.norm(Zd)
+    check_rotate_quant(sq, X, R1, R2, rot=dense)
+    rot.close()
+
+
+@pytest.mark.parametrize("w", [wl.L7B_QKVO, wl.L70B_GATEUP, wl.decode_up(1), wl.decode_up(64), wl.decode_down(1),
+                               wl.decode_down(64)], ids=lambda w: w.name)
+def test_structured_rotation_full_configs(sq, w):
+    X = wl.make_activations(w)
+    R1, R2, rot = _structured_pair(sq, X, w.n1, w.n2, ora.ROT_DEFAULT, seed=w.seed)
+    assert rot.structured
+    rng = np.random.default_rng(4)
+    rows = np.unique(np.concatenate([[0, w.M - 1], rng.integers(0, w.M, size=min(w.M, 96))]))
+    check_rotate_quant(sq, X, R1, R2, rows=rows, rot=rot)
+
+
+def test_structured_rotation_many_short_rows_and_determinism(sq):
+    w = wl.small("stmany", 70001, 8, 64, 8, 78)
+    X = wl.make_activations(w)
+    R1, R2, rot = _structured_pair(sq, X, w.n1, w.n2, ora.ROT_DEFAULT)
+    a = run_rotate_quant(sq, rot, X, want_z=False)
+    b = run_rotate_quant(sq, rot, X, want_z=False)
+    assert np.array_equal(a[0], b[0]) and np.array_equal(a[1].view(np.uint16), b[1].view(np.uint16))
+    rng = np.random.default_rng(2)
+    rows = np.unique(np.concatenate([[0, 1, 2, 3, 65535, 65536, 69999, 70000], rng.integers(0, w.M, size=120)]))
+    check_rotate_quant(sq, X, R1, R2, rows=rows, rot=rot)
 
 
 # ------------------------------------------------------------------ step 3
