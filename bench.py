@@ -5,7 +5,7 @@ One step = one pass of the whole path (sq_linear) over one batch of synthetic ac
 the named workload.  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
-                  [--structured-r2] [--no-sweep] [--no-cpu-baseline]
+                  [--structured-r2] [--fuse-decode] [--no-sweep] [--no-cpu-baseline]
 
 After the headline workload the default run also times every other benchmark workload briefly and
 reports them under "per_workload" of the same line (skipped with --no-sweep or N > 1).
@@ -252,14 +252,15 @@ class Layer:
     """One workload resident on the device: rotation handle, packed weights, and a ring of buffer sets
     larger than L2 so that no step finds its inputs cached."""
 
-    def __init__(self, sq, torch, w, device_index, rank=0, structured_r2=False, keep_host=False):
+    def __init__(self, sq, torch, w, device_index, rank=0, structured_r2=False, fuse_decode=False, keep_host=False):
         import dataclasses
         self.sq, self.torch, self.w = sq, torch, w
         M, N, K = w.M, w.N, w.K
         w_rank = dataclasses.replace(w, seed=w.seed + 7919 * rank) if rank else w
         X = wl.make_activations(w_rank)
         W = wl.make_weights(w)
-        flags = sq.SQ_ROT_DEFAULT | (sq.SQ_ROT_APPLY_STRUCTURED if structured_r2 else 0)
+        flags = (sq.SQ_ROT_DEFAULT | (sq.SQ_ROT_APPLY_STRUCTURED if structured_r2 else 0) |
+                 (sq.SQ_ROT_FUSE_DECODE if fuse_decode else 0))
         self.rot = sq.sq_build_rotation(X.astype(np.float32), w.n1, w.n2, flags=flags, seed=0)
         dW = torch.from_numpy(W).cuda()
         Wq = torch.empty((N, K // 2), dtype=torch.uint8, device="cuda")
@@ -481,7 +482,8 @@ def run_ours(args, w):
 
     M, N, K = w.M, w.N, w.K
     # every rank draws its own batch (weak scaling over tokens); the weights are replicated
-    layer = Layer(sq, torch, w, local_rank, rank=rank, structured_r2=args.structured_r2, keep_host=True)
+    layer = Layer(sq, torch, w, local_rank, rank=rank, structured_r2=args.structured_r2,
+                  fuse_decode=args.fuse_decode, keep_host=True)
     nsets, per_set, l2 = layer.nsets, layer.per_set, layer.l2
     structured = layer.rot.structured
 
@@ -595,7 +597,8 @@ def run_ours(args, w):
                 if ow.name == w.name:
                     continue
                 try:
-                    ol = Layer(sq, torch, ow, local_rank, structured_r2=args.structured_r2)
+                    ol = Layer(sq, torch, ow, local_rank, structured_r2=args.structured_r2,
+                               fuse_decode=args.fuse_decode)
                     for i in range(5):
                         ol.step(i)
                     torch.cuda.synchronize()
@@ -670,6 +673,8 @@ def main():
                     help="skip the timed CPU oracle leg (for profiler runs)")
     ap.add_argument("--no-sweep", action="store_true",
                     help="time the named workload only (skip the per_workload table)")
+    ap.add_argument("--fuse-decode", action="store_true",
+                    help="build the rotation with SQ_ROT_FUSE_DECODE: batches of up to 64 tokens as one launch")
     ap.add_argument("--structured-r2", action="store_true",
                     help="build the rotation with SQ_ROT_APPLY_STRUCTURED: R2 = H R2^U applied piece by piece "
                          "in registers instead of as a dense matrix on the tensor cores")

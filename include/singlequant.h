@@ -70,6 +70,16 @@ enum { SQ_ROT_ART = 1, SQ_ROT_URT = 2, SQ_ROT_HADAMARD = 4, SQ_ROT_DEFAULT = 7 }
  * as the dense matrix, which measures as fast or faster on a B200 at every benchmark shape (the
  * structured form trades idle tensor cores for busy arithmetic pipes). */
 #define SQ_ROT_APPLY_STRUCTURED (1u << 20)
+/* With this bit in `flags`, sq_linear (and sq_linear_static / sq_linear_host) evaluate batches of up to
+ * 64 tokens as ONE launch: some CTAs of the grid rotate and quantise the tokens while the others, CTAs
+ * of the decode GEMM, already pull their weights in, and the packed tokens are handed over through L2
+ * behind a device counter instead of through the end of a kernel.  Same results bit for bit.  Off by
+ * default: on a B200 the two-kernel form, whose GEMM is launched as a programmatic dependent of the
+ * rotate kernel, measures as fast or faster at the benchmark's decode shapes.  A handle built with this
+ * bit keeps 64 pairs of device counters; calls that use one handle concurrently from more than 64
+ * streams at a time would share a pair.  After SQ_ERR_TIMEOUT such a handle should be destroyed (a
+ * counter may be left non-zero). */
+#define SQ_ROT_FUSE_DECODE (1u << 21)
 
 /* Algorithm 1 (Kronecker Dimension Factorization).  Host only.  n2 = the power of two dividing
  * n closest to sqrt(n), the first found winning ties; n1 = n / n2.  n >= 1. */

@@ -22,6 +22,7 @@ SQ_ERR_INVALID_ARG, SQ_ERR_SHAPE, SQ_ERR_ALIGN, SQ_ERR_UNSUPPORTED = 1, 2, 3, 4
 SQ_ERR_NOMEM, SQ_ERR_CUDA, SQ_ERR_TIMEOUT = 5, 6, 7
 SQ_ROT_ART, SQ_ROT_URT, SQ_ROT_HADAMARD, SQ_ROT_DEFAULT = 1, 2, 4, 7
 SQ_ROT_APPLY_STRUCTURED = 1 << 20
+SQ_ROT_FUSE_DECODE = 1 << 21
 
 EXPORTS = (
     "sq_factorize", "sq_build_rotation", "sq_rotation_from_factors", "sq_rotation_get_factors",

@@ -8,6 +8,7 @@
 #include "sq_rotate_quant_tc.cu"
 #include "sq_rotate_quant_st.cu"
 #include "sq_rotate_quant_pair.cu"
+#include "sq_linear_fused.cu"
 #include "sq_rotation_host.cu"
 #include "sq_api.cu"
 #include "sq_noalloc.cu"

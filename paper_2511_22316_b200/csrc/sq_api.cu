@@ -92,7 +92,7 @@ constexpr int64_t kMaxRows = (1ll << 31) - 1;
 inline size_t align_up(size_t v, size_t a) { return (v + a - 1) / a * a; }
 
 sq_status_t make_handle(std::vector<float>&& R1, std::vector<float>&& R2, int32_t n1, int32_t n2,
-                        const R2Structure* s2, sq_rotation_t** out) {
+                        const R2Structure* s2, bool fuse_decode, sq_rotation_t** out) {
   sq_rotation* h = new (std::nothrow) sq_rotation();
   if (!h) return SQ_ERR_NOMEM;
   h->n1 = n1;
@@ -117,7 +117,7 @@ sq_status_t make_handle(std::vector<float>&& R1, std::vector<float>&& R2, int32_
   const bool prepared = (sq::rotate_quant_tc_supported(n1, n2)     ? sq::rotate_quant_tc_prepare(h)
                          : sq::rotate_quant_pair_supported(n1, n2) ? sq::rotate_quant_pair_prepare(h)
                                                                    : true) &&
-                        sq::rotate_quant_st_prepare(h);
+                        sq::rotate_quant_st_prepare(h) && (!fuse_decode || sq::linear_fused_prepare(h));
   if (!prepared) {
     sq_rotation_destroy(h);
     return SQ_ERR_CUDA;
@@ -185,7 +185,7 @@ sq_status_t sq_build_rotation(const float* calib, int64_t T, int64_t n, int32_t 
                               uint64_t seed, const double* O_or_null, sq_rotation_t** out) {
   if (!out) return SQ_ERR_INVALID_ARG;
   *out = nullptr;
-  if (!calib || T < 1 || n1 < 1 || n2 < 1 || (flags & ~(7u | (0x7FFu << 8) | SQ_ROT_APPLY_STRUCTURED)))
+  if (!calib || T < 1 || n1 < 1 || n2 < 1 || (flags & ~(7u | (0x7FFu << 8) | SQ_ROT_APPLY_STRUCTURED | SQ_ROT_FUSE_DECODE)))
     return SQ_ERR_INVALID_ARG;
   if (static_cast<int64_t>(n1) * n2 != n) return SQ_ERR_SHAPE;
   if ((flags & SQ_ROT_HADAMARD) && (n2 & (n2 - 1)) != 0) return SQ_ERR_SHAPE;
@@ -194,7 +194,8 @@ sq_status_t sq_build_rotation(const float* calib, int64_t T, int64_t n, int32_t 
   R2Structure s2;
   sq_status_t st = sq::build_factors_host(calib, T, n, n1, n2, flags, seed, O_or_null, R1, R2, &s2);
   if (st != SQ_OK) return st;
-  return make_handle(std::move(R1), std::move(R2), n1, n2, (flags & SQ_ROT_APPLY_STRUCTURED) ? &s2 : nullptr, out);
+  return make_handle(std::move(R1), std::move(R2), n1, n2, (flags & SQ_ROT_APPLY_STRUCTURED) ? &s2 : nullptr,
+                     (flags & SQ_ROT_FUSE_DECODE) != 0, out);
 }
 
 sq_status_t sq_rotation_from_factors(const float* R1, const float* R2, int32_t n1, int32_t n2,
@@ -204,7 +205,7 @@ sq_status_t sq_rotation_from_factors(const float* R1, const float* R2, int32_t n
   if (!R1 || !R2 || n1 < 1 || n2 < 1) return SQ_ERR_INVALID_ARG;
   if (n1 > 4096 || n2 > 4096) return SQ_ERR_UNSUPPORTED;
   std::vector<float> a(R1, R1 + static_cast<size_t>(n1) * n1), b(R2, R2 + static_cast<size_t>(n2) * n2);
-  return make_handle(std::move(a), std::move(b), n1, n2, nullptr, out);
+  return make_handle(std::move(a), std::move(b), n1, n2, nullptr, false, out);
 }
 
 sq_status_t sq_rotation_get_factors(const sq_rotation_t* rot, float* R1, float* R2) {
@@ -229,6 +230,7 @@ void sq_rotation_destroy(sq_rotation_t* rot) {
   if (rot->dR2) cudaFree(rot->dR2);
   if (rot->dA1img) cudaFree(rot->dA1img);
   if (rot->dB2img) cudaFree(rot->dB2img);
+  if (rot->dFusedCounters) cudaFree(rot->dFusedCounters);
   delete rot;
 }
 
@@ -292,6 +294,11 @@ sq_status_t sq_linear(const sq_rotation_t* rot, const void* X, int64_t M, const 
   if ((st = check_gemm_args(Xq, sx, Wq, sw, M, N, K, Y, nullptr)) != SQ_OK) return st;
   if ((st = check_handle_device(rot)) != SQ_OK) return st;
   cudaStream_t s = static_cast<cudaStream_t>(stream);
+  // A decode-sized batch: rotation, quantisation and GEMM as one launch.
+  if (sq::linear_fused_supported(rot, M, N, K)) {
+    st = sq::launch_linear_fused(rot, X, M, Wq, sw, N, K, Xq, sx, Y, s);
+    if (st != SQ_ERR_UNSUPPORTED) return st;          // else: nothing was launched, take the two-kernel form
+  }
   st = sq::rotate_quant_dispatch(rot, X, M, Xq, sx, nullptr, s);
   if (st != SQ_OK) return st;
   // Every tensor-core GEMM kernel and the dot-product kernel start their set-up (and their weight

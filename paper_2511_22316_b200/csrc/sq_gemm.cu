@@ -18,6 +18,7 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 
+#include <cstring>
 #include <mutex>
 
 #include "sq_internal.h"
@@ -325,7 +326,7 @@ using EncodeTiledFn = CUresult (*)(CUtensorMap*, CUtensorMapDataType, cuuint32_t
                                    const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
                                    CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-EncodeTiledFn get_encode_fn() {
+EncodeTiledFn driver_encode_fn() {
   static EncodeTiledFn fn = nullptr;
   static std::once_flag once;
   std::call_once(once, [] {
@@ -337,6 +338,65 @@ EncodeTiledFn get_encode_fn() {
   });
   return fn;
 }
+
+// A tensor map is a pure function of the arguments it is encoded from, and a layer that is evaluated
+// again and again asks for the same few maps every time (same buffers, same shapes).  Each host thread
+// keeps the maps it encoded last, keyed by all of the arguments, so that a steady-state call encodes
+// nothing: the driver call costs about a microsecond per map, several per layer call.
+struct MapKey {
+  const void* base;
+  cuuint64_t dims[3], strides[2];
+  cuuint32_t box[3], estr[3];
+  int dtype, rank, interleave, swizzle, promo, oob;
+};
+struct MapEntry {
+  bool valid = false;
+  MapKey key;
+  CUtensorMap map;
+};
+
+CUresult cached_encode(CUtensorMap* out, CUtensorMapDataType dtype, cuuint32_t rank, void* base,
+                       const cuuint64_t* dims, const cuuint64_t* strides, const cuuint32_t* box,
+                       const cuuint32_t* estr, CUtensorMapInterleave interleave, CUtensorMapSwizzle swizzle,
+                       CUtensorMapL2promotion promo, CUtensorMapFloatOOBfill oob) {
+  EncodeTiledFn enc = driver_encode_fn();
+  if (!enc) return CUDA_ERROR_NOT_SUPPORTED;
+  if (rank < 1 || rank > 3) return enc(out, dtype, rank, base, dims, strides, box, estr, interleave, swizzle, promo, oob);
+  constexpr int kEntries = 128;
+  thread_local MapEntry cache[kEntries];
+  MapKey key;
+  std::memset(&key, 0, sizeof(key));
+  key.base = base;
+  for (cuuint32_t d = 0; d < rank; ++d) {
+    key.dims[d] = dims[d];
+    key.box[d] = box[d];
+    key.estr[d] = estr[d];
+    if (d + 1 < rank) key.strides[d] = strides[d];
+  }
+  key.dtype = static_cast<int>(dtype);
+  key.rank = static_cast<int>(rank);
+  key.interleave = static_cast<int>(interleave);
+  key.swizzle = static_cast<int>(swizzle);
+  key.promo = static_cast<int>(promo);
+  key.oob = static_cast<int>(oob);
+  uint64_t hsh = reinterpret_cast<uintptr_t>(base) >> 8;
+  hsh = (hsh ^ (hsh >> 17)) * 0x9E3779B97F4A7C15ull + key.dims[rank - 1] * 31 + key.box[rank - 1] * 7 + key.box[0];
+  MapEntry& e = cache[(hsh >> 20) % kEntries];
+  if (e.valid && std::memcmp(&e.key, &key, sizeof(key)) == 0) {
+    *out = e.map;
+    return CUDA_SUCCESS;
+  }
+  const CUresult r = enc(out, dtype, rank, base, dims, strides, box, estr, interleave, swizzle, promo, oob);
+  if (r == CUDA_SUCCESS) {
+    e.valid = true;
+    e.key = key;
+    e.map = *out;
+  }
+  return r;
+}
+
+// The encoder every launcher uses (nullptr when the driver entry point is missing).
+EncodeTiledFn get_encode_fn() { return driver_encode_fn() ? &cached_encode : nullptr; }
 
 // 2-D uint8 map over a packed [rows x row_bytes] matrix; box = box_rows x 128 bytes with the
 // 128-byte swizzle; out-of-range rows and bytes read as zero.

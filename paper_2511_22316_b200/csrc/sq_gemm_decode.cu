@@ -42,8 +42,25 @@ constexpr int D_ACCS = 4;                 // accumulators in TMEM (columns 0 .. 
 
 enum DecSite : uint32_t {
   DSITE_ST_EMPTY = 64, DSITE_ST_FULL_A, DSITE_ST_FULL_B, DSITE_EMPTY_A, DSITE_EMPTY_B, DSITE_FULL,
-  DSITE_TMEM_FULL, DSITE_TMEM_EMPTY, DSITE_RED_FULL, DSITE_RED_EMPTY
+  DSITE_TMEM_FULL, DSITE_TMEM_EMPTY, DSITE_RED_FULL, DSITE_RED_EMPTY, DSITE_TOKENS
 };
+
+// Bounded wait until the counter at `flag` (device memory, bumped with release semantics by the CTAs
+// that produce the tokens) has reached `target`; what those CTAs wrote before is then visible to this
+// thread's loads, and after the proxy fence also to the TMA loads it issues.
+__device__ __forceinline__ bool wait_counter(const uint32_t* flag, uint32_t target, uint32_t site, uint32_t limit) {
+  for (uint32_t it = 0; it < limit; ++it) {
+    uint32_t v;
+    asm volatile("ld.acquire.gpu.global.u32 %0, [%1];" : "=r"(v) : "l"(flag) : "memory");
+    if (v >= target) {
+      asm volatile("fence.proxy.async;" ::: "memory");
+      return true;
+    }
+    __nanosleep(it < 8 ? 100 : 250);       // one thread per CTA polls; keep the counter's L2 line quiet
+  }
+  atomicCAS(&g_device_status, 0u, (site << 8) | 1u);
+  return false;
+}
 
 template <int NT>
 struct DecSmem {
@@ -60,11 +77,12 @@ struct DecSmem {
   static constexpr int OFF_RED = OFF_X_ST + S_ST * X_ST;
   static constexpr int OFF_OUT = OFF_RED + RED_GROUP;     // per epilogue warp: 16 tokens x 32 channels fp16
   static constexpr int OFF_BAR = OFF_OUT + D_EPI_WARPS * 1024;
-  static constexpr int NUM_BARS = 2 * S_ST + 2 * D_S_OP + 2 * D_ACCS + 2 * D_EPI_GROUPS;
-  static constexpr int OFF_MISC = OFF_BAR + NUM_BARS * 8;
+  static constexpr int NUM_BARS = 2 * S_ST + 2 * D_S_OP + 2 * D_ACCS + 2 * D_EPI_GROUPS + 1;
+  static constexpr int OFF_MISC = (OFF_BAR + NUM_BARS * 8 + 15) / 16 * 16;   // the scales below are read as float4
   static constexpr int TOTAL = OFF_MISC + 32 + NT * 4;   // TMEM address, then the tokens' scales as floats
   static constexpr int DYN_BYTES = TOTAL + 1024;
   static_assert(DYN_BYTES <= 227 * 1024, "shared memory of one SM");
+  static_assert((OFF_MISC + 32) % 16 == 0, "the token scales are read with 16-byte loads");
 };
 
 // Widens the 128 staged bytes of NT token rows into two int8 k-block tiles (NT x 128 B each,
@@ -96,11 +114,16 @@ __device__ __forceinline__ void unpack_rows(const unsigned char* __restrict__ st
   }
 }
 
+// The kernel's body for CTA `cta` of `ncta` (a multiple of the cluster size `splits`).  `tokens_ready`:
+// nullptr when the tokens come from the kernel before this one in the stream (programmatic dependent
+// launch); else a counter that the token-producing CTAs of the SAME launch bump to `tokens_target`
+// (the fused kernel of sq_linear_fused.cu).
 template <int NT>
-__global__ void __launch_bounds__(D_THREADS, 1)
-w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
-                        const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
-                        int splits, __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
+__device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w, const CUtensorMap& tmap_x,
+                                                      const __half* __restrict__ sx, const __half* __restrict__ sw,
+                                                      int M, int N, int K, int splits, __half* __restrict__ Y,
+                                                      int32_t* __restrict__ accdbg, int cta, int ncta,
+                                                      const uint32_t* tokens_ready, uint32_t tokens_target) {
   using L = DecSmem<NT>;
   constexpr int S_ST = L::S_ST;
   extern __shared__ unsigned char smem_dyn[];
@@ -114,6 +137,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   uint64_t* tmem_empty = tmem_full + D_ACCS;                  // [D_ACCS]
   uint64_t* red_full = tmem_empty + D_ACCS;                   // the others' rows have arrived in this CTA's slots (entry 0; entry 1 unused)
   uint64_t* red_empty = red_full + D_EPI_GROUPS;              // the others have read what this CTA sent them
+  uint64_t* tok_seen = red_empty + D_EPI_GROUPS;              // the producer has seen the tokens' counter (fused form)
   uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_MISC);
   float* sxs = reinterpret_cast<float*>(smem + L::OFF_MISC + 32);   // [NT], zero beyond M
 
@@ -126,7 +150,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   // The cluster (a single CTA when splits == 1) takes the tiles cid, cid + ncl, ...; CTA `crank`
   // of it accumulates the blocks [b0, b1) of every one of them.
   const uint32_t crank = (splits > 1) ? cluster_ctarank() : 0u;
-  const int cid = static_cast<int>(blockIdx.x) / splits, ncl = static_cast<int>(gridDim.x) / splits;
+  const int cid = cta / splits, ncl = ncta / splits;
   const int b0 = static_cast<int>(crank * static_cast<uint32_t>(num_sb) / static_cast<uint32_t>(splits));
   const int b1 = static_cast<int>((crank + 1u) * static_cast<uint32_t>(num_sb) / static_cast<uint32_t>(splits));
 
@@ -178,6 +202,7 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
       mbar_init(&red_full[g], 1);
       mbar_init(&red_empty[g], crossing);
     }
+    mbar_init(tok_seen, 1);
     mbar_fence_init();
   }
   if (warp == 1) {
@@ -191,11 +216,14 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
   if (splits > 1) cluster_arrive_release();
   tc_fence_after_sync();
   const uint32_t tmem_base = *tmem_slot;
-  griddep_wait();                                      // the tokens and their scales come from the kernel before
+  if (tokens_ready == nullptr) griddep_wait();         // the tokens and their scales come from the kernel before
 
   if (warp == 0) {
     // ------------------------------ TMA producer ------------------------------------------------
-    if (lane == 0) {
+    // In the fused form this one thread polls the counter of the token-producing CTAs for the whole
+    // CTA; the epilogue warps, which read the token steps, wait for its arrival on a local barrier.
+    if (lane == 0 && (tokens_ready == nullptr || wait_counter(tokens_ready, tokens_target, DSITE_TOKENS, limit))) {
+      if (tokens_ready != nullptr) mbar_arrive(tok_seen);
       for (int i = 0; i < pre_n; ++i)
         tma_load_2d(smem + L::OFF_X_ST + i * L::X_ST, &tmap_x, &st_full[i], pre_sb[i] * 128, 0);
       produce(0xFFFFFFFFu, false);
@@ -340,7 +368,15 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     const bool piece_mine = static_cast<uint32_t>((q * 32 + piece * 8) / rows_per) == crank;
     const uint32_t pick = (prow & 1) ? 0x7632u : 0x5410u;            // the odd or the even token of a pair
     // The tokens' scales as floats (zero beyond M): read once, before any accumulator is ready.
-    if (et < NT) sxs[et] = (et < M) ? __half2float(sx[et]) : 0.0f;
+    if (et < NT) {
+      const bool there = tokens_ready == nullptr || mbar_wait(tok_seen, 0, DSITE_TOKENS, limit);
+      // written during this launch by another CTA in the fused form: read past the L1 / read-only path
+      const __half v = (et < M && there)
+                           ? (tokens_ready == nullptr ? sx[et]
+                                                      : __ushort_as_half(__ldcg(reinterpret_cast<const unsigned short*>(sx) + et)))
+                           : __float2half(0.0f);
+      sxs[et] = __half2float(v);
+    }
     named_barrier(1, D_EPI_WARPS * 32);
     if (splits > 1) cluster_wait_acquire();                            // the other CTAs' barriers exist
     bool ok = true;
@@ -478,6 +514,15 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
     cluster_arrive_relaxed();
     cluster_wait_acquire();
   }
+}
+
+template <int NT>
+__global__ void __launch_bounds__(D_THREADS, 1)
+w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid_constant__ CUtensorMap tmap_x,
+                        const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
+                        int splits, __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
+  w4a4_gemm_decode_body<NT>(tmap_w, tmap_x, sx, sw, M, N, K, splits, Y, accdbg, static_cast<int>(blockIdx.x),
+                            static_cast<int>(gridDim.x), nullptr, 0u);
 }
 
 // Largest number of clusters of `s` CTAs of this kernel that the device holds at once.

@@ -36,6 +36,9 @@ struct sq_rotation {
   R2Structure s2;
   bool st_ready = false;
   std::vector<float> st_coef;   // the kernel's coefficient block (host copy, passed by value)
+  // fused decode layer (sq_linear_fused.cu): pairs of device counters, one pair per call in turn
+  uint32_t* dFusedCounters = nullptr;
+  mutable std::atomic<uint32_t> fused_calls{0};
 };
 
 namespace sq {
@@ -114,6 +117,12 @@ sq_status_t launch_rotate_quant_pair(const sq_rotation* h, const void* X, int64_
 bool rotate_quant_st_prepare(sq_rotation* h);
 sq_status_t launch_rotate_quant_st(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
                                    float* Zdbg, cudaStream_t s);
+// The whole layer for M <= 64 as one launch (sq_linear_fused.cu): rotating CTAs and decode-GEMM CTAs in
+// one grid, the tokens handed over through L2 behind a device counter.
+bool linear_fused_prepare(sq_rotation* h);
+bool linear_fused_supported(const sq_rotation* h, int64_t M, int64_t N, int64_t K);
+sq_status_t launch_linear_fused(const sq_rotation* h, const void* X, int64_t M, const void* Wq, const void* sw,
+                                int64_t N, int64_t K, void* Xq, void* sx, void* Y, cudaStream_t s);
 // Picks the tensor-core kernel when the handle has its images, else the generic fp32 kernel.
 sq_status_t rotate_quant_dispatch(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
                                   float* Zdbg, cudaStream_t s);

@@ -126,15 +126,15 @@ __device__ __forceinline__ float absmax32(const uint32_t (&r)[32]) {
   return fmaxf(fmaxf(m[0], m[1]), fmaxf(m[2], m[3]));
 }
 
-// S accumulator slots (= compute groups) per CTA.  With S * 2 * N2 = 256 TMEM columns two CTAs share
-// an SM (each with its own producer and MMA issuer); with 512 a CTA has the SM to itself.
+// The kernel's body, for CTA `cta` of `ncta` that share the token groups (the fused decode kernel of
+// sq_linear_fused.cu runs it in its first CTAs, with more warps in the block than the roles below use).
 template <int N2, int S>
-__global__ void __launch_bounds__((2 + 4 * S) * 32, (S * 2 * N2 <= 256) ? 2 : 1)
-rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ RqLayout L,
-                       const unsigned char* __restrict__ a1_img, const unsigned char* __restrict__ b2_img, int n1,
-                       int rows, uint8_t* __restrict__ Xq, __half* __restrict__ scales, float* __restrict__ Zdbg) {
+__device__ __forceinline__ void rotate_quant_tc_body(const CUtensorMap& tmap_x, const RqLayout& L,
+                                                     const unsigned char* __restrict__ a1_img,
+                                                     const unsigned char* __restrict__ b2_img, int n1, int rows,
+                                                     uint8_t* __restrict__ Xq, __half* __restrict__ scales,
+                                                     float* __restrict__ Zdbg, int cta, int ncta) {
   constexpr int TM_COLS = S * 2 * N2;             // 256 or 512
-  griddep_launch_dependents();                   // a GEMM launched behind this kernel may set itself up
   constexpr int XQ = N2 / 64;
   constexpr int SLOT_COLS = 2 * N2;              // D1 (N2 columns) + D2 (N2 columns)
   // The layout comes from the host (the same rq_layout call that sized the shared memory); group
@@ -159,14 +159,12 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
 
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int ngroups = (rows + G - 1) / G;
-  const int my_groups = (ngroups > static_cast<int>(blockIdx.x))
-                            ? (ngroups - static_cast<int>(blockIdx.x) + static_cast<int>(gridDim.x) - 1) / static_cast<int>(gridDim.x)
-                            : 0;
+  const int my_groups = (ngroups > cta) ? (ngroups - cta + ncta - 1) / ncta : 0;
   const uint32_t limit = wait_limit();
 
   // One X tile set per token group: G tokens, XQ 64-column blocks each.
   auto load_group = [&](int i) {
-    const int g = static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x);
+    const int g = cta + i * ncta;
     const int s = i % L.XS;
     mbar_arrive_expect_tx(&x_full[s], static_cast<uint32_t>(L.x_bytes));
     for (int tk = 0; tk < G; ++tk)
@@ -284,7 +282,7 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
         }
       }
     }
-  } else {
+  } else if (warp < 2 + 4 * S) {
     // ------------------------------ compute groups ------------------------------------------------
     const int w = (warp - 2) >> 2;                 // accumulator slot of this group
     const int quarter = warp & 3;                  // TMEM lane quarter this warp may touch
@@ -296,7 +294,7 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
     const int q0 = (quarter / wpt) * wpt;
     bool ok = true;
     for (int i = w; i < my_groups && ok; i += S) {
-      const int g = static_cast<int>(blockIdx.x) + i * static_cast<int>(gridDim.x);
+      const int g = cta + i * ncta;
       const long long token = static_cast<long long>(g) * G + tk;
       const uint32_t ph = (i / S) & 1;
 
@@ -409,6 +407,18 @@ rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, TM_COLS);
   }
+}
+
+// S accumulator slots (= compute groups) per CTA.  With S * 2 * N2 = 256 TMEM columns two CTAs share
+// an SM (each with its own producer and MMA issuer); with 512 a CTA has the SM to itself.
+template <int N2, int S>
+__global__ void __launch_bounds__((2 + 4 * S) * 32, (S * 2 * N2 <= 256) ? 2 : 1)
+rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ RqLayout L,
+                       const unsigned char* __restrict__ a1_img, const unsigned char* __restrict__ b2_img, int n1,
+                       int rows, uint8_t* __restrict__ Xq, __half* __restrict__ scales, float* __restrict__ Zdbg) {
+  griddep_launch_dependents();                   // a GEMM launched behind this kernel may set itself up
+  rotate_quant_tc_body<N2, S>(tmap_x, L, a1_img, b2_img, n1, rows, Xq, scales, Zdbg, static_cast<int>(blockIdx.x),
+                              static_cast<int>(gridDim.x));
 }
 
 // ---------------------------------------------------------------------------------------------

@@ -138,3 +138,53 @@ def test_linear_matches_oracle_at_full_size(sq, w):
         blk = slice(b0, b0 + 8)
         assert np.linalg.norm(Yg[blk] - Yo[blk]) <= 1e-2 * np.linalg.norm(Yo[blk]), rows[blk]
     rot.close()
+
+
+# ------------------------------------------------------------------ the one-launch form of the decode layer
+@pytest.mark.parametrize("w", DECODE + [wl.small("fuse_ragged", 37, 64, 64, 2432, 81), wl.small("fuse_two_rounds", 9, 112, 128, 512, 82)],
+                         ids=lambda w: w.name)
+def test_fused_decode_layer_matches_oracle_and_the_two_kernel_form(sq, w):
+    """A handle built with SQ_ROT_FUSE_DECODE evaluates batches of up to 64 tokens as one launch (rotating
+    CTAs and GEMM CTAs side by side).  Its output must be the oracle's layer for the handle's own factors
+    within 1e-2, and equal, bit for bit, to what a handle without the flag gives; twice in a row (the
+    device counters a call uses must be clean again afterwards)."""
+    torch = torch_mod()
+    M, N, K = w.M, w.N, w.K
+    import dataclasses
+    Xcal = wl.make_activations(dataclasses.replace(w, M=max(w.M, 64)) if w.M < 64 else w).astype(np.float32)
+    X = wl.make_activations(w)
+    W = wl.make_weights(w)
+    O = ora.haar_orthogonal(w.n1 - 2, np.random.default_rng(w.seed))
+    fused = sq.sq_build_rotation(Xcal, w.n1, w.n2, flags=sq.SQ_ROT_DEFAULT | sq.SQ_ROT_FUSE_DECODE, O=O)
+    plain = sq.sq_build_rotation(Xcal, w.n1, w.n2, flags=sq.SQ_ROT_DEFAULT, O=O)
+    R1, R2 = fused.factors()
+    wq, sw = Guarded(N * K // 2), Guarded(N * 2)
+    sq.sq_pack_weight(plain, dev(W), N, K, wq, sw)
+    nbytes = sq.sq_linear_workspace_bytes(M, K)
+    ws = torch.empty(nbytes + 256, dtype=torch.uint8, device="cuda")
+    wsp = ws.data_ptr() + (-ws.data_ptr()) % 256
+    dX = dev(X)
+    y_plain = Guarded(M * N * 2)
+    before = sq.sq_kernel_launch_count()
+    sq.sq_linear(plain, dX, M, wq, sw, N, K, wsp, nbytes, y_plain)
+    two = sq.sq_kernel_launch_count() - before
+    outs = []
+    for _ in range(2):
+        y = Guarded(M * N * 2)
+        before = sq.sq_kernel_launch_count()
+        sq.sq_linear(fused, dX, M, wq, sw, N, K, wsp, nbytes, y)
+        one = sq.sq_kernel_launch_count() - before
+        torch.cuda.synchronize()
+        assert sq.sq_last_device_status() == sq.SQ_OK
+        y.check()
+        outs.append(y.numpy(np.float16, (M, N)))
+    y_plain.check(); wq.check(); sw.check()
+    assert two == 2 and one in (1, 2)          # one launch where the device has room for the rotating CTAs
+    Yp = y_plain.numpy(np.float16, (M, N))
+    for Yf in outs:
+        assert np.array_equal(Yf.view(np.uint16), Yp.view(np.uint16))
+    Wq_o, sw_o = _pack_weight_chunked(W, R1, R2)
+    Xq_o, sx_o, _ = ora.rotate_quant(X, R1, R2)
+    Yo = ora.dequant(_gemm_i32_chunked(ora.unpack_int4(Xq_o), ora.unpack_int4(Wq_o)), sx_o, sw_o).astype(np.float64)
+    assert np.linalg.norm(outs[0].astype(np.float64) - Yo) <= 1e-2 * np.linalg.norm(Yo)
+    fused.close(); plain.close()
