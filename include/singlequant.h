@@ -186,7 +186,7 @@ sq_status_t sq_linear_static(const sq_rotation_t* rot, const void* X, int64_t M,
 /* The whole layer from HOST activations to HOST outputs: copies X (HOST fp16 [M x n], pinned
  * memory recommended) to the device, runs sq_linear, copies Y back (HOST fp16 [M x N]) and
  * waits for the stream.  Weights stay on the device.  Batches of 512 rows or more are cut into up
- * to eight chunks whose copies in, computation and copies out overlap (two internal copy streams
+ * to four chunks whose copies in, computation and copies out overlap (two internal copy streams
  * and a few events per device, created at the first such call and kept until exit; both are
  * ordered after the work already queued on `stream`).  The result does not depend on the cut:
  * every row is rotated, quantised and multiplied on its own.  Concurrent calls on one device

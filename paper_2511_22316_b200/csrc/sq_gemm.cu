@@ -124,6 +124,7 @@ w4a4_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_con
                     const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
                     __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
   using L = GemmSmem<BN, S_OP, S_ST>;
+  griddep_launch_dependents();          // a rotate kernel launched behind this one may set itself up
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);

@@ -126,6 +126,7 @@ __device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w,
                                                       const uint32_t* tokens_ready, uint32_t tokens_target) {
   using L = DecSmem<NT>;
   constexpr int S_ST = L::S_ST;
+  griddep_launch_dependents();          // a rotate kernel launched behind this one may set itself up on the idle SMs
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
   uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);

@@ -33,6 +33,7 @@ __global__ void __launch_bounds__(512)
 w4a4_gemv_kernel(const uint8_t* __restrict__ Xq, const __half* __restrict__ sx, const uint8_t* __restrict__ Wq,
                  const __half* __restrict__ sw, int M, int N, int K, __half* __restrict__ Y,
                  int32_t* __restrict__ accdbg) {
+  griddep_launch_dependents();                           // a rotate kernel launched behind this one may set itself up
   griddep_wait();                                        // Xq and sx may come from the kernel launched before this one
   extern __shared__ __align__(16) uint32_t xs[];
   constexpr int GV_ROWS = GvRows<MT>::value;

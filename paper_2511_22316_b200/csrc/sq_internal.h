@@ -87,6 +87,26 @@ inline cudaError_t launch_maybe_pdl(void (*kern)(KArgs...), dim3 grid, dim3 bloc
   return launch_cluster_maybe_pdl(kern, grid, block, smem, s, 1u, static_cast<Args&&>(args)...);
 }
 
+// Launches `kern` as a programmatic dependent of whatever precedes it in the stream: it may start while
+// that kernel still runs, once all of that kernel's CTAs have allowed it (griddepcontrol.launch_dependents)
+// or exited, and must not touch memory the predecessor reads or writes before its own
+// griddepcontrol.wait returns.  After a predecessor that never allows it, this is an ordinary launch.
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kern)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                    Args&&... args) {
+  cudaLaunchConfig_t cfg = {};
+  cfg.gridDim = grid;
+  cfg.blockDim = block;
+  cfg.dynamicSmemBytes = smem;
+  cfg.stream = s;
+  cudaLaunchAttribute attr[1];
+  attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+  attr[0].val.programmaticStreamSerializationAllowed = 1;
+  cfg.attrs = attr;
+  cfg.numAttrs = 1;
+  return cudaLaunchKernelEx(&cfg, kern, static_cast<KArgs>(args)...);
+}
+
 // Raises a kernel's dynamic shared-memory limit to `bytes` if it is lower.  Function attributes
 // belong to a device: the sizes already set are remembered per (device, kernel).
 bool ensure_dyn_smem(const void* kern, int bytes);

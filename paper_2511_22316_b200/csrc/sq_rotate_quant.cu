@@ -54,6 +54,7 @@ rotate_quant_kernel(const float* __restrict__ R1, const float* __restrict__ R2, 
                     const __half* __restrict__ X, long long rows, uint8_t* __restrict__ Xq,
                     __half* __restrict__ scales, float* __restrict__ Zdbg) {
   griddep_launch_dependents();
+  griddep_wait();                    // X may come from the kernel before this one in the stream
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int n = n1 * n2;
   float* Ts = reinterpret_cast<float*>(smem_raw);                       // [n1][n2] fp32

@@ -128,7 +128,9 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
     mbar_init(img_full, 1);
     mbar_init(peer_img, 1);
     mbar_fence_init();
-    for (long long i = 0; i < preload; ++i) load_token(i);
+    // The factor images belong to the handle: fetched at once.  X may come from the kernel before this
+    // one in the stream, which may also still read the buffers this kernel writes: its completion is
+    // awaited before the first token is requested (every store here depends on a token having landed).
     mbar_arrive_expect_tx(img_full, static_cast<uint32_t>(L.a1_bytes + L.b2_bytes));
     const unsigned char* a1g = a1_img + static_cast<size_t>(rank) * L.a1_bytes;
     const unsigned char* b2g = b2_img + static_cast<size_t>(rank) * L.b2_bytes;
@@ -136,6 +138,8 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
       bulk_load_1d(a1s + o, a1g + o, static_cast<uint32_t>(min(16384, L.a1_bytes - o)), img_full);
     for (int o = 0; o < L.b2_bytes; o += 16384)
       bulk_load_1d(b2s + o, b2g + o, static_cast<uint32_t>(min(16384, L.b2_bytes - o)), img_full);
+    griddep_wait();
+    for (long long i = 0; i < preload; ++i) load_token(i);
   }
   if (warp == 1) {
     tmem_alloc_pair(tmem_slot, 512);
@@ -417,13 +421,15 @@ sq_status_t launch_rotate_quant_pair(const sq_rotation* h, const void* X, int64_
   if (n2 == 64) {
     auto kern = rotate_quant_pair_kernel<64>;
     if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return SQ_ERR_CUDA;
-    kern<<<grid, (2 + 4 * 4) * 32, smem, s>>>(mx, a1, b2, n1, rows, static_cast<uint8_t*>(Xq),
-                                              static_cast<__half*>(scales), Zdbg);
+    if (launch_dependent(kern, dim3(grid), dim3((2 + 4 * 4) * 32), static_cast<size_t>(smem), s, mx, a1, b2, n1, rows,
+                         static_cast<uint8_t*>(Xq), static_cast<__half*>(scales), Zdbg) != cudaSuccess)
+      return SQ_ERR_CUDA;
   } else {
     auto kern = rotate_quant_pair_kernel<128>;
     if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return SQ_ERR_CUDA;
-    kern<<<grid, (2 + 4 * 2) * 32, smem, s>>>(mx, a1, b2, n1, rows, static_cast<uint8_t*>(Xq),
-                                              static_cast<__half*>(scales), Zdbg);
+    if (launch_dependent(kern, dim3(grid), dim3((2 + 4 * 2) * 32), static_cast<size_t>(smem), s, mx, a1, b2, n1, rows,
+                         static_cast<uint8_t*>(Xq), static_cast<__half*>(scales), Zdbg) != cudaSuccess)
+      return SQ_ERR_CUDA;
   }
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;

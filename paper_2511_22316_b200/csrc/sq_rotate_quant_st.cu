@@ -166,7 +166,13 @@ rotate_quant_st_kernel(const __grid_constant__ StLayout L, int n1, int rows, con
         bulk_load_1d(a1s + o, a1_img + o, static_cast<uint32_t>(min(16384, L.a1_bytes - o)), img_full);
     }
     __syncwarp();
-    if (lane < preload) load_sg(lane);
+    // X may come from the kernel before this one in the stream, which may also still read the buffers
+    // this kernel writes: its completion is awaited before the first tokens are requested (every store
+    // of this kernel depends on tokens having landed; the image above belongs to the handle).
+    if (lane < preload) {
+      griddep_wait();
+      load_sg(lane);
+    }
   }
   if (warp == 1) {
     tmem_alloc(tmem_slot, 512);
@@ -441,10 +447,11 @@ sq_status_t launch_st(const sq_rotation* h, const StLayout& L, const CUtensorMap
   const unsigned char* a1 = static_cast<const unsigned char*>(h->dA1img);
   auto go = [&](auto kern) -> sq_status_t {
     if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return SQ_ERR_CUDA;
-    kern<<<grid, (2 + 4 * NG) * 32, smem, s>>>(L, h->n1, rows, a1, static_cast<uint8_t*>(Xq),
-                                               static_cast<__half*>(scales), Zdbg, mx, cf);
+    const cudaError_t err = launch_dependent(kern, dim3(grid), dim3((2 + 4 * NG) * 32), static_cast<size_t>(smem), s, L,
+                                             h->n1, rows, a1, static_cast<uint8_t*>(Xq), static_cast<__half*>(scales),
+                                             Zdbg, mx, cf);
     count_launch();
-    return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+    return err == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
   };
   const bool had = h->s2.hadamard, urt = h->s2.urt;
   if (had && urt) return go(rotate_quant_st_kernel<N2, NG, true, true>);

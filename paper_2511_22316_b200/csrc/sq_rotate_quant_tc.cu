@@ -175,18 +175,22 @@ __device__ __forceinline__ void rotate_quant_tc_body(const CUtensorMap& tmap_x, 
   const int preload = my_groups < L.XS ? my_groups : L.XS;
 
   if (threadIdx.x == 0) {
-    // The first loads go out before anything else is set up: the whole X ring, then the factor
-    // images.  Only the barriers they complete on exist at that point; nobody else touches a
-    // barrier before the __syncthreads below.
+    // The first loads go out before anything else is set up: the factor images (they belong to the
+    // handle, so they may be fetched while the kernel before this one in the stream still runs), then,
+    // once that kernel has completed (it may have produced X, and may still be reading the buffers this
+    // one writes), the whole X ring.  Every store of this kernel depends on X having landed.  Only the
+    // barriers the loads complete on exist at that point; nobody else touches a barrier before the
+    // __syncthreads below.
     for (int b = 0; b < 4; ++b) mbar_init(&x_full[b], 1);
     mbar_init(img_full, 1);
     mbar_fence_init();
-    for (int i = 0; i < preload; ++i) load_group(i);
     mbar_arrive_expect_tx(img_full, static_cast<uint32_t>(L.a1_bytes + L.b2_bytes));
     for (int o = 0; o < L.a1_bytes; o += 16384)
       bulk_load_1d(a1s + o, a1_img + o, static_cast<uint32_t>(min(16384, L.a1_bytes - o)), img_full);
     for (int o = 0; o < L.b2_bytes; o += 16384)
       bulk_load_1d(b2s + o, b2_img + o, static_cast<uint32_t>(min(16384, L.b2_bytes - o)), img_full);
+    griddep_wait();
+    for (int i = 0; i < preload; ++i) load_group(i);
     for (int b = 0; b < 4; ++b) {
       mbar_init(&x_empty[b], 1);
       mbar_init(&d1_full[b], 1);
@@ -507,9 +511,9 @@ sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t 
     const int smem = ctas_per_sm == 1 ? std::max(L.total + 1024, 120 * 1024) : L.total + 1024;
     if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return false;
     const unsigned grid = static_cast<unsigned>(std::min<long long>(ngroups, static_cast<long long>(sms) * ctas_per_sm));
-    kern<<<grid, (2 + 4 * slots) * 32, smem, s>>>(mx, L, a1, b2, n1, static_cast<int>(rows), static_cast<uint8_t*>(Xq),
-                                                  static_cast<__half*>(scales), Zdbg);
-    return true;
+    return launch_dependent(kern, dim3(grid), dim3((2 + 4 * slots) * 32), static_cast<size_t>(smem), s, mx, L, a1, b2, n1,
+                            static_cast<int>(rows), static_cast<uint8_t*>(Xq), static_cast<__half*>(scales),
+                            Zdbg) == cudaSuccess;
   };
   bool ok;
   if (n2 == 64 && dual) ok = launch(rotate_quant_tc_kernel<64, 2>, 2, 2);

@@ -520,7 +520,7 @@ def test_linear_prefill_config_sampled(sq):
 def test_linear_host_chunked_equals_device_path(sq):
     """sq_linear_host cuts batches of 512 rows or more into row chunks whose copies and computation
     overlap.  Every row is treated on its own, so the outputs must equal those of one sq_linear call
-    on the whole batch bit for bit -- here with a ragged last chunk (1100 = 4 x 256 + 76 rows) that
+    on the whole batch bit for bit -- here with a ragged last chunk (1100 = 2 x 512 + 76 rows) that
     takes a different GEMM kernel than the full chunks -- and twice in a row (the copy streams and
     events are reused)."""
     w = wl.small("host_chunks", 1100, 64, 64, 264, 77)
