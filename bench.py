@@ -5,7 +5,7 @@ One step = one pass of the whole path (sq_linear) over one batch of synthetic ac
 the named workload.  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
-                  [--structured-r2] [--fuse-decode] [--no-sweep] [--no-cpu-baseline]
+                  [--structured-r2] [--fuse-decode] [--no-sweep] [--no-cpu-baseline] [--quick]
 
 After the headline workload the default run also times every other benchmark workload briefly and
 reports them under "per_workload" of the same line (skipped with --no-sweep or N > 1).
@@ -42,12 +42,13 @@ INT8_OVER_BF16 = 2.0      # nominal dense ratio (4.5 POPS int8 : 2.25 PFLOP/s bf
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (bytes; None until a capture exists for that kernel and workload).
 NCU_TRAFFIC = {
-    ("gemm", "llama2_7b_qkvo_prefill"): 12632320,           # w4a4_gemm_pair_kernel: reads (Y stays in L2)
-    ("rotate_quant", "llama2_7b_qkvo_prefill"): 16888064,   # rotate_quant_tc_kernel
+    ("gemm", "llama2_7b_qkvo_prefill"): 12632832,           # w4a4_gemm_pair_kernel: reads (Y stays in L2)
+    ("rotate_quant", "llama2_7b_qkvo_prefill"): 16888576,   # rotate_quant_tc_kernel
+    ("rotate_quant_st", "llama2_7b_qkvo_prefill"): 16873472,  # rotate_quant_st_kernel (--structured-r2)
     ("gemm", "llama3_8b_up_decode_m16"): 29457152,          # w4a4_gemm_decode_kernel, K not split
-    ("gemm", "llama3_8b_down_decode_m16"): 29518848,        # w4a4_gemm_decode_kernel, K over clusters of 4
-    ("gemm", "llama3_8b_up_decode_m1"): 29409280,           # w4a4_gemv_kernel
-    ("rotate_quant", "llama2_7b_down_prefill"): 45403904,   # rotate_quant_pair_kernel
+    ("gemm", "llama3_8b_down_decode_m16"): 29519616,        # w4a4_gemm_decode_kernel, K over clusters of 4
+    ("gemm", "llama3_8b_up_decode_m1"): 29409024,           # w4a4_gemv_kernel
+    ("rotate_quant", "llama2_7b_down_prefill"): 45412608,   # rotate_quant_pair_kernel
 }
 
 
@@ -453,7 +454,7 @@ def rooflines(w, rq_ms, gemm_ms, pk, structured, yard=None):
             roof_gemm["yardstick"] = dict(yard, frac=gemm_tops / yard["tops"])
     roof_rq = {"kernel": rotate_kernel_name(w, structured), "bound": "hbm", "achieved": rq_gbs, "peak": pk["hbm_gbs"],
                "unit": "GB/s", "frac": rq_gbs / pk["hbm_gbs"],
-               "traffic": NCU_TRAFFIC.get(("rotate_quant", w.name)) if not structured else None,
+               "traffic": NCU_TRAFFIC.get(("rotate_quant_st" if structured else "rotate_quant", w.name)),
                "peak_source": f"{pk['source']} copy bandwidth", "ms_per_launch": rq_ms,
                "algorithmic_bytes": rotate_quant_bytes(w), "frac_of_spec_8000": rq_gbs / 8000.0}
     return roof_gemm, roof_rq
@@ -516,7 +517,7 @@ def run_ours(args, w):
     # ---- the same step for at least half a second, so that several clock samples fall inside it:
     # the step time and the clocks it ran at (time x median SM MHz lets a reader normalise) -----------
     sustained = None
-    if rank == 0 and world == 1:
+    if rank == 0 and world == 1 and not args.quick:
         n_sus = max(args.steps, int(np.ceil(600.0 / max(ms_total / args.steps, 1e-3))))
         n_sus = min(n_sus, 400000)
         t0 = time.perf_counter()
@@ -551,7 +552,7 @@ def run_ours(args, w):
     sync_all()
     e2e_ms = h0.elapsed_time(h1) / e2e_steps
     status = sq.sq_last_device_status()
-    link_ms = link_yardstick(torch, M * K * 2, M * N * 2) if (rank == 0 and world == 1) else None
+    link_ms = link_yardstick(torch, M * K * 2, M * N * 2) if (rank == 0 and world == 1 and not args.quick) else None
     del hws
 
     # ---- max over ranks ---------------------------------------------------------------------
@@ -567,7 +568,7 @@ def run_ours(args, w):
         pk = peaks()
         value = world * ops_per_step(w) / (ms_per_step * 1e-3) / 1e12
         e2e_value = world * ops_per_step(w) / (e2e_ms * 1e-3) / 1e12
-        yard = int8_yardstick(torch, w, l2) if world == 1 else None
+        yard = int8_yardstick(torch, w, l2) if (world == 1 and not args.quick) else None
         roof_gemm, roof_rq = rooflines(w, rq_ms, gemm_ms, pk, structured, yard)
         dominant, other = (roof_gemm, roof_rq) if gemm_ms >= rq_ms else (roof_rq, roof_gemm)
 
@@ -678,7 +679,12 @@ def main():
     ap.add_argument("--structured-r2", action="store_true",
                     help="build the rotation with SQ_ROT_APPLY_STRUCTURED: R2 = H R2^U applied piece by piece "
                          "in registers instead of as a dense matrix on the tensor cores")
+    ap.add_argument("--quick", action="store_true",
+                    help="the K timed steps and the per-kernel attribution only: no sustained pass, no yardsticks, "
+                         "no per-workload table, no CPU baseline (for profiler runs)")
     args = ap.parse_args()
+    if args.quick:
+        args.no_sweep = args.no_cpu_baseline = True
     if args.steps is None:
         args.steps = 20 if args.impl == "reference" else 20000
     w = wl.by_name(args.workload)
