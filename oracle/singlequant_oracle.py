@@ -247,8 +247,8 @@ def build_rotation(calib: np.ndarray, n1: int, n2: int, flags: int = ROT_DEFAULT
                    return_f64: bool = False, art_steps: int = 1):
     """Paragraph "The Overall SingleQuant Method": R1 = (R1^U R^A)^T, R2 = H R2^U.
 
-    The paper builds ART/URT "according to" the activation X without saying which vectors; the
-    reading taken here (listed with the other readings in the design notes):
+    The paper builds ART/URT "according to" the activation X without saying which vectors.  Any
+    choice yields an orthogonal R; the reading taken here:
       1. t* = the calibration token with the largest |entry|; A = its n1 x n2 reshape;
          (p*, q*) = position of that entry; c = column q* of A (length n1).
       2. R^A from c (ART).  c' = R^A c.
