@@ -53,8 +53,8 @@ __global__ void __launch_bounds__(512)
 rotate_quant_kernel(const float* __restrict__ R1, const float* __restrict__ R2, int n1, int n2,
                     const __half* __restrict__ X, long long rows, uint8_t* __restrict__ Xq,
                     __half* __restrict__ scales, float* __restrict__ Zdbg) {
-  griddep_launch_dependents();
   griddep_wait();                    // X may come from the kernel before this one in the stream
+  griddep_launch_dependents();       // a GEMM launched behind this kernel may set itself up from here on
   extern __shared__ __align__(16) unsigned char smem_raw[];
   const int n = n1 * n2;
   float* Ts = reinterpret_cast<float*>(smem_raw);                       // [n1][n2] fp32

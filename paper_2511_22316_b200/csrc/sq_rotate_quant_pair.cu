@@ -77,7 +77,6 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
                          uint8_t* __restrict__ Xq, __half* __restrict__ scales, float* __restrict__ Zdbg) {
   constexpr int S = 256 / N2;
   constexpr int SLOT_COLS = 2 * N2;
-  griddep_launch_dependents();                   // a GEMM launched behind this kernel may set itself up
   const RqPairLayout L = rq_pair_layout(n1, N2);
   const int n = n1 * N2;
 
@@ -139,6 +138,9 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
     for (int o = 0; o < L.b2_bytes; o += 16384)
       bulk_load_1d(b2s + o, b2g + o, static_cast<uint32_t>(min(16384, L.b2_bytes - o)), img_full);
     griddep_wait();
+    // only now may a GEMM launched behind this kernel start (it requests its weights before it waits for
+    // this kernel, and this kernel's predecessor may have been writing them)
+    griddep_launch_dependents();
     for (long long i = 0; i < preload; ++i) load_token(i);
   }
   if (warp == 1) {

@@ -99,7 +99,6 @@ rotate_quant_st_kernel(const __grid_constant__ StLayout L, int n1, int rows, con
                        const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ StCoef<N2> cf) {
   constexpr int NS = kStSlots;
   constexpr int CH = 128 / N2;                    // tokens side by side in a slot's columns
-  griddep_launch_dependents();                    // a GEMM launched behind this kernel may set itself up
   const int n = n1 * N2;
   const int G = L.G, LS = L.LS;
 
@@ -169,9 +168,12 @@ rotate_quant_st_kernel(const __grid_constant__ StLayout L, int n1, int rows, con
     // X may come from the kernel before this one in the stream, which may also still read the buffers
     // this kernel writes: its completion is awaited before the first tokens are requested (every store
     // of this kernel depends on tokens having landed; the image above belongs to the handle).
-    if (lane < preload) {
+    if (lane < preload || lane == 0) {
       griddep_wait();
-      load_sg(lane);
+      // only now may a GEMM launched behind this kernel start (it requests its weights before it waits
+      // for this kernel, and this kernel's predecessor may have been writing them)
+      if (lane == 0) griddep_launch_dependents();
+      if (lane < preload) load_sg(lane);
     }
   }
   if (warp == 1) {

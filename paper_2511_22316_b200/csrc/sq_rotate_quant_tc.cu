@@ -190,6 +190,9 @@ __device__ __forceinline__ void rotate_quant_tc_body(const CUtensorMap& tmap_x, 
     for (int o = 0; o < L.b2_bytes; o += 16384)
       bulk_load_1d(b2s + o, b2_img + o, static_cast<uint32_t>(min(16384, L.b2_bytes - o)), img_full);
     griddep_wait();
+    // Only now may a GEMM launched behind this kernel start: it requests its weights before it waits for
+    // this kernel, and whatever precedes this kernel (sq_pack_weight, say) may have been writing them.
+    griddep_launch_dependents();
     for (int i = 0; i < preload; ++i) load_group(i);
     for (int b = 0; b < 4; ++b) {
       mbar_init(&x_empty[b], 1);
@@ -420,7 +423,6 @@ __global__ void __launch_bounds__((2 + 4 * S) * 32, (S * 2 * N2 <= 256) ? 2 : 1)
 rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ RqLayout L,
                        const unsigned char* __restrict__ a1_img, const unsigned char* __restrict__ b2_img, int n1,
                        int rows, uint8_t* __restrict__ Xq, __half* __restrict__ scales, float* __restrict__ Zdbg) {
-  griddep_launch_dependents();                   // a GEMM launched behind this kernel may set itself up
   rotate_quant_tc_body<N2, S>(tmap_x, L, a1_img, b2_img, n1, rows, Xq, scales, Zdbg, static_cast<int>(blockIdx.x),
                               static_cast<int>(gridDim.x));
 }
