@@ -8,7 +8,7 @@
 //
 // Warp roles per CTA: warp 0 = TMA producer; warp 1 = MMA issuer in the leader CTA and a relay in
 // the other (it tells the leader when its half of a tile has landed); then one group of four
-// warps per accumulator slot.  The per-token absmax spans both CTAs: each group reduces its 128
+// warps per accumulator slot (eight, two per lane quarter, when n2 = 128).  The per-token absmax spans both CTAs: each group reduces its 128
 // lanes and swaps the result with its partner group through the other CTA's shared memory.
 #include <cuda.h>
 #include <cuda_fp16.h>
@@ -50,11 +50,12 @@ __host__ __device__ inline RqPairLayout rq_pair_layout(int n1, int n2) {
   L.off_a1 = 0;
   L.off_b2 = L.a1_bytes;
   L.off_x = L.off_b2 + L.b2_bytes;
-  const int room = kMaxDynSmem - 1024 - 1024 - L.off_x;
+  const int extra = (n2 == 128) ? 2048 : 0;       // per-lane absmax swap of the eight-warp slot form
+  const int room = kMaxDynSmem - 1024 - 1024 - extra - L.off_x;
   const int xs = room / L.x_tile;
   L.XS = xs > 4 ? 4 : xs;
   L.off_misc = L.off_x + L.XS * L.x_tile;
-  L.total = L.off_misc + 1024;
+  L.total = L.off_misc + 1024 + extra;
   return L;
 }
 
@@ -70,8 +71,8 @@ __device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t sb
   return d;
 }
 
-template <int N2>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((2 + 4 * (256 / N2)) * 32, 1)
+template <int N2, int CW>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((2 + 4 * CW * (256 / N2)) * 32, 1)
 rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigned char* __restrict__ a1_img,
                          const unsigned char* __restrict__ b2_img, int n1, long long rows,
                          uint8_t* __restrict__ Xq, __half* __restrict__ scales, float* __restrict__ Zdbg) {
@@ -120,7 +121,7 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
       mbar_init(&x_empty[b], 1);
       mbar_init(&xp_full[b], 1);
       mbar_init(&d1_full[b], 1);
-      mbar_init(&a2_ready[b], 8);
+      mbar_init(&a2_ready[b], 8 * CW);
       mbar_init(&d2_full[b], 1);
       mbar_init(&amax_bar[b], 1);
     }
@@ -228,6 +229,127 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
           ok = false;
         }
       }
+    }
+  } else if (CW == 2) {
+    // ------------------------------ compute groups, two warps per lane quarter ---------------------
+    // Eight warps per accumulator slot: warp (quarter, cp) owns columns [cp * N2/2, (cp+1) * N2/2) of its
+    // lane quarter, 16 at a time; the lane's scale is the larger of the two halves' (swapped through
+    // shared memory behind the group barrier, which also orders the reads of D1 before its overwrite).
+    constexpr int HC = N2 / 2;
+    const int gi = (warp - 2) >> 2;
+    const int w = gi >> 1, cp = gi & 1;
+    const int quarter = warp & 3;
+    const int lane_g = quarter * 32 + lane;
+    const int pp = static_cast<int>(rank) * 128 + lane_g;
+    const uint32_t lane_addr = static_cast<uint32_t>(quarter * 32) << 16;
+    const uint32_t d1 = tmem_base + w * SLOT_COLS + lane_addr + cp * HC, d2 = d1 + N2;
+    const bool live = pp < n1;
+    float* lane_m = reinterpret_cast<float*>(smem + L.off_misc + 1024);       // [S][2][128 lanes]
+    bool ok = true;
+    for (long long i = w; i < my_tokens && ok; i += S) {
+      const long long token = pair + i * npairs;
+      const uint32_t ph = (i / S) & 1;
+      ok = mbar_wait(&d1_full[w], ph, RQP_D1_FULL, limit);
+      if (!ok) break;
+      tc_fence_after_sync();
+      float m = 0.0f;
+#pragma unroll
+      for (int c = 0; c < HC / 16; ++c) {
+        uint32_t r[16];
+        tmem_ld_32x32b_x16(d1 + 16 * c, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 16; e += 2)
+          m = fmaxf(m, fmaxf(fabsf(__uint_as_float(r[e])), fabsf(__uint_as_float(r[e + 1]))));
+      }
+      lane_m[(w * 2 + cp) * 128 + lane_g] = m;
+      named_barrier(1 + w, 256);
+      m = fmaxf(m, lane_m[(w * 2 + (cp ^ 1)) * 128 + lane_g]);
+      int ebits = static_cast<int>((__float_as_uint(m) >> 23) & 0xFF);
+      int k = 13 - (ebits - 127);
+      if (m == 0.0f) k = 0;
+      k = max(-126, min(127, k));
+      const float sc = __uint_as_float(static_cast<uint32_t>(k + 127) << 23);
+      const int uexp = -(k + 2 * kFactorScaleLog2) + 127;
+      const float un = (uexp >= 1) ? __uint_as_float(static_cast<uint32_t>(min(uexp, 254)) << 23) : 0.0f;
+#pragma unroll
+      for (int c = 0; c < HC / 16; ++c) {
+        uint32_t r[16], o[16];
+        tmem_ld_32x32b_x16(d1 + 16 * c, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 8; ++e) {
+          const float v0 = __uint_as_float(r[2 * e]), v1 = __uint_as_float(r[2 * e + 1]);
+          const __half2 hh = __floats2half2_rn(v0 * sc, v1 * sc);
+          const float2 hf = __half22float2(hh);
+          o[e] = *reinterpret_cast<const uint32_t*>(&hh);
+          o[8 + e] = pack_half2(fmaf(v0, sc, -hf.x), fmaf(v1, sc, -hf.y));
+        }
+        tmem_st_32x32b_x16(d1 + 16 * c, o);
+      }
+      tmem_wait_st();
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive_cluster(&a2_ready[w], 0);
+
+      ok = mbar_wait(&d2_full[w], ph, RQP_D2_FULL, limit);
+      if (!ok) break;
+      tc_fence_after_sync();
+      float zm = 0.0f;
+#pragma unroll
+      for (int c = 0; c < HC / 16; ++c) {
+        uint32_t r[16];
+        tmem_ld_32x32b_x16(d2 + 16 * c, r);
+        tmem_wait_ld();
+#pragma unroll
+        for (int e = 0; e < 16; e += 2)
+          zm = fmaxf(zm, fmaxf(fabsf(__uint_as_float(r[e])), fabsf(__uint_as_float(r[e + 1]))));
+      }
+      zm *= un;
+#pragma unroll
+      for (int o = 16; o > 0; o >>= 1) zm = fmaxf(zm, __shfl_xor_sync(0xffffffffu, zm, o));
+      float* amax_w = amax_x + (w * 2 + ph) * 8;
+      if (lane == 0) amax_w[quarter * 2 + cp] = zm;
+      named_barrier(1 + w, 256);
+      float amax = fmaxf(fmaxf(fmaxf(amax_w[0], amax_w[1]), fmaxf(amax_w[2], amax_w[3])),
+                         fmaxf(fmaxf(amax_w[4], amax_w[5]), fmaxf(amax_w[6], amax_w[7])));
+      if (lane_g == 0 && cp == 0) st_f32_peer_and_arrive(&amax_peer[w * 2 + ph], amax, &amax_bar[w], rank ^ 1u);
+      ok = mbar_wait_acq_cluster(&amax_bar[w], ph, RQP_AMAX, limit);
+      if (!ok) break;
+      amax = fmaxf(amax, amax_peer[w * 2 + ph]);
+      __half delta;
+      float inv;
+      row_scale(amax, delta, inv);
+      const float inv_un = inv * un;
+      const bool clamp = __half2float(delta) < 6.103515625e-05f;
+      uint8_t* orow = Xq + token * (n / 2) + static_cast<long long>(pp) * (N2 / 2) + cp * (HC / 2);
+      float* zrow = (Zdbg != nullptr && live) ? Zdbg + token * n + static_cast<long long>(pp) * N2 + cp * HC : nullptr;
+#pragma unroll
+      for (int c = 0; c < HC / 16; ++c) {
+        uint32_t r[16];
+        tmem_ld_32x32b_x16(d2 + 16 * c, r);
+        tmem_wait_ld();
+        float t[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          t[e] = __fadd_rn(__fmul_rn(__uint_as_float(r[e]), inv_un), 0.5f);
+          if (clamp) t[e] = fminf(fmaxf(t[e], -8.0f), 7.5f);
+        }
+        uint2 pk;
+        pk.x = pack8_codes(t);
+        pk.y = pack8_codes(t + 8);
+        if (live) {
+          *reinterpret_cast<uint2*>(orow + 8 * c) = pk;
+          if (zrow) {
+#pragma unroll
+            for (int e = 0; e < 16; e += 4)
+              *reinterpret_cast<float4*>(zrow + 16 * c + e) =
+                  make_float4(__uint_as_float(r[e]) * un, __uint_as_float(r[e + 1]) * un,
+                              __uint_as_float(r[e + 2]) * un, __uint_as_float(r[e + 3]) * un);
+          }
+        }
+      }
+      if (pp == 0 && cp == 0) scales[token] = delta;
     }
   } else {
     // ------------------------------ compute groups ------------------------------------------------
@@ -421,15 +543,16 @@ sq_status_t launch_rotate_quant_pair(const sq_rotation* h, const void* X, int64_
   const unsigned char* a1 = static_cast<const unsigned char*>(h->dA1img);
   const unsigned char* b2 = static_cast<const unsigned char*>(h->dB2img);
   if (n2 == 64) {
-    auto kern = rotate_quant_pair_kernel<64>;
+    auto kern = rotate_quant_pair_kernel<64, 1>;
     if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return SQ_ERR_CUDA;
     if (launch_dependent(kern, dim3(grid), dim3((2 + 4 * 4) * 32), static_cast<size_t>(smem), s, mx, a1, b2, n1, rows,
                          static_cast<uint8_t*>(Xq), static_cast<__half*>(scales), Zdbg) != cudaSuccess)
       return SQ_ERR_CUDA;
   } else {
-    auto kern = rotate_quant_pair_kernel<128>;
+    // two slots of eight warps (18 warps in the CTA instead of 10)
+    auto kern = rotate_quant_pair_kernel<128, 2>;
     if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return SQ_ERR_CUDA;
-    if (launch_dependent(kern, dim3(grid), dim3((2 + 4 * 2) * 32), static_cast<size_t>(smem), s, mx, a1, b2, n1, rows,
+    if (launch_dependent(kern, dim3(grid), dim3((2 + 4 * 2 * 2) * 32), static_cast<size_t>(smem), s, mx, a1, b2, n1, rows,
                          static_cast<uint8_t*>(Xq), static_cast<__half*>(scales), Zdbg) != cudaSuccess)
       return SQ_ERR_CUDA;
   }
