@@ -18,7 +18,8 @@ Conventions (paper, Section "SingleQuant", paragraph "Kronecker Product"):
   * V (R1 (x) R2) = rvec(R1^T V_mat R2)                                   (Eq. "eq18").
 
 Parity status: every function below is pinned by tests/test_oracle_*.py against closed forms,
-brute force or library routines.  Agreement with the authors' own R1, R2 (which depend on
+brute force or library routines (the weight-only variant and the grouped layer at the end of the
+file by tests/test_oracle_weight_only.py).  Agreement with the authors' own R1, R2 (which depend on
 choices the paper leaves open: the calibration vector, the random block O, the order of the
 Givens chain) is "parity unpinned": no code, weights or data of theirs is available.
 """
@@ -453,3 +454,118 @@ def linear_fp(X: np.ndarray, W: np.ndarray) -> np.ndarray:
 def kron_dense(R1: np.ndarray, R2: np.ndarray) -> np.ndarray:
     """The explicit n x n matrix R1 (x) R2 (small sizes only; used by the pins)."""
     return np.kron(np.asarray(R1, dtype=np.float64), np.asarray(R2, dtype=np.float64))
+
+
+# --------------------------------------------------------------------------------------
+# Weight-only variant (Appendix "Weight-only Quantization", Table "wquant": W4A16 / W3A16) and the
+# grouped form of the layer for mixture-of-experts blocks (Section "Results on Mixtral Models")
+#
+# The paper gives the setting only: the same rotation, weights quantised to 4 or 3 bits with one
+# step per output channel, activations left in 16 bits.  Readings taken here: the activations are
+# rotated online exactly as in the W4A4 path and rounded once to fp16; a b-bit code is the W4A4
+# quantiser with 7 replaced by 2^(b-1) - 1 and the clamp by [-2^(b-1), 2^(b-1) - 1]; the product
+# is the plain real-valued one with a single rounding of the result to fp16.
+# --------------------------------------------------------------------------------------
+def quantize_rows_bits(Z: np.ndarray, bits: int, decision: str = "f64") -> Tuple[np.ndarray, np.ndarray]:
+    """Q_Delta of Section 3.2 with b bits: Delta_t = fp16(max_c |Z_tc| / (2^(b-1) - 1)), code =
+    floor(z / Delta + 1/2) clamped to [-2^(b-1), 2^(b-1) - 1]; an all-zero row has Delta = 0 and
+    codes 0.  `decision` as in quantize_rows.  Returns (codes int8, Delta fp16)."""
+    if bits < 2 or bits > 8:
+        raise ValueError("bits")
+    qmax = 2 ** (bits - 1) - 1
+    qmin = -(2 ** (bits - 1))
+    ft = {"f64": np.float64, "f32": np.float32}[decision]
+    Z = np.asarray(Z, dtype=ft)
+    T = Z.shape[0]
+    codes = np.zeros(Z.shape, dtype=np.int8)
+    delta = np.zeros(T, dtype=np.float16)
+    for t in range(T):
+        amax = ft(np.max(np.abs(Z[t]))) if Z.shape[1] else ft(0)
+        delta[t] = np.float16(ft(amax / ft(qmax)))
+        d = ft(delta[t])
+        if d > 0:
+            if decision == "f64":
+                q = np.floor(Z[t] / d + 0.5)
+            else:
+                inv = ft(ft(1.0) / d)
+                q = np.floor(((Z[t] * inv).astype(ft) + ft(0.5)).astype(ft))
+            codes[t] = np.clip(q, qmin, qmax).astype(np.int8)
+    return codes, delta
+
+
+# Storage order of the weight-only format: nibble position i (bits 4i .. 4i+3 of a little-endian
+# 32-bit word) holds channel WO_ORDER[i] of the word's eight consecutive channels, so that
+# (word >> 4s) & 0x000F000F is the pair (channel 2s, channel 2s + 1) in the two 16-bit halves.
+WO_ORDER = (0, 2, 4, 6, 1, 3, 5, 7)
+
+
+def pack_int4_interleaved(codes: np.ndarray) -> np.ndarray:
+    """Two's-complement nibbles in the weight-only storage order (see WO_ORDER); K % 8 == 0."""
+    codes = np.asarray(codes, dtype=np.int8)
+    K = codes.shape[-1]
+    assert K % 8 == 0
+    u = (codes.astype(np.uint8) & np.uint8(0x0F)).reshape(codes.shape[:-1] + (K // 8, 8))
+    out = np.zeros(codes.shape[:-1] + (K // 8, 4), dtype=np.uint8)
+    for pos in range(8):
+        nib = u[..., WO_ORDER[pos]]
+        out[..., pos // 2] |= (nib << np.uint8(4 * (pos % 2))).astype(np.uint8)
+    return out.reshape(codes.shape[:-1] + (K // 2,))
+
+
+def unpack_int4_interleaved(packed: np.ndarray) -> np.ndarray:
+    """Inverse of pack_int4_interleaved: sign-extended int8 codes in channel order."""
+    packed = np.asarray(packed, dtype=np.uint8)
+    Kb = packed.shape[-1]
+    assert Kb % 4 == 0
+    b = packed.reshape(packed.shape[:-1] + (Kb // 4, 4))
+    out = np.zeros(packed.shape[:-1] + (Kb // 4, 8), dtype=np.int8)
+    for pos in range(8):
+        nib = ((b[..., pos // 2] >> np.uint8(4 * (pos % 2))) & np.uint8(0x0F)).astype(np.int16)
+        out[..., WO_ORDER[pos]] = np.where(nib >= 8, nib - 16, nib).astype(np.int8)
+    return out.reshape(packed.shape[:-1] + (Kb * 2,))
+
+
+def rotate_f16(X: np.ndarray, R1: Optional[np.ndarray], R2: Optional[np.ndarray]) -> np.ndarray:
+    """The rotated activations of the weight-only path: Eq. "eq18" in float64, one rounding to fp16."""
+    Z = np.asarray(X, dtype=np.float64) if R1 is None else rotate(X, R1, R2)
+    return Z.astype(np.float16)
+
+
+def pack_weight_wo(W: np.ndarray, R1, R2, bits: int, decision: str = "f64"):
+    """Offline weight path of the weight-only variant: rotate the rows of W, b-bit codes with one
+    step per output channel, stored in the weight-only order.  Returns (packed uint8 [C x n/2],
+    Delta fp16 [C], rotated rows float64)."""
+    Z = np.asarray(W, dtype=np.float64) if R1 is None else rotate(W, R1, R2)
+    codes, delta = quantize_rows_bits(Z, bits, decision)
+    return pack_int4_interleaved(codes), delta, Z
+
+
+def gemm_w4a16(Z16: np.ndarray, codes: np.ndarray, sw: np.ndarray) -> np.ndarray:
+    """Y[t, c] = fp16((sum_k Z16[t, k] * code[c, k]) * s_w[c]): the real-valued product in float64
+    with one final rounding."""
+    acc = np.asarray(Z16, dtype=np.float64) @ np.asarray(codes, dtype=np.float64).T
+    return (acc * np.asarray(sw, dtype=np.float64)[None, :]).astype(np.float16)
+
+
+def linear_wo(X: np.ndarray, W: np.ndarray, R1, R2, bits: int, decision: str = "f64") -> np.ndarray:
+    """The weight-only layer: fp16 rotated activations against b-bit pre-rotated weights."""
+    Wq, sw, _ = pack_weight_wo(W, R1, R2, bits, decision)
+    return gemm_w4a16(rotate_f16(X, R1, R2), unpack_int4_interleaved(Wq), sw)
+
+
+def linear_grouped(X: np.ndarray, offsets, Ws, rotations, decision: str = "f64") -> np.ndarray:
+    """The W4A4 layer of a mixture-of-experts block: the tokens are sorted by expert, expert e owns
+    rows offsets[e] .. offsets[e+1]-1 of X and has its own weights Ws[e] [C x n] and its own factor
+    pair rotations[e] = (R1, R2); every expert's rows go through `linear` with that expert's
+    matrices.  Returns Y [T x C]."""
+    X = np.asarray(X)
+    E = len(Ws)
+    assert len(offsets) == E + 1 and offsets[0] == 0 and offsets[-1] == X.shape[0]
+    C = Ws[0].shape[0]
+    Y = np.zeros((X.shape[0], C), dtype=np.float16)
+    for e in range(E):
+        a, b = int(offsets[e]), int(offsets[e + 1])
+        assert a <= b
+        if b > a:
+            Y[a:b] = linear(X[a:b], Ws[e], rotations[e][0], rotations[e][1], decision)
+    return Y
