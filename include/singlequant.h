@@ -197,6 +197,70 @@ sq_status_t sq_linear_host(const sq_rotation_t* rot, const void* X_host, int64_t
                            const void* Wq, const void* sw, int64_t N, int64_t K,
                            void* workspace, size_t workspace_bytes, void* Y_host, void* stream);
 
+/* ---------------------------------------------------------------------------------------------
+ * Weight-only variant (Appendix "Weight-only Quantization", Table "wquant": W4A16 and W3A16): the
+ * same rotation, weights quantised to b = 4 or 3 bits with one step per output channel, activations
+ * left in 16 bits.  The paper states the setting only; taken here: the activations are rotated
+ * online as in the W4A4 path and rounded once to fp16; a b-bit code is the W4A4 quantiser with 7
+ * replaced by 2^(b-1) - 1 and the clamp by [-2^(b-1), 2^(b-1) - 1]; the product is accumulated in
+ * fp32 and rounded once to fp16.
+ *
+ * Storage of the codes ("weight-only order"): one two's-complement nibble per code, for 3 bits too
+ * (the codes then lie in [-4, 3]; the 25 % a 3-bit packing would save is not taken).  Within every
+ * eight consecutive channels, read as a little-endian 32-bit word, nibble position i (bits 4i..4i+3)
+ * holds channel (0, 2, 4, 6, 1, 3, 5, 7)[i]: (word >> 4s) & 0x000F000F is then the pair of channels
+ * (2s, 2s+1) in the two 16-bit halves, which is what the kernel widens to a half2.  This differs from
+ * the channel order sq_pack_weight writes for the W4A4 path; the two formats are not interchangeable.
+ * ------------------------------------------------------------------------------------------- */
+
+/* Offline: rotate the rows of W, quantise to `bits` (4 or 3; else SQ_ERR_INVALID_ARG), store in the
+ * weight-only order.  K % 8 == 0 (SQ_ERR_SHAPE otherwise).
+ *   rot_or_null   NULL = identity rotation
+ *   W             DEVICE fp16 [N x K], K == n of the handle
+ *   Wq            DEVICE uint8 [N x K/2]   (out)
+ *   sw            DEVICE fp16 [N]          (out; Delta_c = fp16(max|row| / (2^(bits-1) - 1))) */
+sq_status_t sq_pack_weight_wo(const sq_rotation_t* rot_or_null, const void* W, int64_t N, int64_t K,
+                              int32_t bits, void* Wq, void* sw, void* stream);
+
+/* Step 1 alone: Z16_t = fp16(R1^T X~_t R2), the rotation accurate to fp32 on chip, one rounding.
+ *   X    DEVICE fp16 [M x n]        Z16  DEVICE fp16 [M x n] (out; may not alias X)
+ * Supported sizes as sq_rotate_quant_act. */
+sq_status_t sq_rotate_act_f16(const sq_rotation_t* rot, const void* X, int64_t M, void* Z16, void* stream);
+
+/* Step 3 of the variant: Y[t,c] = fp16((sum_k Z16[t,k] * code[c,k]) * sw[c]), fp32 accumulation.
+ *   Z16 DEVICE fp16 [M x K]      Wq DEVICE uint8 [N x K/2] (weight-only order)     sw DEVICE fp16 [N]
+ *   Y   DEVICE fp16 [M x N] (out)
+ * K % 8 == 0, K <= 65536.  The tensor-core path needs K % 64 == 0 and N % 8 == 0; other shapes run a
+ * plain fp32 kernel (same definition, another summation order). */
+sq_status_t sq_w4a16_gemm(const void* Z16, const void* Wq, const void* sw, int64_t M, int64_t N, int64_t K,
+                          void* Y, void* stream);
+
+/* The weight-only layer on one stream: rotation into the workspace (Z16), then the product.
+ *   workspace  DEVICE, at least sq_linear_wo_workspace_bytes(M, K) bytes, 256-byte aligned
+ * Every argument of both halves is validated before the first kernel is queued. */
+size_t sq_linear_wo_workspace_bytes(int64_t M, int64_t K);
+sq_status_t sq_linear_wo(const sq_rotation_t* rot, const void* X, int64_t M, const void* Wq, const void* sw,
+                         int64_t N, int64_t K, void* workspace, size_t workspace_bytes, void* Y, void* stream);
+
+/* The W4A4 layer of a mixture-of-experts block (Section "Results on Mixtral Models": the method is
+ * applied to each expert's linear layers).  The tokens are sorted by expert: expert e owns rows
+ * offsets[e] .. offsets[e+1]-1 of X and of Y and has its own packed weights and its own rotation
+ * handle (experts that share an input distribution may share a handle).  Each expert's rows go
+ * through the same kernels as sq_linear, queued back to back on `stream`; experts without tokens
+ * cost nothing.
+ *   rots          HOST array of E handles (all with n1*n2 == K)
+ *   offsets       HOST array of E+1 non-decreasing row offsets, offsets[0] == 0, offsets[E] == M
+ *   X             DEVICE fp16 [M x K]
+ *   Wq, sw        HOST arrays of E DEVICE pointers: uint8 [N x K/2] and fp16 [N] per expert
+ *   workspace     DEVICE, at least sq_linear_workspace_bytes(M, K) bytes, 256-byte aligned (shared by
+ *                 the experts, which run one after the other)
+ *   Y             DEVICE fp16 [M x N] (out)
+ * Every expert's slice must start on a 16-byte boundary (K % 8 == 0 and N % 8 == 0 make every offset
+ * valid; otherwise SQ_ERR_ALIGN).  All arguments are validated before the first kernel is queued. */
+sq_status_t sq_linear_grouped(const sq_rotation_t* const* rots, int32_t E, const int64_t* offsets,
+                              const void* X, const void* const* Wq, const void* const* sw, int64_t N, int64_t K,
+                              void* workspace, size_t workspace_bytes, void* Y, void* stream);
+
 /* Synchronises `stream`, then returns and clears the device status word: SQ_OK, or
  * SQ_ERR_TIMEOUT if any kernel since the last call gave up a bounded wait, or SQ_ERR_CUDA. */
 sq_status_t sq_last_device_status(void* stream);

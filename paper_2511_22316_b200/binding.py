@@ -30,6 +30,8 @@ EXPORTS = (
     "sq_w4a4_gemm", "sq_linear_workspace_bytes", "sq_linear",
     "sq_linear_static", "sq_linear_host_workspace_bytes", "sq_linear_host", "sq_last_device_status",
     "sq_debug_bounded_wait", "sq_kernel_launch_count", "sq_status_string",
+    "sq_pack_weight_wo", "sq_rotate_act_f16", "sq_w4a16_gemm", "sq_linear_wo_workspace_bytes", "sq_linear_wo",
+    "sq_linear_grouped",
 )
 
 
@@ -75,6 +77,15 @@ def load() -> ctypes.CDLL:
     lib.sq_linear_host_workspace_bytes.restype = c_size_t
     lib.sq_linear_host.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_int64,
                                    c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.sq_pack_weight_wo.argtypes = [c_void_p, c_void_p, c_int64, c_int64, c_int32, c_void_p, c_void_p, c_void_p]
+    lib.sq_rotate_act_f16.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p]
+    lib.sq_w4a16_gemm.argtypes = [c_void_p, c_void_p, c_void_p, c_int64, c_int64, c_int64, c_void_p, c_void_p]
+    lib.sq_linear_wo_workspace_bytes.argtypes = [c_int64, c_int64]
+    lib.sq_linear_wo_workspace_bytes.restype = c_size_t
+    lib.sq_linear_wo.argtypes = [c_void_p, c_void_p, c_int64, c_void_p, c_void_p, c_int64, c_int64,
+                                 c_void_p, c_size_t, c_void_p, c_void_p]
+    lib.sq_linear_grouped.argtypes = [POINTER(c_void_p), c_int32, POINTER(c_int64), c_void_p, POINTER(c_void_p),
+                                      POINTER(c_void_p), c_int64, c_int64, c_void_p, c_size_t, c_void_p, c_void_p]
     lib.sq_last_device_status.argtypes = [c_void_p]
     lib.sq_debug_bounded_wait.argtypes = [c_uint32, c_void_p]
     lib.sq_kernel_launch_count.argtypes = []
@@ -245,6 +256,43 @@ def sq_linear_host(rot: Rotation, X_host, M: int, Wq, sw, N: int, K: int, worksp
                    Y_host, stream=None) -> None:
     _check(load().sq_linear_host(rot.handle, _ptr(X_host), M, _ptr(Wq), _ptr(sw), N, K, _ptr(workspace),
                                  workspace_bytes, _ptr(Y_host), _stream(stream)), "sq_linear_host")
+
+
+def sq_pack_weight_wo(rot: Optional[Rotation], W, N: int, K: int, bits: int, Wq, sw, stream=None) -> None:
+    """Offline weight path of the weight-only variant: `bits` = 4 or 3, codes in the weight-only order."""
+    _check(load().sq_pack_weight_wo(None if rot is None else rot.handle, _ptr(W), N, K, int(bits), _ptr(Wq),
+                                    _ptr(sw), _stream(stream)), "sq_pack_weight_wo")
+
+
+def sq_rotate_act_f16(rot: Rotation, X, M: int, Z16, stream=None) -> None:
+    _check(load().sq_rotate_act_f16(rot.handle, _ptr(X), M, _ptr(Z16), _stream(stream)), "sq_rotate_act_f16")
+
+
+def sq_w4a16_gemm(Z16, Wq, sw, M: int, N: int, K: int, Y, stream=None) -> None:
+    _check(load().sq_w4a16_gemm(_ptr(Z16), _ptr(Wq), _ptr(sw), M, N, K, _ptr(Y), _stream(stream)), "sq_w4a16_gemm")
+
+
+def sq_linear_wo_workspace_bytes(M: int, K: int) -> int:
+    return int(load().sq_linear_wo_workspace_bytes(M, K))
+
+
+def sq_linear_wo(rot: Rotation, X, M: int, Wq, sw, N: int, K: int, workspace, workspace_bytes: int, Y,
+                 stream=None) -> None:
+    _check(load().sq_linear_wo(rot.handle, _ptr(X), M, _ptr(Wq), _ptr(sw), N, K, _ptr(workspace), workspace_bytes,
+                               _ptr(Y), _stream(stream)), "sq_linear_wo")
+
+
+def sq_linear_grouped(rots, offsets, X, Wq, sw, N: int, K: int, workspace, workspace_bytes: int, Y,
+                      stream=None) -> None:
+    """The W4A4 layer of a mixture-of-experts block: `rots`, `Wq`, `sw` are sequences with one entry per
+    expert, `offsets` the E + 1 row offsets of the expert-sorted tokens."""
+    E = len(rots)
+    h = (c_void_p * E)(*[r.handle for r in rots])
+    off = (c_int64 * (E + 1))(*[int(o) for o in offsets])
+    wq = (c_void_p * E)(*[_ptr(w) for w in Wq])
+    sws = (c_void_p * E)(*[_ptr(w) for w in sw])
+    _check(load().sq_linear_grouped(h, E, off, _ptr(X), wq, sws, N, K, _ptr(workspace), workspace_bytes, _ptr(Y),
+                                    _stream(stream)), "sq_linear_grouped")
 
 
 def sq_last_device_status(stream=None) -> int:

@@ -12,7 +12,7 @@ PKG = os.path.dirname(os.path.abspath(__file__))
 CSRC = os.path.join(PKG, "csrc")
 LIB = os.path.join(PKG, "libsinglequant.so")
 SOURCES = ["sq_all.cu"]
-DEPS = ["sq_all.cu", "sq_gemm.cu", "sq_gemm_pair.cu", "sq_gemm_decode.cu", "sq_gemv.cu", "sq_rotate_quant.cu", "sq_rotate_quant_tc.cu", "sq_rotate_quant_st.cu", "sq_linear_fused.cu", "sq_rotate_quant_pair.cu", "sq_rotation_host.cu", "sq_api.cu", "sq_noalloc.cu",
+DEPS = ["sq_all.cu", "sq_gemm.cu", "sq_gemm_pair.cu", "sq_gemm_decode.cu", "sq_gemv.cu", "sq_gemm_wo.cu", "sq_rotate_quant.cu", "sq_rotate_quant_tc.cu", "sq_rotate_quant_st.cu", "sq_linear_fused.cu", "sq_rotate_quant_pair.cu", "sq_rotation_host.cu", "sq_api.cu", "sq_noalloc.cu",
         "sq_ptx.cuh", "sq_internal.h", os.path.join("..", "..", "include", "singlequant.h")]
 
 

@@ -81,6 +81,12 @@ sq_status_t rotate_quant_dispatch(const sq_rotation* h, const void* X, int64_t r
   if (h->tc_pair) return launch_rotate_quant_pair(h, X, rows, Xq, scales, Zdbg, s);
   return launch_rotate_quant(h->dR1, h->dR2, h->n1, h->n2, X, rows, Xq, scales, Zdbg, s);
 }
+// Step 1 alone, fp16 rows out (weight-only variant): the same kernels in their rotation-only form.
+sq_status_t rotate_f16_dispatch(const sq_rotation* h, const void* X, int64_t rows, void* Z16, cudaStream_t s) {
+  if (h->tc_ready) return launch_rotate_quant_tc(h, X, rows, Z16, nullptr, nullptr, s, true);
+  if (h->tc_pair) return launch_rotate_quant_pair(h, X, rows, Z16, nullptr, nullptr, s, true);
+  return launch_rotate_quant(h->dR1, h->dR2, h->n1, h->n2, X, rows, Z16, nullptr, nullptr, s, 0);
+}
 }  // namespace sq
 
 namespace {
@@ -429,6 +435,133 @@ sq_status_t sq_linear_host(const sq_rotation_t* rot, const void* X_host, int64_t
                       cudaStreamSynchronize(p->d2h) == cudaSuccess;
   if (st != SQ_OK) return st;
   return synced ? SQ_OK : SQ_ERR_CUDA;
+}
+
+// ---------------------------------------------------------------------------------------------
+// Weight-only variant and the grouped layer
+// ---------------------------------------------------------------------------------------------
+sq_status_t sq_pack_weight_wo(const sq_rotation_t* rot_or_null, const void* W, int64_t N, int64_t K, int32_t bits,
+                              void* Wq, void* sw, void* stream) {
+  if (bits != 3 && bits != 4) return SQ_ERR_INVALID_ARG;
+  if (rot_or_null) {
+    if (static_cast<int64_t>(rot_or_null->n1) * rot_or_null->n2 != K) return SQ_ERR_SHAPE;
+    if (rot_or_null->n2 & 1) return SQ_ERR_SHAPE;
+  }
+  if (K % 8 != 0) return SQ_ERR_SHAPE;
+  sq_status_t st = check_rows_args(W, Wq, sw, nullptr, N, K);
+  if (st != SQ_OK || N == 0) return st;
+  if (rot_or_null && (st = check_handle_device(rot_or_null)) != SQ_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  const int qmax = (1 << (bits - 1)) - 1;
+  if (!rot_or_null)
+    st = sq::launch_rotate_quant(nullptr, nullptr, 1, static_cast<int>(K), W, N, Wq, sw, nullptr, s, qmax);
+  else if (bits == 4)
+    st = sq::rotate_quant_dispatch(rot_or_null, W, N, Wq, sw, nullptr, s);
+  else      // other widths: the fp32 kernel, which takes the number of levels as an argument (offline path)
+    st = sq::launch_rotate_quant(rot_or_null->dR1, rot_or_null->dR2, rot_or_null->n1, rot_or_null->n2, W, N, Wq, sw,
+                                 nullptr, s, qmax);
+  if (st != SQ_OK) return st;
+  return sq::launch_interleave_nibbles(Wq, N, K, s);
+}
+
+sq_status_t sq_rotate_act_f16(const sq_rotation_t* rot, const void* X, int64_t M, void* Z16, void* stream) {
+  if (!rot) return SQ_ERR_INVALID_ARG;
+  const int64_t n = static_cast<int64_t>(rot->n1) * rot->n2;
+  if (rot->n2 & 1) return SQ_ERR_SHAPE;
+  sq_status_t st = check_rows_args(X, Z16, Z16, nullptr, M, n);
+  if (st != SQ_OK || M == 0) return st;
+  if (X == Z16) return SQ_ERR_INVALID_ARG;
+  if ((st = check_handle_device(rot)) != SQ_OK) return st;
+  return sq::rotate_f16_dispatch(rot, X, M, Z16, static_cast<cudaStream_t>(stream));
+}
+
+namespace {
+sq_status_t check_wo_gemm_args(const void* Z16, const void* Wq, const void* sw, int64_t M, int64_t N, int64_t K,
+                               const void* Y) {
+  if (M < 0 || N < 0 || M > kMaxRows || N > kMaxRows) return SQ_ERR_INVALID_ARG;
+  if (K < 8 || (K % 8) != 0) return SQ_ERR_SHAPE;
+  if (K > kMaxK) return SQ_ERR_UNSUPPORTED;
+  if (M == 0 || N == 0) return SQ_OK;
+  if (!Z16 || !Wq || !sw || !Y) return SQ_ERR_INVALID_ARG;
+  if (!sq::aligned16(Z16) || !sq::aligned16(Wq) || !sq::aligned16(sw) || !sq::aligned16(Y)) return SQ_ERR_ALIGN;
+  return SQ_OK;
+}
+}  // namespace
+
+sq_status_t sq_w4a16_gemm(const void* Z16, const void* Wq, const void* sw, int64_t M, int64_t N, int64_t K, void* Y,
+                          void* stream) {
+  sq_status_t st = check_wo_gemm_args(Z16, Wq, sw, M, N, K, Y);
+  if (st != SQ_OK || M == 0 || N == 0) return st;
+  return sq::launch_wo_gemm(Z16, Wq, sw, M, N, K, Y, static_cast<cudaStream_t>(stream));
+}
+
+size_t sq_linear_wo_workspace_bytes(int64_t M, int64_t K) {
+  if (M <= 0 || K <= 0) return 0;
+  return align_up(static_cast<size_t>(M) * K * 2, 256);
+}
+
+sq_status_t sq_linear_wo(const sq_rotation_t* rot, const void* X, int64_t M, const void* Wq, const void* sw,
+                         int64_t N, int64_t K, void* workspace, size_t workspace_bytes, void* Y, void* stream) {
+  if (!rot) return SQ_ERR_INVALID_ARG;
+  if (static_cast<int64_t>(rot->n1) * rot->n2 != K) return SQ_ERR_SHAPE;
+  if (rot->n2 & 1) return SQ_ERR_SHAPE;
+  if (M < 0 || N < 0) return SQ_ERR_INVALID_ARG;
+  if (M == 0 || N == 0) return SQ_OK;
+  if (!workspace) return SQ_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQ_ERR_ALIGN;
+  if (workspace_bytes < sq_linear_wo_workspace_bytes(M, K)) return SQ_ERR_NOMEM;
+  void* Z16 = workspace;
+  sq_status_t st = check_rows_args(X, Z16, Z16, nullptr, M, K);
+  if (st != SQ_OK) return st;
+  if ((st = check_wo_gemm_args(Z16, Wq, sw, M, N, K, Y)) != SQ_OK) return st;
+  if ((st = check_handle_device(rot)) != SQ_OK) return st;
+  cudaStream_t s = static_cast<cudaStream_t>(stream);
+  st = sq::rotate_f16_dispatch(rot, X, M, Z16, s);
+  if (st != SQ_OK) return st;
+  sq::g_pdl_next = true;                  // the product may set itself up while the rotation drains
+  st = sq::launch_wo_gemm(Z16, Wq, sw, M, N, K, Y, s);
+  sq::g_pdl_next = false;
+  return st;
+}
+
+sq_status_t sq_linear_grouped(const sq_rotation_t* const* rots, int32_t E, const int64_t* offsets, const void* X,
+                              const void* const* Wq, const void* const* sw, int64_t N, int64_t K, void* workspace,
+                              size_t workspace_bytes, void* Y, void* stream) {
+  if (!rots || !offsets || !Wq || !sw || E < 1 || N < 0) return SQ_ERR_INVALID_ARG;
+  if (offsets[0] != 0) return SQ_ERR_INVALID_ARG;
+  for (int32_t e = 0; e < E; ++e)
+    if (offsets[e + 1] < offsets[e]) return SQ_ERR_INVALID_ARG;
+  const int64_t M = offsets[E];
+  if (M > kMaxRows) return SQ_ERR_INVALID_ARG;
+  if (M == 0 || N == 0) return SQ_OK;
+  if (!workspace || !X || !Y) return SQ_ERR_INVALID_ARG;
+  if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQ_ERR_ALIGN;
+  if (workspace_bytes < sq_linear_workspace_bytes(M, K)) return SQ_ERR_NOMEM;
+  const unsigned char* Xb = static_cast<const unsigned char*>(X);
+  unsigned char* Yb = static_cast<unsigned char*>(Y);
+  unsigned char* ws = static_cast<unsigned char*>(workspace);
+  // Everything any expert's call would refuse is refused here, before the first kernel is queued.
+  for (int32_t e = 0; e < E; ++e) {
+    const int64_t r0 = offsets[e], r = offsets[e + 1] - r0;
+    if (r == 0) continue;
+    const sq_rotation_t* rot = rots[e];
+    if (!rot) return SQ_ERR_INVALID_ARG;
+    if (static_cast<int64_t>(rot->n1) * rot->n2 != K || (rot->n2 & 1)) return SQ_ERR_SHAPE;
+    void* Xq = ws;
+    void* sx = ws + align_up(static_cast<size_t>(r) * (K / 2), 256);
+    sq_status_t st = check_rows_args(Xb + static_cast<size_t>(r0) * K * 2, Xq, sx, nullptr, r, K);
+    if (st == SQ_OK) st = check_gemm_args(Xq, sx, Wq[e], sw[e], r, N, K, Yb + static_cast<size_t>(r0) * N * 2, nullptr);
+    if (st == SQ_OK) st = check_handle_device(rot);
+    if (st != SQ_OK) return st;
+  }
+  for (int32_t e = 0; e < E; ++e) {
+    const int64_t r0 = offsets[e], r = offsets[e + 1] - r0;
+    if (r == 0) continue;
+    const sq_status_t st = sq_linear(rots[e], Xb + static_cast<size_t>(r0) * K * 2, r, Wq[e], sw[e], N, K, workspace,
+                                     workspace_bytes, Yb + static_cast<size_t>(r0) * N * 2, stream);
+    if (st != SQ_OK) return st;
+  }
+  return SQ_OK;
 }
 
 sq_status_t sq_last_device_status(void* stream) {

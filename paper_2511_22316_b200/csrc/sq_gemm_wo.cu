@@ -1,0 +1,377 @@
+// Weight-only variant of step 3 (Appendix "Weight-only Quantization", Table "wquant": W4A16 / W3A16):
+//   Y[t, c] = fp16((sum_k Z16[t, k] * code[c, k]) * s_w[c])
+// with the rotated activations Z16 in fp16, the pre-rotated weights as b-bit two's-complement codes
+// (b = 4 or 3, one nibble each) and fp32 accumulation.
+//
+// Tensor-core kernel (sm_100a): the activation tile is the A operand exactly as TMA delivers it (128
+// tokens x 64 channels, 128-byte swizzled rows); the packed weights arrive by TMA into a staging
+// ring and eight warps widen them to fp16 in shared memory, written in the swizzled K-major layout
+// the MMA descriptors expect; one thread issues tcgen05.mma kind::f16 into an fp32 accumulator in
+// tensor memory; four warps read it back, multiply by the channel step and store fp16 while the next
+// tile's main loop runs into the other accumulator buffer.
+//
+// Widening a nibble to fp16 without a conversion: for a two's-complement nibble u of the code c,
+// u ^ 8 = c + 8, and the fp16 bit pattern 0x6400 | v is the number 1024 + v (0 <= v < 1024).  So
+// (u ^ 0x6408) read as fp16 is 1032 + c, and one exact fp16 subtraction of 1032 leaves c.  The
+// weight-only storage order puts channels (2s, 2s+1) of every eight at nibble positions (s, s+4) of a
+// 32-bit word, so that (word >> 4s) & 0x000F000F is one such pair in the two halves of a register:
+// a shift, one three-input logic operation and one half2 subtraction per two weights.
+#include <cuda.h>
+#include <cuda_fp16.h>
+
+#include "sq_internal.h"
+#include "sq_ptx.cuh"
+
+namespace sq {
+namespace {
+
+constexpr int WO_BM = 128;              // tokens per tile (UMMA M)
+constexpr int WO_UNPACK_WARPS = 8;
+constexpr int WO_EPI_WARPS = 4;
+constexpr int WO_THREADS = (2 + WO_UNPACK_WARPS + WO_EPI_WARPS) * 32;
+
+enum WoSite : uint32_t { WO_A_EMPTY = 80, WO_A_FULL, WO_ST_EMPTY, WO_ST_FULL, WO_B_EMPTY, WO_B_FULL, WO_TMEM_FULL, WO_TMEM_EMPTY };
+
+// Shared-memory plan: SA activation k-blocks (64 channels, 16 KB), SB widened weight k-blocks
+// (BN rows x 128 bytes), SS staging blocks of packed weights (BN rows x 128 bytes = 256 channels).
+template <int BN, int SA, int SS, int SB>
+struct WoSmem {
+  static constexpr int A_TILE = WO_BM * 128;
+  static constexpr int B_OP = BN * 128;
+  static constexpr int B_ST = BN * 128;
+  static constexpr int OFF_A = 0;
+  static constexpr int OFF_B_OP = OFF_A + SA * A_TILE;
+  static constexpr int OFF_B_ST = OFF_B_OP + SB * B_OP;
+  static constexpr int OFF_BAR = OFF_B_ST + SS * B_ST;
+  static constexpr int NUM_BARS = 2 * SA + 2 * SS + 2 * SB + 4;
+  static constexpr int OFF_TMEM = OFF_BAR + NUM_BARS * 8;
+  static constexpr int TOTAL = OFF_TMEM + 16;
+  static constexpr int DYN_BYTES = TOTAL + 1024;      // slack for the 1024-byte alignment
+};
+
+// Two weights (channels 2s, 2s+1 of the word's eight) as a half2.
+__device__ __forceinline__ uint32_t widen_pair(uint32_t word, int s) {
+  const uint32_t x = ((word >> (4 * s)) & 0x000F000Fu) ^ 0x64086408u;
+  const __half2 v = __hsub2(*reinterpret_cast<const __half2*>(&x), __half2half2(__ushort_as_half(0x6408)));
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+
+__device__ __forceinline__ uint4 widen_word(uint32_t word) {
+  return make_uint4(widen_pair(word, 0), widen_pair(word, 1), widen_pair(word, 2), widen_pair(word, 3));
+}
+
+// Widens k-block h (64 channels = 32 packed bytes) of BN staged rows into BN x 64 fp16.  Staging and
+// operand rows are 128 bytes with the 128-byte swizzle (16-byte chunk c of row r sits at chunk
+// c ^ (r & 7)).  Thread t takes source chunk j = (t >> 3) & 1 of rows 8 * (t >> 4) + (t & 7) + 128 i:
+// a quarter-warp covers eight consecutive rows, so its eight 16-byte loads and each round of eight
+// 16-byte stores fall into eight different bank groups.
+template <int BN>
+__device__ __forceinline__ void widen_tile(const unsigned char* __restrict__ st, unsigned char* __restrict__ op, int t,
+                                           int h) {
+  static_assert(BN % 128 == 0, "tile rows must be a multiple of 128");
+  const int j = (t >> 3) & 1;
+  const int r0 = ((t >> 4) << 3) + (t & 7);
+  const int sw = r0 & 7;
+#pragma unroll
+  for (int i = 0; i < BN / 128; ++i) {
+    const int r = r0 + i * 128;
+    const uint4 w = *reinterpret_cast<const uint4*>(st + r * 128 + ((((h << 1) + j) ^ sw) << 4));
+    unsigned char* dst = op + r * 128;
+    *reinterpret_cast<uint4*>(dst + ((((j << 2) + 0) ^ sw) << 4)) = widen_word(w.x);
+    *reinterpret_cast<uint4*>(dst + ((((j << 2) + 1) ^ sw) << 4)) = widen_word(w.y);
+    *reinterpret_cast<uint4*>(dst + ((((j << 2) + 2) ^ sw) << 4)) = widen_word(w.z);
+    *reinterpret_cast<uint4*>(dst + ((((j << 2) + 3) ^ sw) << 4)) = widen_word(w.w);
+  }
+}
+
+// Persistent kernel: CTA b works on tiles b, b + gridDim.x, ...; tile index = m_tile * tiles_n + n_tile.
+// Warp 0 lane 0: TMA producer.  Warp 1 lane 0: MMA issuer.  Warps 2..9: widen.  Warps 10..13: epilogue.
+template <int BN, int SA, int SS, int SB>
+__global__ void __launch_bounds__(WO_THREADS, 1)
+wo_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_constant__ CUtensorMap tmap_w,
+                  const __half* __restrict__ sw, int M, int N, int K, __half* __restrict__ Y) {
+  using L = WoSmem<BN, SA, SS, SB>;
+  griddep_launch_dependents();          // a rotate kernel launched behind this one may set itself up
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+  uint64_t* a_full = bars;
+  uint64_t* a_empty = a_full + SA;
+  uint64_t* st_full = a_empty + SA;
+  uint64_t* st_empty = st_full + SS;
+  uint64_t* b_full = st_empty + SS;
+  uint64_t* b_empty = b_full + SB;
+  uint64_t* tmem_full = b_empty + SB;         // [2]
+  uint64_t* tmem_empty = tmem_full + 2;       // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_TMEM);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = K / 64;                  // fp16 k-blocks of 64 channels
+  const int num_sb = (num_kb + 3) / 4;        // staging blocks of 256 channels (the last may be partly used)
+  const int tiles_n = (N + BN - 1) / BN, tiles_m = (M + WO_BM - 1) / WO_BM;
+  const int num_tiles = tiles_n * tiles_m;
+  const uint32_t limit = wait_limit();
+
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmap_z);
+    tma_prefetch_desc(&tmap_w);
+    for (int s = 0; s < SA; ++s) {
+      mbar_init(&a_full[s], 1);
+      mbar_init(&a_empty[s], 1);
+    }
+    for (int s = 0; s < SS; ++s) {
+      mbar_init(&st_full[s], 1);
+      mbar_init(&st_empty[s], WO_UNPACK_WARPS);
+    }
+    for (int s = 0; s < SB; ++s) {
+      mbar_init(&b_full[s], WO_UNPACK_WARPS);
+      mbar_init(&b_empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&tmem_full[b], 1);
+      mbar_init(&tmem_empty[b], WO_EPI_WARPS);
+    }
+    mbar_fence_init();
+  }
+  if (warp == 0) {
+    tmem_alloc(tmem_slot, 2 * BN);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();                                     // Z16 may come from the kernel launched before this one
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------------------
+    if (elect_one()) {
+      uint32_t ait = 0, sit = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        const int m0 = (tile / tiles_n) * WO_BM, n0 = (tile % tiles_n) * BN;
+        for (int sb = 0; sb < num_sb && ok; ++sb, ++sit) {
+          const int ss = sit % SS;
+          ok = mbar_wait(&st_empty[ss], ((sit / SS) & 1) ^ 1, WO_ST_EMPTY, limit);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&st_full[ss], L::B_ST);
+          tma_load_2d(smem + L::OFF_B_ST + ss * L::B_ST, &tmap_w, &st_full[ss], sb * 128, n0);
+          for (int h = 0; h < 4 && 4 * sb + h < num_kb; ++h, ++ait) {
+            const int sa = ait % SA;
+            ok = mbar_wait(&a_empty[sa], ((ait / SA) & 1) ^ 1, WO_A_EMPTY, limit);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&a_full[sa], L::A_TILE);
+            tma_load_2d(smem + L::OFF_A + sa * L::A_TILE, &tmap_z, &a_full[sa], (4 * sb + h) * 64, m0);
+          }
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer --------------------------------------------
+    if (elect_one()) {
+      constexpr uint32_t idesc = umma_idesc(/*c=f32*/ 1, /*a=f16*/ 0, /*b=f16*/ 0, WO_BM, BN);
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+        const uint32_t b = tcount & 1;
+        ok = mbar_wait(&tmem_empty[b], ((tcount >> 1) & 1) ^ 1, WO_TMEM_EMPTY, limit);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t tmem_d = tmem_base + b * BN;
+        for (int kb = 0; kb < num_kb; ++kb, ++it) {
+          const int sa = it % SA, sbo = it % SB;
+          ok = mbar_wait(&a_full[sa], (it / SA) & 1, WO_A_FULL, limit) &&
+               mbar_wait(&b_full[sbo], (it / SB) & 1, WO_B_FULL, limit);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t a_base = smem_u32(smem + L::OFF_A + sa * L::A_TILE);
+          const uint32_t b_base = smem_u32(smem + L::OFF_B_OP + sbo * L::B_OP);
+#pragma unroll
+          for (int k = 0; k < 4; ++k) {                // 4 x (K = 16 fp16) per 128-byte row
+            umma_f16(tmem_d, umma_desc_sw128(a_base + k * 32), umma_desc_sw128(b_base + k * 32), idesc,
+                     (kb | k) != 0 ? 1u : 0u);
+          }
+          umma_commit(&a_empty[sa]);                    // both operand stages are free when the MMAs retire
+          umma_commit(&b_empty[sbo]);
+        }
+        umma_commit(&tmem_full[b]);                     // accumulator complete (or abandoned)
+      }
+    }
+  } else if (warp < 2 + WO_UNPACK_WARPS) {
+    // ------------------------------ widening warps ------------------------------------------
+    const int t = threadIdx.x - 64;                    // 0 .. 255
+    uint32_t it = 0, sit = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int sb = 0; sb < num_sb && ok; ++sb, ++sit) {
+        const int ss = sit % SS;
+        ok = mbar_wait(&st_full[ss], (sit / SS) & 1, WO_ST_FULL, limit);
+        if (!ok) break;
+        for (int h = 0; h < 4 && 4 * sb + h < num_kb; ++h, ++it) {
+          const int s = it % SB;
+          ok = mbar_wait(&b_empty[s], ((it / SB) & 1) ^ 1, WO_B_EMPTY, limit);
+          if (!ok) break;
+          widen_tile<BN>(smem + L::OFF_B_ST + ss * L::B_ST, smem + L::OFF_B_OP + s * L::B_OP, t, h);
+          fence_proxy_async_smem();                     // generic-proxy stores -> visible to the MMA
+          __syncwarp();
+          if (lane == 0) mbar_arrive(&b_full[s]);
+        }
+        if (!ok) break;
+        __syncwarp();
+        if (lane == 0) mbar_arrive(&st_empty[ss]);
+      }
+    }
+  } else {
+    // ------------------------------ epilogue warps ------------------------------------------
+    const int quarter = warp & 3;                       // TMEM lanes this warp may read
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+      const int m0 = (tile / tiles_n) * WO_BM, n0 = (tile % tiles_n) * BN;
+      const uint32_t b = tcount & 1;
+      ok = mbar_wait(&tmem_full[b], (tcount >> 1) & 1, WO_TMEM_FULL, limit);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const int row = m0 + quarter * 32 + lane;
+      const uint32_t tmem_d = tmem_base + b * BN + (static_cast<uint32_t>(quarter * 32) << 16);
+#pragma unroll 1
+      for (int c = 0; c < BN / 32; ++c) {
+        uint32_t r[32];
+        tmem_ld_32x32b_x32(tmem_d + c * 32, r);
+        tmem_wait_ld();
+        const int col0 = n0 + c * 32;
+        if (row < M && col0 < N) {
+          __half* yrow = Y + static_cast<size_t>(row) * N + col0;
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {                 // groups of 8 columns (N % 8 == 0)
+            if (col0 + g * 8 < N) {
+              const uint4 swraw = __ldg(reinterpret_cast<const uint4*>(sw + col0 + g * 8));
+              const __half2* swh = reinterpret_cast<const __half2*>(&swraw);
+              uint4 out;
+              uint32_t* o = reinterpret_cast<uint32_t*>(&out);
+#pragma unroll
+              for (int e = 0; e < 4; ++e) {
+                const float2 sc = __half22float2(swh[e]);
+                const __half2 hv = __floats2half2_rn(__uint_as_float(r[g * 8 + 2 * e]) * sc.x,
+                                                     __uint_as_float(r[g * 8 + 2 * e + 1]) * sc.y);
+                o[e] = *reinterpret_cast<const uint32_t*>(&hv);
+              }
+              *reinterpret_cast<uint4*>(yrow + g * 8) = out;
+            }
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tmem_empty[b]);       // this warp's quarter of the buffer is drained
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 0) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 2 * BN);
+  }
+}
+
+// Plain kernel for shapes the tensor-core path does not take (K % 64 != 0, N % 8 != 0): one thread per
+// output channel, fp32 multiply-adds in channel order; gridDim.y strides over the token rows.
+__global__ void wo_gemm_simple_kernel(const __half* __restrict__ Z16, const uint8_t* __restrict__ Wq,
+                                      const __half* __restrict__ sw, int M, int N, int K, __half* __restrict__ Y) {
+  const int c = blockIdx.x * blockDim.x + threadIdx.x;
+  if (c >= N) return;
+  const uint32_t* wrow = reinterpret_cast<const uint32_t*>(Wq + static_cast<size_t>(c) * (K / 2));
+  const float swv = __half2float(sw[c]);
+  for (int t = blockIdx.y; t < M; t += gridDim.y) {
+    const __half* z = Z16 + static_cast<size_t>(t) * K;
+    float acc = 0.0f;
+    for (int g = 0; g < K / 8; ++g) {
+      const uint32_t word = wrow[g];
+#pragma unroll
+      for (int s = 0; s < 4; ++s) {
+        const int c0 = (static_cast<int>(word << (28 - 4 * s))) >> 28;          // nibble position s: channel 2s
+        const int c1 = (static_cast<int>(word << (12 - 4 * s))) >> 28;          // nibble position s + 4: channel 2s + 1
+        acc = fmaf(__half2float(z[8 * g + 2 * s]), static_cast<float>(c0), acc);
+        acc = fmaf(__half2float(z[8 * g + 2 * s + 1]), static_cast<float>(c1), acc);
+      }
+    }
+    Y[static_cast<size_t>(t) * N + c] = __float2half_rn(acc * swv);
+  }
+}
+
+// Channel order -> weight-only storage order, one 32-bit word (eight channels) per thread, in place.
+__global__ void interleave_nibbles_kernel(uint32_t* __restrict__ words, long long count) {
+  for (long long i = blockIdx.x * static_cast<long long>(blockDim.x) + threadIdx.x; i < count;
+       i += static_cast<long long>(gridDim.x) * blockDim.x) {
+    const uint32_t w = words[i];
+    uint32_t o = 0;
+#pragma unroll
+    for (int s = 0; s < 4; ++s) {
+      o |= ((w >> (8 * s)) & 0xFu) << (4 * s);               // channel 2s     -> position s
+      o |= ((w >> (8 * s + 4)) & 0xFu) << (4 * s + 16);      // channel 2s + 1 -> position s + 4
+    }
+    words[i] = o;
+  }
+}
+
+template <int BN, int SA, int SS, int SB>
+sq_status_t launch_wo_tc(const void* Z16, const void* Wq, const void* sw, int M, int N, int K, void* Y, cudaStream_t s) {
+  using L = WoSmem<BN, SA, SS, SB>;
+  static_assert(L::DYN_BYTES <= 227 * 1024, "shared-memory plan does not fit");
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return SQ_ERR_CUDA;
+  CUtensorMap mz, mw;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(M)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
+  const cuuint32_t box[2] = {64, WO_BM};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&mz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(Z16), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return SQ_ERR_CUDA;
+  if (!make_packed_map(&mw, Wq, N, K / 2, BN)) return SQ_ERR_CUDA;
+  auto kern = wo_gemm_tc_kernel<BN, SA, SS, SB>;
+  if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), L::DYN_BYTES)) return SQ_ERR_CUDA;
+  const int sms = sm_count();
+  if (sms <= 0) return SQ_ERR_CUDA;
+  const int tiles = ((N + BN - 1) / BN) * ((M + WO_BM - 1) / WO_BM);
+  const int grid = tiles < sms ? tiles : sms;
+  const cudaError_t err = launch_maybe_pdl(kern, dim3(grid), dim3(WO_THREADS), L::DYN_BYTES, s, mz, mw,
+                                           static_cast<const __half*>(sw), M, N, K, static_cast<__half*>(Y));
+  count_launch();
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
+}
+
+}  // namespace
+
+sq_status_t launch_wo_gemm(const void* Z16, const void* Wq, const void* sw, int64_t M, int64_t N, int64_t K, void* Y,
+                           cudaStream_t s) {
+  if (M == 0 || N == 0) return SQ_OK;
+  const bool tc_ok = (K % 64 == 0) && (N % 8 == 0);
+  if (tc_ok) {
+    // 256-channel tiles where they fill the device with enough token rows to use them
+    if (M > 128 && N >= 256 * 64) return launch_wo_tc<256, 4, 2, 3>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
+    return launch_wo_tc<128, 6, 2, 4>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
+  }
+  dim3 block(128), grid((unsigned)((N + 127) / 128), (unsigned)(M < 65535 ? M : 65535));
+  wo_gemm_simple_kernel<<<grid, block, 0, s>>>(static_cast<const __half*>(Z16), static_cast<const uint8_t*>(Wq),
+                                               static_cast<const __half*>(sw), (int)M, (int)N, (int)K,
+                                               static_cast<__half*>(Y));
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+}
+
+sq_status_t launch_interleave_nibbles(void* Wq, int64_t rows, int64_t K, cudaStream_t s) {
+  const long long count = static_cast<long long>(rows) * (K / 8);
+  if (count == 0) return SQ_OK;
+  const int sms = sm_count();
+  if (sms <= 0) return SQ_ERR_CUDA;
+  const long long want = (count + 255) / 256;
+  const unsigned grid = static_cast<unsigned>(want < static_cast<long long>(sms) * 16 ? want : static_cast<long long>(sms) * 16);
+  interleave_nibbles_kernel<<<grid, 256, 0, s>>>(static_cast<uint32_t*>(Wq), count);
+  count_launch();
+  return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+}
+
+}  // namespace sq

@@ -119,19 +119,20 @@ sq_status_t build_factors_host(const float* calib, int64_t T, int64_t n, int32_t
                                std::vector<float>& R1, std::vector<float>& R2, R2Structure* s2);
 
 // Steps 1+2 (sq_rotate_quant.cu).  R1/R2 device fp32 or both nullptr for the identity.
+// qmax = 2^(b-1) - 1 for b-bit codes (7: INT4); qmax = 0: rotation only, Xq receives fp16 rows.
 sq_status_t launch_rotate_quant(const float* dR1, const float* dR2, int n1, int n2, const void* X,
-                                int64_t rows, void* Xq, void* scales, float* Zdbg, cudaStream_t s);
+                                int64_t rows, void* Xq, void* scales, float* Zdbg, cudaStream_t s, int qmax = 7);
 
 // Tensor-core variant of steps 1+2 (sq_rotate_quant_tc.cu).
 bool rotate_quant_tc_supported(int n1, int n2);
 bool rotate_quant_tc_prepare(sq_rotation* h);
 sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
-                                   float* Zdbg, cudaStream_t s);
+                                   float* Zdbg, cudaStream_t s, bool f16out = false);
 // Tensor-core variant for 128 < n1 <= 256 on CTA pairs (sq_rotate_quant_pair.cu).
 bool rotate_quant_pair_supported(int n1, int n2);
 bool rotate_quant_pair_prepare(sq_rotation* h);
 sq_status_t launch_rotate_quant_pair(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
-                                     float* Zdbg, cudaStream_t s);
+                                     float* Zdbg, cudaStream_t s, bool f16out = false);
 // Steps 1+2 with R2 applied through its structure (sq_rotate_quant_st.cu): R1^T on the tensor cores,
 // then the Hadamard butterflies and the two rotation chains of URT in registers.
 bool rotate_quant_st_prepare(sq_rotation* h);
@@ -146,6 +147,9 @@ sq_status_t launch_linear_fused(const sq_rotation* h, const void* X, int64_t M, 
 // Picks the tensor-core kernel when the handle has its images, else the generic fp32 kernel.
 sq_status_t rotate_quant_dispatch(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
                                   float* Zdbg, cudaStream_t s);
+
+// Step 1 alone with fp16 rows out (the rotation-only form of the kernels above).
+sq_status_t rotate_f16_dispatch(const sq_rotation* h, const void* X, int64_t rows, void* Z16, cudaStream_t s);
 
 // Step 3 (sq_gemm.cu).
 sq_status_t launch_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw,
@@ -166,6 +170,13 @@ sq_status_t launch_w4a4_gemm_decode(const void* Xq, const void* sx, const void* 
 bool gemv_supported(int64_t M, int64_t N, int64_t K);
 sq_status_t launch_w4a4_gemv(const void* Xq, const void* sx, const void* Wq, const void* sw, int M, int N, int K,
                              void* Y, int32_t* accdbg, cudaStream_t s);
+
+// Weight-only variant (sq_gemm_wo.cu): fp16 activations x b-bit weight codes in the weight-only
+// storage order, fp32 accumulation, one rounding of acc * s_w to fp16.
+sq_status_t launch_wo_gemm(const void* Z16, const void* Wq, const void* sw, int64_t M, int64_t N, int64_t K, void* Y,
+                           cudaStream_t s);
+// Rewrites packed rows [rows x K/2] from channel order into the weight-only storage order, in place.
+sq_status_t launch_interleave_nibbles(void* Wq, int64_t rows, int64_t K, cudaStream_t s);
 
 // Device status word helpers (sq_api.cu).
 sq_status_t read_and_clear_device_status(cudaStream_t s);

@@ -36,23 +36,26 @@ __device__ __forceinline__ float block_max(float v, float* red) {
 
 // The quantiser's decision, in fp32 and in this order of operations:
 //   Delta = fp16(amax / 7); inv = 1 / Delta; code = floor(fl(fl(z * inv) + 0.5)) clamped to [-8, 7].
-__device__ __forceinline__ int quant_code(float z, float inv) {
+// With b bits the 7 becomes qmax = 2^(b-1) - 1 and the clamp [-qmax - 1, qmax] (weight-only variant).
+__device__ __forceinline__ int quant_code(float z, float inv, int qmax = 7) {
   const float t = __fadd_rn(__fmul_rn(z, inv), 0.5f);
   int c = static_cast<int>(floorf(t));
-  return max(-8, min(7, c));
+  return max(-qmax - 1, min(qmax, c));
 }
 
-__device__ __forceinline__ void row_scale(float amax, __half& delta, float& inv) {
-  delta = __float2half_rn(__fdiv_rn(amax, 7.0f));
+__device__ __forceinline__ void row_scale(float amax, __half& delta, float& inv, int qmax = 7) {
+  delta = __float2half_rn(__fdiv_rn(amax, static_cast<float>(qmax)));
   const float d = __half2float(delta);
   inv = (d > 0.0f) ? __fdiv_rn(1.0f, d) : 0.0f;
 }
 
+// `qmax` = 7 for INT4; qmax = 0 means rotation only: Xq then receives the rotated rows as fp16
+// [rows x n] and `scales` is not touched (weight-only variant).
 template <int MAXT, bool VEC>
 __global__ void __launch_bounds__(512)
 rotate_quant_kernel(const float* __restrict__ R1, const float* __restrict__ R2, int n1, int n2,
                     const __half* __restrict__ X, long long rows, uint8_t* __restrict__ Xq,
-                    __half* __restrict__ scales, float* __restrict__ Zdbg) {
+                    __half* __restrict__ scales, float* __restrict__ Zdbg, int qmax) {
   griddep_wait();                    // X may come from the kernel before this one in the stream
   griddep_launch_dependents();       // a GEMM launched behind this kernel may set itself up from here on
   extern __shared__ __align__(16) unsigned char smem_raw[];
@@ -151,12 +154,33 @@ rotate_quant_kernel(const float* __restrict__ R1, const float* __restrict__ R2, 
           for (int j = 0; j < TQ; ++j) amax = fmaxf(amax, fabsf(z[t][i][j]));   // padded entries are 0
       }
     }
+    if (qmax == 0) {
+      // ---- rotation only: the row leaves as fp16 ---------------------------------------------------
+      __half* zrow16 = reinterpret_cast<__half*>(Xq) + row * (long long)n;
+#pragma unroll
+      for (int t = 0; t < MAXT; ++t) {
+        const int tile = tid + t * nthr;
+        if (tile < ntiles) {
+          const int p0 = (tile / tiles_q) * TP, q0 = (tile % tiles_q) * TQ;
+#pragma unroll
+          for (int i = 0; i < TP; ++i) {
+            if (!VEC && p0 + i >= n1) continue;
+            const int c0 = (p0 + i) * n2 + q0;
+#pragma unroll
+            for (int j = 0; j < TQ; ++j)
+              if (VEC || q0 + j < n2) zrow16[c0 + j] = __float2half_rn(z[t][i][j]);
+          }
+        }
+      }
+      __syncthreads();
+      continue;
+    }
     amax = block_max(amax, red);
 
     // ---- quantise, pack, store ---------------------------------------------------------------
     __half delta;
     float inv;
-    row_scale(amax, delta, inv);
+    row_scale(amax, delta, inv, qmax);
     if (tid == 0) scales[row] = delta;
     uint8_t* qrow = Xq + row * (long long)(n / 2);
 #pragma unroll
@@ -168,8 +192,8 @@ rotate_quant_kernel(const float* __restrict__ R1, const float* __restrict__ R2, 
         for (int i = 0; i < TP; ++i) {
           if (!VEC && p0 + i >= n1) continue;
           const int c0 = (p0 + i) * n2 + q0;     // even: n2 is even and q0 is a multiple of 4
-          const int k0 = quant_code(z[t][i][0], inv), k1 = quant_code(z[t][i][1], inv);
-          const int k2 = quant_code(z[t][i][2], inv), k3 = quant_code(z[t][i][3], inv);
+          const int k0 = quant_code(z[t][i][0], inv, qmax), k1 = quant_code(z[t][i][1], inv, qmax);
+          const int k2 = quant_code(z[t][i][2], inv, qmax), k3 = quant_code(z[t][i][3], inv, qmax);
           const uint8_t b0 = static_cast<uint8_t>((k0 & 15) | ((k1 & 15) << 4));
           const uint8_t b1 = static_cast<uint8_t>((k2 & 15) | ((k3 & 15) << 4));
           if (VEC) {
@@ -198,7 +222,7 @@ rotate_quant_kernel(const float* __restrict__ R1, const float* __restrict__ R2, 
 // Identity rotation: quantise the fp16 rows as they are (used by sq_pack_weight with no handle).
 __global__ void __launch_bounds__(256)
 quant_rows_kernel(const __half* __restrict__ X, long long rows, int n, uint8_t* __restrict__ Xq,
-                  __half* __restrict__ scales, float* __restrict__ Zdbg) {
+                  __half* __restrict__ scales, float* __restrict__ Zdbg, int qmax) {
   __shared__ float red[32];
   for (long long row = blockIdx.x; row < rows; row += gridDim.x) {
     const __half* xrow = X + row * n;
@@ -207,12 +231,12 @@ quant_rows_kernel(const __half* __restrict__ X, long long rows, int n, uint8_t* 
     amax = block_max(amax, red);
     __half delta;
     float inv;
-    row_scale(amax, delta, inv);
+    row_scale(amax, delta, inv, qmax);
     if (threadIdx.x == 0) scales[row] = delta;
     uint8_t* qrow = Xq + row * (long long)(n / 2);
     for (int i = threadIdx.x; i < n / 2; i += blockDim.x) {
       const float z0 = __half2float(xrow[2 * i]), z1 = __half2float(xrow[2 * i + 1]);
-      const int k0 = quant_code(z0, inv), k1 = quant_code(z1, inv);
+      const int k0 = quant_code(z0, inv, qmax), k1 = quant_code(z1, inv, qmax);
       qrow[i] = static_cast<uint8_t>((k0 & 15) | ((k1 & 15) << 4));
       if (Zdbg != nullptr) {
         Zdbg[row * (long long)n + 2 * i] = z0;
@@ -225,7 +249,7 @@ quant_rows_kernel(const __half* __restrict__ X, long long rows, int n, uint8_t* 
 template <int MAXT, bool VEC>
 sq_status_t launch_generic(const float* dR1, const float* dR2, int n1, int n2, const void* X, int64_t rows,
                            void* Xq, void* scales, float* Zdbg, int threads, size_t smem, int sms,
-                           cudaStream_t s) {
+                           cudaStream_t s, int qmax) {
   auto kern = rotate_quant_kernel<MAXT, VEC>;
   if (smem > 48 * 1024) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
@@ -237,7 +261,7 @@ sq_status_t launch_generic(const float* dR1, const float* dR2, int n1, int n2, c
   const long long grid = std::min<long long>(rows, static_cast<long long>(sms) * per_sm);
   kern<<<static_cast<unsigned>(grid), threads, smem, s>>>(dR1, dR2, n1, n2, static_cast<const __half*>(X), rows,
                                                          static_cast<uint8_t*>(Xq), static_cast<__half*>(scales),
-                                                         Zdbg);
+                                                         Zdbg, qmax);
   count_launch();
   return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
 }
@@ -245,17 +269,18 @@ sq_status_t launch_generic(const float* dR1, const float* dR2, int n1, int n2, c
 }  // namespace
 
 sq_status_t launch_rotate_quant(const float* dR1, const float* dR2, int n1, int n2, const void* X,
-                                int64_t rows, void* Xq, void* scales, float* Zdbg, cudaStream_t s) {
+                                int64_t rows, void* Xq, void* scales, float* Zdbg, cudaStream_t s, int qmax) {
   if (rows == 0) return SQ_OK;
   const long long n = static_cast<long long>(n1) * n2;
   const int sms = sm_count();
   if (sms <= 0) return SQ_ERR_CUDA;
 
   if (dR1 == nullptr || dR2 == nullptr) {
+    if (qmax == 0) return SQ_ERR_INVALID_ARG;          // rotation only with no rotation: nothing to do here
     const long long grid = std::min<long long>(rows, static_cast<long long>(sms) * 8);
     quant_rows_kernel<<<static_cast<unsigned>(grid), 256, 0, s>>>(static_cast<const __half*>(X), rows,
                                                                    static_cast<int>(n), static_cast<uint8_t*>(Xq),
-                                                                   static_cast<__half*>(scales), Zdbg);
+                                                                   static_cast<__half*>(scales), Zdbg, qmax);
     count_launch();
     return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
   }
@@ -273,8 +298,8 @@ sq_status_t launch_rotate_quant(const float* dR1, const float* dR2, int n1, int 
   if (smem > 227 * 1024) return SQ_ERR_UNSUPPORTED;
 
 #define SQ_DISPATCH(MT)                                                                                      \
-  return vec ? launch_generic<MT, true>(dR1, dR2, n1, n2, X, rows, Xq, scales, Zdbg, threads, smem, sms, s)  \
-             : launch_generic<MT, false>(dR1, dR2, n1, n2, X, rows, Xq, scales, Zdbg, threads, smem, sms, s)
+  return vec ? launch_generic<MT, true>(dR1, dR2, n1, n2, X, rows, Xq, scales, Zdbg, threads, smem, sms, s, qmax)  \
+             : launch_generic<MT, false>(dR1, dR2, n1, n2, X, rows, Xq, scales, Zdbg, threads, smem, sms, s, qmax)
   if (maxt == 1) { SQ_DISPATCH(1); }
   if (maxt == 2) { SQ_DISPATCH(2); }
   SQ_DISPATCH(4);

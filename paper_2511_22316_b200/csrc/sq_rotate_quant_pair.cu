@@ -71,7 +71,7 @@ __device__ __forceinline__ uint64_t umma_desc_mn(uint32_t smem_addr, uint32_t sb
   return d;
 }
 
-template <int N2, int CW>
+template <int N2, int CW, bool F16OUT>
 __global__ void __cluster_dims__(2, 1, 1) __launch_bounds__((2 + 4 * CW * (256 / N2)) * 32, 1)
 rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsigned char* __restrict__ a1_img,
                          const unsigned char* __restrict__ b2_img, int n1, long long rows,
@@ -295,6 +295,30 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
       ok = mbar_wait(&d2_full[w], ph, RQP_D2_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
+      if constexpr (F16OUT) {
+        // rotation only: the rotated row leaves as fp16 (weight-only variant), nothing is quantised
+        __half* zrow16 = reinterpret_cast<__half*>(Xq) + token * n + static_cast<long long>(pp) * N2 + cp * HC;
+#pragma unroll
+        for (int c = 0; c < HC / 16; ++c) {
+          uint32_t r[16];
+          tmem_ld_32x32b_x16(d2 + 16 * c, r);
+          tmem_wait_ld();
+          uint4 lo, hi;
+          lo.x = pack_half2(__uint_as_float(r[0]) * un, __uint_as_float(r[1]) * un);
+          lo.y = pack_half2(__uint_as_float(r[2]) * un, __uint_as_float(r[3]) * un);
+          lo.z = pack_half2(__uint_as_float(r[4]) * un, __uint_as_float(r[5]) * un);
+          lo.w = pack_half2(__uint_as_float(r[6]) * un, __uint_as_float(r[7]) * un);
+          hi.x = pack_half2(__uint_as_float(r[8]) * un, __uint_as_float(r[9]) * un);
+          hi.y = pack_half2(__uint_as_float(r[10]) * un, __uint_as_float(r[11]) * un);
+          hi.z = pack_half2(__uint_as_float(r[12]) * un, __uint_as_float(r[13]) * un);
+          hi.w = pack_half2(__uint_as_float(r[14]) * un, __uint_as_float(r[15]) * un);
+          if (live) {
+            *reinterpret_cast<uint4*>(zrow16 + 16 * c) = lo;
+            *reinterpret_cast<uint4*>(zrow16 + 16 * c + 8) = hi;
+          }
+        }
+        continue;
+      }
       float zm = 0.0f;
 #pragma unroll
       for (int c = 0; c < HC / 16; ++c) {
@@ -410,6 +434,26 @@ rotate_quant_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const unsig
       ok = mbar_wait(&d2_full[w], ph, RQP_D2_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
+      if constexpr (F16OUT) {
+        // rotation only: the rotated row leaves as fp16 (weight-only variant), nothing is quantised
+        __half* zrow16 = reinterpret_cast<__half*>(Xq) + token * n + static_cast<long long>(pp) * N2;
+#pragma unroll
+        for (int c = 0; c < N2 / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld_32x32b_x32(d2 + 32 * c, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            uint4 v;
+            v.x = pack_half2(__uint_as_float(r[e]) * un, __uint_as_float(r[e + 1]) * un);
+            v.y = pack_half2(__uint_as_float(r[e + 2]) * un, __uint_as_float(r[e + 3]) * un);
+            v.z = pack_half2(__uint_as_float(r[e + 4]) * un, __uint_as_float(r[e + 5]) * un);
+            v.w = pack_half2(__uint_as_float(r[e + 6]) * un, __uint_as_float(r[e + 7]) * un);
+            if (live) *reinterpret_cast<uint4*>(zrow16 + 32 * c + e) = v;
+          }
+        }
+        continue;
+      }
       float zm = 0.0f;
 #pragma unroll
       for (int c = 0; c < N2 / 32; ++c) {
@@ -521,7 +565,7 @@ bool rotate_quant_pair_prepare(sq_rotation* h) {
 }
 
 sq_status_t launch_rotate_quant_pair(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
-                                     float* Zdbg, cudaStream_t s) {
+                                     float* Zdbg, cudaStream_t s, bool f16out) {
   const int n1 = h->n1, n2 = h->n2;
   const RqPairLayout L = rq_pair_layout(n1, n2);
   EncodeTiledFn enc = get_encode_fn();
@@ -543,14 +587,14 @@ sq_status_t launch_rotate_quant_pair(const sq_rotation* h, const void* X, int64_
   const unsigned char* a1 = static_cast<const unsigned char*>(h->dA1img);
   const unsigned char* b2 = static_cast<const unsigned char*>(h->dB2img);
   if (n2 == 64) {
-    auto kern = rotate_quant_pair_kernel<64, 1>;
+    auto kern = f16out ? rotate_quant_pair_kernel<64, 1, true> : rotate_quant_pair_kernel<64, 1, false>;
     if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return SQ_ERR_CUDA;
     if (launch_dependent(kern, dim3(grid), dim3((2 + 4 * 4) * 32), static_cast<size_t>(smem), s, mx, a1, b2, n1, rows,
                          static_cast<uint8_t*>(Xq), static_cast<__half*>(scales), Zdbg) != cudaSuccess)
       return SQ_ERR_CUDA;
   } else {
     // two slots of eight warps (18 warps in the CTA instead of 10)
-    auto kern = rotate_quant_pair_kernel<128, 2>;
+    auto kern = f16out ? rotate_quant_pair_kernel<128, 2, true> : rotate_quant_pair_kernel<128, 2, false>;
     if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return SQ_ERR_CUDA;
     if (launch_dependent(kern, dim3(grid), dim3((2 + 4 * 2 * 2) * 32), static_cast<size_t>(smem), s, mx, a1, b2, n1, rows,
                          static_cast<uint8_t*>(Xq), static_cast<__half*>(scales), Zdbg) != cudaSuccess)

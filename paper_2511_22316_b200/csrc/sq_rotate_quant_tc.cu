@@ -130,7 +130,7 @@ __device__ __forceinline__ float absmax32(const uint32_t (&r)[32]) {
 
 // The kernel's body, for CTA `cta` of `ncta` that share the token groups (the fused decode kernel of
 // sq_linear_fused.cu runs it in its first CTAs, with more warps in the block than the roles below use).
-template <int N2, int S, int CW = 1>
+template <int N2, int S, int CW = 1, bool F16OUT = false>
 __device__ __forceinline__ void rotate_quant_tc_body(const CUtensorMap& tmap_x, const RqLayout& L,
                                                      const unsigned char* __restrict__ a1_img,
                                                      const unsigned char* __restrict__ b2_img, int n1, int rows,
@@ -361,6 +361,31 @@ __device__ __forceinline__ void rotate_quant_tc_body(const CUtensorMap& tmap_x, 
       ok = mbar_wait(&d2_full[w], ph, RQ_D2_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
+      if constexpr (F16OUT) {
+        // rotation only: the rotated row leaves as fp16 (weight-only variant), nothing is quantised
+        const bool live16 = (pp < n1) && (token < rows);
+        __half* zrow16 = reinterpret_cast<__half*>(Xq) + token * n + pp * N2 + cp * HC;
+#pragma unroll
+        for (int c = 0; c < HC / 16; ++c) {
+          uint32_t r[16];
+          tmem_ld_32x32b_x16(d2 + 16 * c, r);
+          tmem_wait_ld();
+          uint4 lo, hi;
+          lo.x = pack_half2(__uint_as_float(r[0]) * un, __uint_as_float(r[1]) * un);
+          lo.y = pack_half2(__uint_as_float(r[2]) * un, __uint_as_float(r[3]) * un);
+          lo.z = pack_half2(__uint_as_float(r[4]) * un, __uint_as_float(r[5]) * un);
+          lo.w = pack_half2(__uint_as_float(r[6]) * un, __uint_as_float(r[7]) * un);
+          hi.x = pack_half2(__uint_as_float(r[8]) * un, __uint_as_float(r[9]) * un);
+          hi.y = pack_half2(__uint_as_float(r[10]) * un, __uint_as_float(r[11]) * un);
+          hi.z = pack_half2(__uint_as_float(r[12]) * un, __uint_as_float(r[13]) * un);
+          hi.w = pack_half2(__uint_as_float(r[14]) * un, __uint_as_float(r[15]) * un);
+          if (live16) {
+            *reinterpret_cast<uint4*>(zrow16 + 16 * c) = lo;
+            *reinterpret_cast<uint4*>(zrow16 + 16 * c + 8) = hi;
+          }
+        }
+        continue;
+      }
       float zm = 0.0f;
 #pragma unroll
       for (int c = 0; c < HC / 16; ++c) {
@@ -477,6 +502,27 @@ __device__ __forceinline__ void rotate_quant_tc_body(const CUtensorMap& tmap_x, 
       ok = mbar_wait(&d2_full[w], ph, RQ_D2_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
+      if constexpr (F16OUT) {
+        // rotation only: the rotated row leaves as fp16 (weight-only variant), nothing is quantised
+        const bool live16 = (pp < n1) && (token < rows);
+        __half* zrow16 = reinterpret_cast<__half*>(Xq) + token * n + pp * N2;
+#pragma unroll
+        for (int c = 0; c < N2 / 32; ++c) {
+          uint32_t r[32];
+          tmem_ld_32x32b_x32(d2 + 32 * c, r);
+          tmem_wait_ld();
+#pragma unroll
+          for (int e = 0; e < 32; e += 8) {
+            uint4 v;
+            v.x = pack_half2(__uint_as_float(r[e]) * un, __uint_as_float(r[e + 1]) * un);
+            v.y = pack_half2(__uint_as_float(r[e + 2]) * un, __uint_as_float(r[e + 3]) * un);
+            v.z = pack_half2(__uint_as_float(r[e + 4]) * un, __uint_as_float(r[e + 5]) * un);
+            v.w = pack_half2(__uint_as_float(r[e + 6]) * un, __uint_as_float(r[e + 7]) * un);
+            if (live16) *reinterpret_cast<uint4*>(zrow16 + 32 * c + e) = v;
+          }
+        }
+        continue;
+      }
       float zm = 0.0f;
 #pragma unroll
       for (int c = 0; c < N2 / 32; ++c) {
@@ -543,12 +589,12 @@ __device__ __forceinline__ void rotate_quant_tc_body(const CUtensorMap& tmap_x, 
 
 // S accumulator slots (= compute groups) per CTA.  With S * 2 * N2 = 256 TMEM columns two CTAs share
 // an SM (each with its own producer and MMA issuer); with 512 a CTA has the SM to itself.
-template <int N2, int S, int CW = 1>
+template <int N2, int S, int CW = 1, bool F16OUT = false>
 __global__ void __launch_bounds__((2 + 4 * S * CW) * 32, (S * 2 * N2 <= 256) ? 2 : 1)
 rotate_quant_tc_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ RqLayout L,
                        const unsigned char* __restrict__ a1_img, const unsigned char* __restrict__ b2_img, int n1,
                        int rows, uint8_t* __restrict__ Xq, __half* __restrict__ scales, float* __restrict__ Zdbg) {
-  rotate_quant_tc_body<N2, S, CW>(tmap_x, L, a1_img, b2_img, n1, rows, Xq, scales, Zdbg, static_cast<int>(blockIdx.x),
+  rotate_quant_tc_body<N2, S, CW, F16OUT>(tmap_x, L, a1_img, b2_img, n1, rows, Xq, scales, Zdbg, static_cast<int>(blockIdx.x),
                               static_cast<int>(gridDim.x));
 }
 
@@ -610,7 +656,7 @@ bool rotate_quant_tc_prepare(sq_rotation* h) {
 }
 
 sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t rows, void* Xq, void* scales,
-                                   float* Zdbg, cudaStream_t s) {
+                                   float* Zdbg, cudaStream_t s, bool f16out) {
   const int n1 = h->n1, n2 = h->n2;
   if (rows > 0x7FFFFFFF) return SQ_ERR_UNSUPPORTED;   // the kernel counts token groups in 32 bits
   // n2 = 64 with images small enough: two CTAs per SM, two accumulator slots each.
@@ -646,7 +692,12 @@ sq_status_t launch_rotate_quant_tc(const sq_rotation* h, const void* X, int64_t 
   // n2 = 128 (one CTA per SM, two slots): eight warps per slot, 18 in all instead of 10 -- measured 10 %
   // faster on 4096 x 8192 (39.7 -> 35.5 us) and 0.8 us on the decode batches (6.6 -> 5.8 us).  With n2 = 64
   // and two CTAs per SM the same split leaves 56 registers per thread and was slower (12.0 -> 15.9 us).
-  if (n2 == 64 && dual) ok = launch(rotate_quant_tc_kernel<64, 2>, 2, 2);
+  if (f16out) {
+    // rotation only: Xq receives the rotated rows as fp16 [rows x n], `scales` is not touched
+    if (n2 == 64 && dual) ok = launch(rotate_quant_tc_kernel<64, 2, 1, true>, 2, 2);
+    else if (n2 == 64) ok = launch(rotate_quant_tc_kernel<64, 4, 1, true>, 4, 1);
+    else ok = launch(rotate_quant_tc_kernel<128, 2, 2, true>, 2, 1, 2);
+  } else if (n2 == 64 && dual) ok = launch(rotate_quant_tc_kernel<64, 2>, 2, 2);
   else if (n2 == 64) ok = launch(rotate_quant_tc_kernel<64, 4>, 4, 1);
   else ok = launch(rotate_quant_tc_kernel<128, 2, 2>, 2, 1, 2);
   if (!ok) return SQ_ERR_CUDA;
