@@ -8,7 +8,8 @@ the named workload.  Prints ONE JSON line.
                   [--structured-r2] [--fuse-decode] [--no-sweep] [--no-cpu-baseline] [--quick]
 
 After the headline workload the default run also times every other benchmark workload briefly and
-reports them under "per_workload" of the same line (skipped with --no-sweep or N > 1).
+reports them under "per_workload" of the same line, and the weight-only variant (W4A16 / W3A16) and the
+grouped mixture-of-experts layer under "variants" (all skipped with --no-sweep or N > 1).
 
 N > 1: launched under torchrun, one process per GPU; the path shards over tokens with no
 collective (each rank owns its own batch and a replica of the packed weights), so scaling is
@@ -460,6 +461,167 @@ def rooflines(w, rq_ms, gemm_ms, pk, structured, yard=None):
     return roof_gemm, roof_rq
 
 
+def _graph_ms(torch, fn, count):
+    """Milliseconds per call of `fn(i)` replayed from a CUDA graph of `count` back-to-back calls."""
+    gstream = torch.cuda.Stream()
+    gstream.wait_stream(torch.cuda.current_stream())
+    graph = torch.cuda.CUDAGraph()
+    with torch.cuda.stream(gstream):
+        with torch.cuda.graph(graph, stream=gstream):
+            for i in range(count):
+                fn(i)
+        graph.replay()
+        gstream.synchronize()
+        g0, g1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        g0.record(gstream)
+        for _ in range(5):
+            graph.replay()
+        g1.record(gstream)
+        gstream.synchronize()
+        ms = g0.elapsed_time(g1) / (5 * count)
+    torch.cuda.current_stream().wait_stream(gstream)
+    torch.cuda.synchronize()
+    return ms
+
+
+def _events_ms(torch, fn, count):
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for i in range(count):
+        fn(i)
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / count
+
+
+def weight_only_entry(sq, torch, w, bits, pk, l2):
+    """The weight-only layer (fp16 rotated activations x b-bit weights) on one workload: the step through
+    sq_linear_wo, its two kernels from graph replays, roofline fractions, and a library fp16 GEMM of the
+    same shape (torch.matmul, no unpacking, no scaling) as the yardstick."""
+    M, N, K = w.M, w.N, w.K
+    X = wl.make_activations(w)
+    W = wl.make_weights(w)
+    rot = sq.sq_build_rotation(X.astype(np.float32), w.n1, w.n2, seed=0)
+    dW = torch.from_numpy(W).cuda()
+    Wq = torch.empty((N, K // 2), dtype=torch.uint8, device="cuda")
+    sw = torch.empty((N,), dtype=torch.float16, device="cuda")
+    sq.sq_pack_weight_wo(rot, dW, N, K, bits, Wq, sw)
+    torch.cuda.synchronize()
+    per_set = M * K * 2 * 2 + M * N * 2 + N * K // 2
+    nsets = max(2, int(np.ceil(1.5 * l2 / per_set)) + 1)
+    ws_bytes = sq.sq_linear_wo_workspace_bytes(M, K)
+    dX = torch.from_numpy(X).cuda()
+    sets = []
+    for _ in range(nsets):
+        ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
+        sets.append({"X": dX.clone(), "Wq": Wq.clone(), "sw": sw.clone(), "ws": ws,
+                     "ws_ptr": ws.data_ptr() + (-ws.data_ptr()) % 256,
+                     "Y": torch.empty((M, N), dtype=torch.float16, device="cuda")})
+
+    def step(i):
+        t = sets[i % nsets]
+        sq.sq_linear_wo(rot, t["X"], M, t["Wq"], t["sw"], N, K, t["ws_ptr"], ws_bytes, t["Y"])
+
+    def rotate(i):
+        t = sets[i % nsets]
+        sq.sq_rotate_act_f16(rot, t["X"], M, t["ws_ptr"])
+
+    def gemm(i):
+        t = sets[i % nsets]
+        sq.sq_w4a16_gemm(t["ws_ptr"], t["Wq"], t["sw"], M, N, K, t["Y"])
+
+    for i in range(5):
+        step(i)
+    torch.cuda.synchronize()
+    count = min(100, 4 * nsets)
+    step_ms = _events_ms(torch, step, 100 if M <= 2048 else 30)
+    rot_ms, gemm_ms = _graph_ms(torch, rotate, count), _graph_ms(torch, gemm, count)
+    flops = 2.0 * M * N * K
+    gemm_bytes_wo = N * K / 2.0 + 2.0 * M * K + 2.0 * M * N + 2.0 * N
+    rot_bytes = 4.0 * M * K
+    if M <= 64:
+        gbs = gemm_bytes_wo / (gemm_ms * 1e-3) / 1e9
+        roof = {"kernel": "wo_gemm_tc_kernel", "bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / pk["hbm_gbs"], "traffic": None, "ms_per_launch": gemm_ms,
+                "algorithmic_bytes": gemm_bytes_wo}
+    else:
+        tf = flops / (gemm_ms * 1e-3) / 1e12
+        roof = {"kernel": "wo_gemm_tc_kernel", "bound": "tensor", "achieved": tf, "peak": pk["bf16_tflops"],
+                "unit": "TFLOP/s", "frac": tf / pk["bf16_tflops"], "traffic": None, "ms_per_launch": gemm_ms,
+                "peak_source": f"{pk['source']} bf16 burst (fp16 runs at the same rate)", "algorithmic_flops": flops}
+        try:
+            A = [torch.randn((M, K), dtype=torch.float16, device="cuda") for _ in range(nsets)]
+            B = [torch.randn((N, K), dtype=torch.float16, device="cuda") for _ in range(min(nsets, 4))]
+            lib_ms = _events_ms(torch, lambda i: torch.matmul(A[i % nsets], B[i % len(B)].t()), 20)
+            lib_ms = _events_ms(torch, lambda i: torch.matmul(A[i % nsets], B[i % len(B)].t()), 20)
+            roof["yardstick"] = {"name": "torch.matmul fp16 x fp16 (library GEMM, dense fp16 weights)", "ms": lib_ms,
+                                 "tflops": flops / (lib_ms * 1e-3) / 1e12, "frac": lib_ms / gemm_ms}
+            del A, B
+        except Exception as exc:
+            sys.stderr.write(f"fp16 yardstick skipped: {exc}\n")
+    rgbs = rot_bytes / (rot_ms * 1e-3) / 1e9
+    out = {"M": M, "N": N, "K": K, "bits": bits, "ms_per_step": step_ms, "value": flops / (step_ms * 1e-3) / 1e12,
+           "unit": "TFLOP/s (2MNK per step)", "gemm": roof,
+           "rotate": {"kernel": rotate_kernel_name(w) + " (rotation only, fp16 out)", "bound": "hbm", "achieved": rgbs,
+                      "peak": pk["hbm_gbs"], "unit": "GB/s", "frac": rgbs / pk["hbm_gbs"], "traffic": None,
+                      "ms_per_launch": rot_ms, "algorithmic_bytes": rot_bytes},
+           "device_status": sq.sq_last_device_status()}
+    rot.close()
+    del sets
+    torch.cuda.empty_cache()
+    return out
+
+
+def grouped_entry(sq, torch, l2):
+    """A mixture-of-experts up-projection through sq_linear_grouped: 8 experts of 4096 -> 14336 (the shape of
+    Mixtral 8x7B's expert layers), 2048 tokens routed to two experts each by a seeded uniform draw, sorted
+    by expert; one rotation handle shared by the experts (they see the same input), weights per expert."""
+    E, K, N, n1, n2, T = 8, 4096, 14336, 64, 64, 2048
+    rng = np.random.default_rng(2024)
+    choice = np.stack([rng.permutation(E)[:2] for _ in range(T)])          # two distinct experts per token
+    counts = np.bincount(choice.reshape(-1), minlength=E)
+    offsets = np.concatenate([[0], np.cumsum(counts)]).astype(np.int64)
+    M = int(offsets[-1])
+    base = wl.small("moe_up", T, n1, n2, N, seed=88)
+    Xtok = wl.make_activations(base)
+    order = np.argsort(choice.reshape(-1), kind="stable")
+    X = Xtok[order // 2]                                                      # token rows, expert-sorted
+    rot = sq.sq_build_rotation(Xtok.astype(np.float32), n1, n2, seed=0)
+    wqs, sws = [], []
+    for e in range(E):
+        We = torch.from_numpy((0.02 * np.random.default_rng(100 + e).standard_normal((N, K))).astype(np.float16)).cuda()
+        q = torch.empty((N, K // 2), dtype=torch.uint8, device="cuda")
+        s_ = torch.empty((N,), dtype=torch.float16, device="cuda")
+        sq.sq_pack_weight(rot, We, N, K, q, s_)
+        wqs.append(q); sws.append(s_)
+        del We
+    torch.cuda.synchronize()
+    dX = torch.from_numpy(X).cuda()
+    Y = torch.empty((M, N), dtype=torch.float16, device="cuda")
+    ws_bytes = sq.sq_linear_workspace_bytes(M, K)
+    ws = torch.empty(ws_bytes + 256, dtype=torch.uint8, device="cuda")
+    wsp = ws.data_ptr() + (-ws.data_ptr()) % 256
+    rots = [rot] * E
+
+    def step(i):
+        sq.sq_linear_grouped(rots, offsets, dX, wqs, sws, N, K, wsp, ws_bytes, Y)
+
+    for i in range(3):
+        step(i)
+    torch.cuda.synchronize()
+    before = sq.sq_kernel_launch_count()
+    ms = _events_ms(torch, step, 20)
+    launches = (sq.sq_kernel_launch_count() - before) // 20
+    ops = 2.0 * M * N * K
+    out = {"experts": E, "tokens": T, "top_k": 2, "rows": M, "rows_per_expert": counts.tolist(), "N": N, "K": K,
+           "ms_per_step": ms, "value": ops / (ms * 1e-3) / 1e12, "unit": UNIT, "kernels_per_step": int(launches),
+           "note": "weights of the eight experts (235 MB packed) exceed L2, activations are re-read from L2",
+           "device_status": sq.sq_last_device_status()}
+    rot.close()
+    torch.cuda.empty_cache()
+    return out
+
+
 def run_ours(args, w):
     import torch
     from paper_2511_22316_b200 import binding as sq
@@ -624,6 +786,20 @@ def run_ours(args, w):
                     del ol
                 except Exception as exc:
                     per_workload[ow.name] = {"error": str(exc)}
+        # ---- the weight-only variant and the grouped layer, briefly ---------------------------------
+        variants = None
+        if world == 1 and not args.no_sweep:
+            variants = {"weight_only": {}, "grouped": None}
+            for ow, bits in ((wl.L7B_QKVO, 4), (wl.L7B_QKVO, 3), (wl.L70B_GATEUP, 4), (wl.decode_up(16), 4),
+                             (wl.decode_down(16), 4)):
+                try:
+                    variants["weight_only"][f"{ow.name}_w{bits}a16"] = weight_only_entry(sq, torch, ow, bits, pk, l2)
+                except Exception as exc:
+                    variants["weight_only"][f"{ow.name}_w{bits}a16"] = {"error": str(exc)}
+            try:
+                variants["grouped"] = grouped_entry(sq, torch, l2)
+            except Exception as exc:
+                variants["grouped"] = {"error": str(exc)}
         sampler.stop()
 
         line = {
@@ -654,6 +830,8 @@ def run_ours(args, w):
             line["cpu_baseline"] = cpu
         if per_workload is not None:
             line["per_workload"] = per_workload
+        if variants is not None:
+            line["variants"] = variants
         print(json.dumps(line))
     if dist is not None:
         dist.barrier()

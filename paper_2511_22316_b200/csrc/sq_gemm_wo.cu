@@ -275,6 +275,262 @@ wo_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_const
   }
 }
 
+// Decode-sized batches (M <= 64): the product is bound by reading the packed weights once, so the
+// operands swap roles.  A tile is 128 OUTPUT CHANNELS (the MMA's M and the accumulator's lanes), the
+// tokens are the MMA's N (16, 32 or 64): the token tiles are a few KB straight from TMA, and an MMA
+// with a narrow N takes a third of the time.  The widened weights never touch shared memory: each
+// thread of a converter group reads the 128 packed bytes of "its" channel from the staging ring,
+// widens them in registers and stores them into a ring in tensor memory (tcgen05.st), from where the
+// MMA takes its A operand -- through shared memory the fp16 operand alone cost 128 KB of traffic per
+// 256 channels and bounded the kernel (20 us on 14336 x 4096 against 28.7 us with 64-channel stages,
+// whose hand-overs cost 920 cycles each).  A stage is a whole staging block: 256 channels, sixteen
+// MMAs.  Two converter groups alternate stages (a third group and a third operand stage changed
+// nothing).  What bounds a stage now, at about 1300 cycles: not the MMAs (issuing half of them changes
+// nothing) and only a little the widening arithmetic (dropping it saves 15 %); what remains is moving
+// the 64 KB fp16 operand of a stage into tensor memory.  K is not split over CTAs: a layer with few
+// output channels (4096: 32 tiles) keeps only that many SMs busy.  The accumulator holds one channel
+// per thread and the tokens along its registers; a warp's stores of one token cover 32 consecutive
+// channels.
+constexpr int WOD_CONV_GROUPS = 2;
+constexpr int WOD_CONV_WARPS = 4 * WOD_CONV_GROUPS;
+constexpr int WOD_THREADS = (2 + WOD_CONV_WARPS + WO_EPI_WARPS) * 32;
+constexpr int WOD_A_STAGES = 2;           // tensor-memory operand stages of 128 columns (256 fp16 channels)
+constexpr int WOD_A_COL0 = 128;           // accumulators: columns [0, 2 NT); operand ring: [128, 384)
+
+template <int NT, int ST, int SS>
+struct WoDecSmem {
+  static constexpr int T_KB = NT * 128;               // tokens x 64 channels fp16 (one k-block)
+  static constexpr int T_TILE = 4 * T_KB;             // a stage: four k-blocks
+  static constexpr int W_ST = 128 * 128;              // 128 channels x 256 packed codes
+  static constexpr int OFF_T = 0;
+  static constexpr int OFF_W_ST = OFF_T + ST * T_TILE;
+  static constexpr int OFF_BAR = OFF_W_ST + SS * W_ST;
+  static constexpr int NUM_BARS = 2 * ST + 2 * SS + 2 * WOD_A_STAGES + 4;
+  static constexpr int OFF_TMEM = OFF_BAR + NUM_BARS * 8;
+  static constexpr int TOTAL = OFF_TMEM + 16;
+  static constexpr int DYN_BYTES = TOTAL + 1024;
+};
+
+template <int NT, int ST, int SS>
+__global__ void __launch_bounds__(WOD_THREADS, 1)
+wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_constant__ CUtensorMap tmap_w,
+                      const __half* __restrict__ sw, int M, int N, int K, __half* __restrict__ Y) {
+  using L = WoDecSmem<NT, ST, SS>;
+  griddep_launch_dependents();
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+  uint64_t* t_full = bars;
+  uint64_t* t_empty = t_full + ST;
+  uint64_t* st_full = t_empty + ST;
+  uint64_t* st_empty = st_full + SS;
+  uint64_t* a_full = st_empty + SS;
+  uint64_t* a_empty = a_full + WOD_A_STAGES;
+  uint64_t* tmem_full = a_empty + WOD_A_STAGES;   // [2]
+  uint64_t* tmem_empty = tmem_full + 2;           // [2]
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_TMEM);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const int num_kb = K / 64;
+  const int num_sb = (num_kb + 3) / 4;        // stages per tile (the last may hold fewer than four k-blocks)
+  const int num_tiles = (N + 127) / 128;
+  const uint32_t limit = wait_limit();
+
+  // The weights do not depend on the kernel before this one: the first ring-full of them is requested
+  // before anything else is set up and before that kernel's completion is awaited.
+  int pre = 0;
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmap_w);
+    for (int s = 0; s < SS; ++s) mbar_init(&st_full[s], 1);
+    mbar_fence_init();
+    {
+      int t = blockIdx.x, sb = 0;
+      while (pre < SS && t < num_tiles) {
+        mbar_arrive_expect_tx(&st_full[pre], L::W_ST);
+        tma_load_2d(smem + L::OFF_W_ST + pre * L::W_ST, &tmap_w, &st_full[pre], sb * 128, t * 128);
+        ++pre;
+        if (++sb >= num_sb) {
+          sb = 0;
+          t += gridDim.x;
+        }
+      }
+    }
+    tma_prefetch_desc(&tmap_z);
+    for (int s = 0; s < ST; ++s) {
+      mbar_init(&t_full[s], 1);
+      mbar_init(&t_empty[s], 1);
+    }
+    for (int s = 0; s < SS; ++s) mbar_init(&st_empty[s], 4);          // the four warps of one converter group
+    for (int s = 0; s < WOD_A_STAGES; ++s) {
+      mbar_init(&a_full[s], 4);
+      mbar_init(&a_empty[s], 1);
+    }
+    for (int b = 0; b < 2; ++b) {
+      mbar_init(&tmem_full[b], 1);
+      mbar_init(&tmem_empty[b], WO_EPI_WARPS);
+    }
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc(tmem_slot, 512);
+    tmem_relinquish();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();                                     // Z16 may come from the kernel launched before this one
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------------------
+    if (lane == 0) {
+      uint32_t sit = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+        for (int sb = 0; sb < num_sb && ok; ++sb, ++sit) {
+          if (sit >= static_cast<uint32_t>(pre)) {          // the first `pre` blocks are on their way already
+            const int ss = sit % SS;
+            ok = mbar_wait(&st_empty[ss], ((sit / SS) & 1) ^ 1, WO_ST_EMPTY, limit);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&st_full[ss], L::W_ST);
+            tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, &tmap_w, &st_full[ss], sb * 128, tile * 128);
+          }
+          const int st = sit % ST;
+          const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
+          ok = mbar_wait(&t_empty[st], ((sit / ST) & 1) ^ 1, WO_A_EMPTY, limit);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&t_full[st], static_cast<uint32_t>(nk * L::T_KB));
+          for (int h = 0; h < nk; ++h)
+            tma_load_2d(smem + L::OFF_T + st * L::T_TILE + h * L::T_KB, &tmap_z, &t_full[st], (4 * sb + h) * 64, 0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer --------------------------------------------
+    if (elect_one()) {
+      constexpr uint32_t idesc = umma_idesc(/*c=f32*/ 1, /*a=f16*/ 0, /*b=f16*/ 0, 128, NT);
+      // descriptors of a stage differ from the ring's first by constants in the start-address field
+      // (16-byte units, no carry out of it): formed once, the stage's MMAs unrolled
+      const uint64_t t_desc0 = umma_desc_sw128(smem_u32(smem + L::OFF_T));
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+        const uint32_t b = tcount & 1;
+        ok = mbar_wait(&tmem_empty[b], ((tcount >> 1) & 1) ^ 1, WO_TMEM_EMPTY, limit);
+        if (!ok) break;
+        tc_fence_after_sync();
+        const uint32_t tmem_d = tmem_base + b * NT;
+        for (int sb = 0; sb < num_sb; ++sb, ++it) {
+          const int st = it % ST, sa = it % WOD_A_STAGES;
+          const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
+          ok = mbar_wait(&t_full[st], (it / ST) & 1, WO_A_FULL, limit) &&
+               mbar_wait(&a_full[sa], (it / WOD_A_STAGES) & 1, WO_B_FULL, limit);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t a_tmem = tmem_base + WOD_A_COL0 + sa * 128;
+          const uint64_t td = t_desc0 + static_cast<uint64_t>((st * L::T_TILE) >> 4);
+#pragma unroll
+          for (int h = 0; h < 4; ++h) {
+            if (h < nk) {
+#pragma unroll
+              for (int k = 0; k < 4; ++k)         // K = 16 fp16: eight 32-bit columns of A, 32 bytes of a token row
+                umma_f16_ts(tmem_d, a_tmem + 32 * h + 8 * k, td + ((h * L::T_KB + k * 32) >> 4), idesc,
+                            (sb | h | k) != 0 ? 1u : 0u);
+            }
+          }
+          umma_commit(&t_empty[st]);
+          umma_commit(&a_empty[sa]);
+        }
+        umma_commit(&tmem_full[b]);
+      }
+    }
+  } else if (warp < 2 + WOD_CONV_WARPS) {
+    // ------------------------------ weight converters: staging -> registers -> tensor memory ------
+    const int q = warp & 3;
+    const int grp = (warp - 2) >> 2;                    // this group's stages: it % WOD_CONV_GROUPS == grp
+    const int r = q * 32 + lane;                        // channel of the tile = TMEM lane
+    const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
+      for (int sb = 0; sb < num_sb && ok; ++sb, ++it) {
+        if ((it % WOD_CONV_GROUPS) != static_cast<uint32_t>(grp)) continue;
+        const int ss = it % SS, sa = it % WOD_A_STAGES;
+        const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
+        ok = mbar_wait(&st_full[ss], (it / SS) & 1, WO_ST_FULL, limit);
+        if (!ok) break;
+        const unsigned char* row = smem + L::OFF_W_ST + ss * L::W_ST + r * 128;
+        uint4 w[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) w[c] = *reinterpret_cast<const uint4*>(row + ((c ^ (r & 7)) << 4));
+        ok = mbar_wait(&a_empty[sa], ((it / WOD_A_STAGES) & 1) ^ 1, WO_B_EMPTY, limit);
+        if (!ok) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {                   // k-block h: chunks 2h, 2h+1 -> 32 columns
+          if (h < nk) {
+            uint32_t v[32];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+              const uint4 x = w[2 * h + j];
+              const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+              for (int g = 0; g < 4; ++g)
+#pragma unroll
+                for (int p = 0; p < 4; ++p) v[16 * j + 4 * g + p] = widen_pair(xs[g], p);
+            }
+            tmem_st_32x32b_x32(tmem_base + lane_addr + WOD_A_COL0 + sa * 128 + h * 32, v);
+          }
+        }
+        tmem_wait_st();
+        tc_fence_before_sync();
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive(&a_full[sa]);
+          mbar_arrive(&st_empty[ss]);
+        }
+      }
+    }
+  } else {
+    // ------------------------------ epilogue warps ------------------------------------------
+    const int quarter = warp & 3;
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+      const uint32_t b = tcount & 1;
+      const int ch = tile * 128 + quarter * 32 + lane;
+      const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;
+      ok = mbar_wait(&tmem_full[b], (tcount >> 1) & 1, WO_TMEM_FULL, limit);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t tmem_d = tmem_base + b * NT + (static_cast<uint32_t>(quarter * 32) << 16);
+#pragma unroll
+      for (int c = 0; c < NT / 16; ++c) {
+        uint32_t r[16];
+        tmem_ld_32x32b_x16(tmem_d + c * 16, r);
+        tmem_wait_ld();
+        if (ch < N) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int tok = c * 16 + e;
+            if (tok < M) Y[static_cast<size_t>(tok) * N + ch] = __float2half_rn(__uint_as_float(r[e]) * swv);
+          }
+        }
+      }
+      tc_fence_before_sync();
+      __syncwarp();
+      if (lane == 0) mbar_arrive(&tmem_empty[b]);
+    }
+  }
+
+  tc_fence_before_sync();
+  __syncthreads();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc(tmem_base, 512);
+  }
+}
+
 // Plain kernel for shapes the tensor-core path does not take (K % 64 != 0, N % 8 != 0): one thread per
 // output channel, fp32 multiply-adds in channel order; gridDim.y strides over the token rows.
 __global__ void wo_gemm_simple_kernel(const __half* __restrict__ Z16, const uint8_t* __restrict__ Wq,
@@ -343,12 +599,47 @@ sq_status_t launch_wo_tc(const void* Z16, const void* Wq, const void* sw, int M,
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
 }
 
+template <int NT, int ST, int SS>
+sq_status_t launch_wo_decode(const void* Z16, const void* Wq, const void* sw, int M, int N, int K, void* Y,
+                             cudaStream_t s) {
+  using L = WoDecSmem<NT, ST, SS>;
+  static_assert(L::DYN_BYTES <= 227 * 1024, "shared-memory plan does not fit");
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return SQ_ERR_CUDA;
+  CUtensorMap mz, mw;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(M)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
+  const cuuint32_t box[2] = {64, NT};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&mz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(Z16), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return SQ_ERR_CUDA;
+  if (!make_packed_map(&mw, Wq, N, K / 2, 128)) return SQ_ERR_CUDA;
+  auto kern = wo_gemm_decode_kernel<NT, ST, SS>;
+  if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), L::DYN_BYTES)) return SQ_ERR_CUDA;
+  const int sms = sm_count();
+  if (sms <= 0) return SQ_ERR_CUDA;
+  const int tiles = (N + 127) / 128;
+  const int grid = tiles < sms ? tiles : sms;
+  const cudaError_t err = launch_maybe_pdl(kern, dim3(grid), dim3(WOD_THREADS), L::DYN_BYTES, s, mz, mw,
+                                           static_cast<const __half*>(sw), M, N, K, static_cast<__half*>(Y));
+  count_launch();
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
+}
+
 }  // namespace
 
 sq_status_t launch_wo_gemm(const void* Z16, const void* Wq, const void* sw, int64_t M, int64_t N, int64_t K, void* Y,
                            cudaStream_t s) {
   if (M == 0 || N == 0) return SQ_OK;
   const bool tc_ok = (K % 64 == 0) && (N % 8 == 0);
+  if (tc_ok && M <= 64 && N >= 128) {
+    // decode-sized batches: weights as the M operand, a deep ring of packed weights in flight
+    if (M <= 16) return launch_wo_decode<16, 4, 8>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
+    if (M <= 32) return launch_wo_decode<32, 4, 8>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
+    return launch_wo_decode<64, 3, 6>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
+  }
   if (tc_ok) {
     // 256-channel tiles where they fill the device with enough token rows to use them
     if (M > 128 && N >= 256 * 64) return launch_wo_tc<256, 4, 2, 3>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
