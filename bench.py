@@ -6,6 +6,7 @@ the named workload.  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
                   [--structured-r2] [--fuse-decode] [--no-sweep] [--no-cpu-baseline] [--quick]
+                  [--variants-only]
 
 After the headline workload the default run also times every other benchmark workload briefly and
 reports them under "per_workload" of the same line, and the weight-only variant (W4A16 / W3A16) and the
@@ -494,7 +495,7 @@ def _events_ms(torch, fn, count):
     return e0.elapsed_time(e1) / count
 
 
-def weight_only_entry(sq, torch, w, bits, pk, l2):
+def weight_only_entry(sq, torch, w, bits, pk, l2, quick=False):
     """The weight-only layer (fp16 rotated activations x b-bit weights) on one workload: the step through
     sq_linear_wo, its two kernels from graph replays, roofline fractions, and a library fp16 GEMM of the
     same shape (torch.matmul, no unpacking, no scaling) as the yardstick."""
@@ -533,8 +534,8 @@ def weight_only_entry(sq, torch, w, bits, pk, l2):
     for i in range(5):
         step(i)
     torch.cuda.synchronize()
-    count = min(100, 4 * nsets)
-    step_ms = _events_ms(torch, step, 100 if M <= 2048 else 30)
+    count = 4 if quick else min(100, 4 * nsets)
+    step_ms = _events_ms(torch, step, 4 if quick else (100 if M <= 2048 else 30))
     rot_ms, gemm_ms = _graph_ms(torch, rotate, count), _graph_ms(torch, gemm, count)
     flops = 2.0 * M * N * K
     gemm_bytes_wo = N * K / 2.0 + 2.0 * M * K + 2.0 * M * N + 2.0 * N
@@ -550,6 +551,8 @@ def weight_only_entry(sq, torch, w, bits, pk, l2):
                 "unit": "TFLOP/s", "frac": tf / pk["bf16_tflops"], "traffic": None, "ms_per_launch": gemm_ms,
                 "peak_source": f"{pk['source']} bf16 burst (fp16 runs at the same rate)", "algorithmic_flops": flops}
         try:
+            if quick:
+                raise RuntimeError("quick run")
             A = [torch.randn((M, K), dtype=torch.float16, device="cuda") for _ in range(nsets)]
             B = [torch.randn((N, K), dtype=torch.float16, device="cuda") for _ in range(min(nsets, 4))]
             lib_ms = _events_ms(torch, lambda i: torch.matmul(A[i % nsets], B[i % len(B)].t()), 20)
@@ -620,6 +623,21 @@ def grouped_entry(sq, torch, l2):
     rot.close()
     torch.cuda.empty_cache()
     return out
+
+
+def run_variants_only(args, w):
+    import torch
+    from paper_2511_22316_b200 import binding as sq
+    from paper_2511_22316_b200 import build as sqbuild
+    if not torch.cuda.is_available():
+        raise RuntimeError("bench.py needs a CUDA device: the hot path has no CPU fallback")
+    torch.cuda.set_device(0)
+    sqbuild.build()
+    sq.load()
+    l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    entry = weight_only_entry(sq, torch, w, 4, peaks(), l2, quick=args.quick)
+    print(json.dumps({"variants": {"weight_only": {f"{w.name}_w4a16": entry}}, "n_gpus": 1, "data": "synthetic"}))
+    return 0
 
 
 def run_ours(args, w):
@@ -860,6 +878,9 @@ def main():
     ap.add_argument("--quick", action="store_true",
                     help="the K timed steps and the per-kernel attribution only: no sustained pass, no yardsticks, "
                          "no per-workload table, no CPU baseline (for profiler runs)")
+    ap.add_argument("--variants-only", action="store_true",
+                    help="time only the weight-only variant of the named workload (W4A16) and print it under "
+                         "\"variants\" (for profiler runs of those kernels)")
     args = ap.parse_args()
     if args.quick:
         args.no_sweep = args.no_cpu_baseline = True
@@ -868,6 +889,8 @@ def main():
     w = wl.by_name(args.workload)
     if args.impl == "reference":
         return run_reference(args, w)
+    if args.variants_only:
+        return run_variants_only(args, w)
     return run_ours(args, w)
 
 

@@ -15,7 +15,8 @@
 // (u ^ 0x6408) read as fp16 is 1032 + c, and one exact fp16 subtraction of 1032 leaves c.  The
 // weight-only storage order puts channels (2s, 2s+1) of every eight at nibble positions (s, s+4) of a
 // 32-bit word, so that (word >> 4s) & 0x000F000F is one such pair in the two halves of a register:
-// a shift, one three-input logic operation and one half2 subtraction per two weights.
+// a shift, one three-input logic operation and one half2 subtraction per two weights (half of the pairs
+// need no shift: see widen_high).
 #include <cuda.h>
 #include <cuda_fp16.h>
 
@@ -49,15 +50,31 @@ struct WoSmem {
   static constexpr int DYN_BYTES = TOTAL + 1024;      // slack for the 1024-byte alignment
 };
 
-// Two weights (channels 2s, 2s+1 of the word's eight) as a half2.
-__device__ __forceinline__ uint32_t widen_pair(uint32_t word, int s) {
-  const uint32_t x = ((word >> (4 * s)) & 0x000F000Fu) ^ 0x64086408u;
+// Eight weights of one packed word as four half2 (channel pairs (0,1), (2,3), (4,5), (6,7)).  Nibble
+// positions 0 and 4 sit in the low four mantissa bits of the two halves: (w & 0x000F000F) ^ 0x64086408 is
+// (1032 + code) twice, minus 1032.  Positions 1 and 5 sit four bits higher: (w & 0x00F000F0) ^ 0x64806480
+// is 1024 + 16 (code + 8), and one fused multiply-add, x / 16 - 72, leaves the code -- exact in fp16, and
+// it spares the shift (the logic pipe is the busier one here).  One shift by 8 brings positions 2, 3, 6, 7
+// to where 0, 1, 4, 5 were.
+__device__ __forceinline__ uint32_t widen_low(uint32_t w) {
+  const uint32_t x = (w & 0x000F000Fu) ^ 0x64086408u;
   const __half2 v = __hsub2(*reinterpret_cast<const __half2*>(&x), __half2half2(__ushort_as_half(0x6408)));
   return *reinterpret_cast<const uint32_t*>(&v);
 }
+__device__ __forceinline__ uint32_t widen_high(uint32_t w) {
+  const uint32_t x = (w & 0x00F000F0u) ^ 0x64806480u;
+  const __half2 v = __hfma2(*reinterpret_cast<const __half2*>(&x), __half2half2(__ushort_as_half(0x2C00)),   // 1/16
+                            __half2half2(__ushort_as_half(0xD480)));                                      // -72
+  return *reinterpret_cast<const uint32_t*>(&v);
+}
+__device__ __forceinline__ uint32_t widen_pair(uint32_t word, int s) {
+  const uint32_t w = (s & 2) ? (word >> 8) : word;
+  return (s & 1) ? widen_high(w) : widen_low(w);
+}
 
 __device__ __forceinline__ uint4 widen_word(uint32_t word) {
-  return make_uint4(widen_pair(word, 0), widen_pair(word, 1), widen_pair(word, 2), widen_pair(word, 3));
+  const uint32_t w8 = word >> 8;
+  return make_uint4(widen_low(word), widen_high(word), widen_low(w8), widen_high(w8));
 }
 
 // Widens k-block h (64 channels = 32 packed bytes) of BN staged rows into BN x 64 fp16.  Staging and
@@ -475,9 +492,13 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
               const uint4 x = w[2 * h + j];
               const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
 #pragma unroll
-              for (int g = 0; g < 4; ++g)
-#pragma unroll
-                for (int p = 0; p < 4; ++p) v[16 * j + 4 * g + p] = widen_pair(xs[g], p);
+              for (int g = 0; g < 4; ++g) {
+                const uint4 f = widen_word(xs[g]);
+                v[16 * j + 4 * g + 0] = f.x;
+                v[16 * j + 4 * g + 1] = f.y;
+                v[16 * j + 4 * g + 2] = f.z;
+                v[16 * j + 4 * g + 3] = f.w;
+              }
             }
             tmem_st_32x32b_x32(tmem_base + lane_addr + WOD_A_COL0 + sa * 128 + h * 32, v);
           }
@@ -641,8 +662,10 @@ sq_status_t launch_wo_gemm(const void* Z16, const void* Wq, const void* sw, int6
     return launch_wo_decode<64, 3, 6>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
   }
   if (tc_ok) {
-    // 256-channel tiles where they fill the device with enough token rows to use them
-    if (M > 128 && N >= 256 * 64) return launch_wo_tc<256, 4, 2, 3>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
+    // 256-channel tiles wherever there are enough token rows and channels: the kernel is bound by shared
+    // memory (the fp16 operand is written and read there), and a wider tile moves fewer bytes per flop
+    // (2048 x 4096 x 4096: 103 us with 128-channel tiles)
+    if (M > 128 && N >= 256) return launch_wo_tc<256, 4, 2, 3>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
     return launch_wo_tc<128, 6, 2, 4>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
   }
   dim3 block(128), grid((unsigned)((N + 127) / 128), (unsigned)(M < 65535 ? M : 65535));
