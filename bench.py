@@ -51,6 +51,10 @@ NCU_TRAFFIC = {
     ("gemm", "llama3_8b_down_decode_m16"): 29519616,        # w4a4_gemm_decode_kernel, K over clusters of 4
     ("gemm", "llama3_8b_up_decode_m1"): 29409024,           # w4a4_gemv_kernel
     ("rotate_quant", "llama2_7b_down_prefill"): 45412608,   # rotate_quant_pair_kernel
+    ("rotate_quant", "llama2_70b_gateup_prefill"): 69889536,   # rotate_quant_tc_kernel, n2 = 128
+    ("rotate_quant", "llama2_70b_down_prefill"): 275649024,    # rotate_quant_pair_kernel, n2 = 128
+    ("wo_gemm", "llama3_8b_up_decode_m16"): 29547264,       # wo_gemm_decode_kernel (W4A16)
+    ("wo_gemm", "llama2_7b_qkvo_prefill"): 25196544,        # wo_gemm_tc_kernel (W4A16; Y stayed in L2)
 }
 
 
@@ -542,13 +546,15 @@ def weight_only_entry(sq, torch, w, bits, pk, l2, quick=False):
     rot_bytes = 4.0 * M * K
     if M <= 64:
         gbs = gemm_bytes_wo / (gemm_ms * 1e-3) / 1e9
-        roof = {"kernel": "wo_gemm_tc_kernel", "bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
-                "frac": gbs / pk["hbm_gbs"], "traffic": None, "ms_per_launch": gemm_ms,
+        roof = {"kernel": "wo_gemv_kernel" if M <= 2 else "wo_gemm_decode_kernel", "bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+                "frac": gbs / pk["hbm_gbs"], "traffic": NCU_TRAFFIC.get(("wo_gemm", w.name)) if bits == 4 else None,
+                "ms_per_launch": gemm_ms,
                 "algorithmic_bytes": gemm_bytes_wo}
     else:
         tf = flops / (gemm_ms * 1e-3) / 1e12
         roof = {"kernel": "wo_gemm_tc_kernel", "bound": "tensor", "achieved": tf, "peak": pk["bf16_tflops"],
-                "unit": "TFLOP/s", "frac": tf / pk["bf16_tflops"], "traffic": None, "ms_per_launch": gemm_ms,
+                "unit": "TFLOP/s", "frac": tf / pk["bf16_tflops"],
+                "traffic": NCU_TRAFFIC.get(("wo_gemm", w.name)) if bits == 4 else None, "ms_per_launch": gemm_ms,
                 "peak_source": f"{pk['source']} bf16 burst (fp16 runs at the same rate)", "algorithmic_flops": flops}
         try:
             if quick:
@@ -808,7 +814,8 @@ def run_ours(args, w):
         variants = None
         if world == 1 and not args.no_sweep:
             variants = {"weight_only": {}, "grouped": None}
-            for ow, bits in ((wl.L7B_QKVO, 4), (wl.L7B_QKVO, 3), (wl.L70B_GATEUP, 4), (wl.decode_up(16), 4),
+            for ow, bits in ((wl.L7B_QKVO, 4), (wl.L7B_QKVO, 3), (wl.L7B_GATEUP, 4), (wl.L70B_GATEUP, 4),
+                             (wl.decode_up(1), 4), (wl.decode_down(1), 4), (wl.decode_up(16), 4),
                              (wl.decode_down(16), 4)):
                 try:
                     variants["weight_only"][f"{ow.name}_w{bits}a16"] = weight_only_entry(sq, torch, ow, bits, pk, l2)

@@ -20,6 +20,8 @@
 #include <cuda.h>
 #include <cuda_fp16.h>
 
+#include <algorithm>
+
 #include "sq_internal.h"
 #include "sq_ptx.cuh"
 
@@ -552,6 +554,120 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
   }
 }
 
+// One or two tokens: dot products on the CUDA cores.  The product is pure streaming then (29 MB of
+// packed weights against a few MFLOP), and the tensor-core forms pay more in hand-overs than the read
+// costs.  Each warp takes four weight rows at a time; every lane reads 16-byte pieces of them straight
+// from global memory (coalesced, several in flight), widens the nibbles to half2 as above, converts to
+// fp32 and multiplies with the tokens, which the CTA holds in shared memory as fp32.  Accumulation is
+// fp32 throughout; a row's sum is completed by one warp (shuffle reduction): deterministic.
+constexpr int WOV_ROWS = 4, WOV_UNROLL = 2;
+
+template <int MT>
+__global__ void __launch_bounds__(512)
+wo_gemv_kernel(const __half* __restrict__ Z16, const uint8_t* __restrict__ Wq, const __half* __restrict__ sw, int M,
+               int N, int K, __half* __restrict__ Y) {
+  griddep_launch_dependents();
+  griddep_wait();                                        // Z16 may come from the kernel launched before this one
+  // Tokens as fp32, laid out [token][word of a piece g][half h][piece c][4]: the lanes of a warp work on
+  // consecutive pieces c, so their 16-byte reads for one (g, h) are contiguous (no bank conflicts).
+  extern __shared__ __align__(16) float zs[];
+  const int nchunk = K / 32;                             // 16-byte pieces of packed weights per row
+  for (int i = threadIdx.x; i < MT * (K / 8); i += blockDim.x) {
+    const int t = i / (K / 8), c = i % (K / 8);
+    uint4 v = make_uint4(0u, 0u, 0u, 0u);
+    if (t < M) v = __ldg(reinterpret_cast<const uint4*>(Z16 + static_cast<size_t>(t) * K) + c);
+    const __half2* h = reinterpret_cast<const __half2*>(&v);
+    const float2 a = __half22float2(h[0]), b = __half22float2(h[1]), c2 = __half22float2(h[2]), d = __half22float2(h[3]);
+    const int piece = c >> 2, g = c & 3;
+    float* base = zs + static_cast<size_t>(t) * K;
+    *reinterpret_cast<float4*>(base + ((g * 2 + 0) * nchunk + piece) * 4) = make_float4(a.x, a.y, b.x, b.y);
+    *reinterpret_cast<float4*>(base + ((g * 2 + 1) * nchunk + piece) * 4) = make_float4(c2.x, c2.y, d.x, d.y);
+  }
+  __syncthreads();
+
+  const int lane = threadIdx.x & 31;
+  const int warps_per_cta = blockDim.x >> 5;
+  const long long ntask = (N + WOV_ROWS - 1) / WOV_ROWS;
+  const long long wstride = static_cast<long long>(gridDim.x) * warps_per_cta;
+  for (long long task = static_cast<long long>(threadIdx.x >> 5) * gridDim.x + blockIdx.x; task < ntask; task += wstride) {
+    const int row0 = static_cast<int>(task) * WOV_ROWS;
+    float acc[WOV_ROWS][MT];
+#pragma unroll
+    for (int r = 0; r < WOV_ROWS; ++r)
+#pragma unroll
+      for (int t = 0; t < MT; ++t) acc[r][t] = 0.0f;
+    const uint4* wrow[WOV_ROWS];
+#pragma unroll
+    for (int r = 0; r < WOV_ROWS; ++r)
+      wrow[r] = reinterpret_cast<const uint4*>(Wq + static_cast<size_t>(min(row0 + r, N - 1)) * (K / 2));
+    for (int c0 = lane; c0 < nchunk; c0 += 32 * WOV_UNROLL) {
+      uint4 wv[WOV_UNROLL][WOV_ROWS];
+#pragma unroll
+      for (int u = 0; u < WOV_UNROLL; ++u) {
+        const int c = c0 + 32 * u;
+#pragma unroll
+        for (int r = 0; r < WOV_ROWS; ++r)
+          wv[u][r] = (c < nchunk) ? __ldcs(wrow[r] + c) : make_uint4(0u, 0u, 0u, 0u);
+      }
+#pragma unroll
+      for (int u = 0; u < WOV_UNROLL; ++u) {
+        const int c = c0 + 32 * u;
+        if (c < nchunk) {
+#pragma unroll
+          for (int g = 0; g < 4; ++g) {                   // word g of the piece: channels 32 c + 8 g .. + 7
+            float zf[MT][8];
+#pragma unroll
+            for (int t = 0; t < MT; ++t) {
+              const float4 z0 = *reinterpret_cast<const float4*>(zs + static_cast<size_t>(t) * K + ((g * 2 + 0) * nchunk + c) * 4);
+              const float4 z1 = *reinterpret_cast<const float4*>(zs + static_cast<size_t>(t) * K + ((g * 2 + 1) * nchunk + c) * 4);
+              zf[t][0] = z0.x; zf[t][1] = z0.y; zf[t][2] = z0.z; zf[t][3] = z0.w;
+              zf[t][4] = z1.x; zf[t][5] = z1.y; zf[t][6] = z1.z; zf[t][7] = z1.w;
+            }
+#pragma unroll
+            for (int r = 0; r < WOV_ROWS; ++r) {
+              const uint32_t word = g == 0 ? wv[u][r].x : (g == 1 ? wv[u][r].y : (g == 2 ? wv[u][r].z : wv[u][r].w));
+              const uint4 f = widen_word(word);
+              const float2 w01 = __half22float2(*reinterpret_cast<const __half2*>(&f.x));
+              const float2 w23 = __half22float2(*reinterpret_cast<const __half2*>(&f.y));
+              const float2 w45 = __half22float2(*reinterpret_cast<const __half2*>(&f.z));
+              const float2 w67 = __half22float2(*reinterpret_cast<const __half2*>(&f.w));
+#pragma unroll
+              for (int t = 0; t < MT; ++t) {
+                float a = acc[r][t];
+                a = fmaf(zf[t][0], w01.x, a); a = fmaf(zf[t][1], w01.y, a);
+                a = fmaf(zf[t][2], w23.x, a); a = fmaf(zf[t][3], w23.y, a);
+                a = fmaf(zf[t][4], w45.x, a); a = fmaf(zf[t][5], w45.y, a);
+                a = fmaf(zf[t][6], w67.x, a); a = fmaf(zf[t][7], w67.y, a);
+                acc[r][t] = a;
+              }
+            }
+          }
+        }
+      }
+    }
+#pragma unroll
+    for (int r = 0; r < WOV_ROWS; ++r)
+#pragma unroll
+      for (int t = 0; t < MT; ++t) {
+        float a = acc[r][t];
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) a += __shfl_xor_sync(0xffffffffu, a, o);
+        acc[r][t] = a;
+      }
+    if (lane < WOV_ROWS * MT) {
+      const int r = lane / MT, t = lane % MT;
+      float a = 0.0f;
+#pragma unroll
+      for (int rr = 0; rr < WOV_ROWS; ++rr)
+#pragma unroll
+        for (int tt = 0; tt < MT; ++tt)
+          if (rr == r && tt == t) a = acc[rr][tt];
+      const int row = row0 + r;
+      if (row < N && t < M) Y[static_cast<size_t>(t) * N + row] = __float2half_rn(a * __half2float(__ldg(sw + row)));
+    }
+  }
+}
+
 // Plain kernel for shapes the tensor-core path does not take (K % 64 != 0, N % 8 != 0): one thread per
 // output channel, fp32 multiply-adds in channel order; gridDim.y strides over the token rows.
 __global__ void wo_gemm_simple_kernel(const __half* __restrict__ Z16, const uint8_t* __restrict__ Wq,
@@ -649,12 +765,34 @@ sq_status_t launch_wo_decode(const void* Z16, const void* Wq, const void* sw, in
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
 }
 
+template <int MT>
+sq_status_t launch_wo_gemv(const void* Z16, const void* Wq, const void* sw, int M, int N, int K, void* Y, cudaStream_t s) {
+  const int sms = sm_count();
+  if (sms <= 0) return SQ_ERR_CUDA;
+  const long long ntask = (N + WOV_ROWS - 1) / WOV_ROWS;
+  const int warps = gemv_warps(ntask, sms);
+  const int smem = MT * K * 4;
+  auto kern = wo_gemv_kernel<MT>;
+  if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), smem)) return SQ_ERR_CUDA;
+  const unsigned grid = static_cast<unsigned>(std::min<long long>(sms, (ntask + warps - 1) / warps));
+  const cudaError_t err = launch_maybe_pdl(kern, dim3(grid), dim3(warps * 32), static_cast<size_t>(smem), s,
+                                           static_cast<const __half*>(Z16), static_cast<const uint8_t*>(Wq),
+                                           static_cast<const __half*>(sw), M, N, K, static_cast<__half*>(Y));
+  count_launch();
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
+}
+
 }  // namespace
 
 sq_status_t launch_wo_gemm(const void* Z16, const void* Wq, const void* sw, int64_t M, int64_t N, int64_t K, void* Y,
                            cudaStream_t s) {
   if (M == 0 || N == 0) return SQ_OK;
   const bool tc_ok = (K % 64 == 0) && (N % 8 == 0);
+  if (M <= 2 && K % 32 == 0 && static_cast<int64_t>(M) * K * 4 <= 200 * 1024) {
+    // one or two tokens: dot products on the CUDA cores
+    if (M == 1) return launch_wo_gemv<1>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
+    return launch_wo_gemv<2>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
+  }
   if (tc_ok && M <= 64 && N >= 128) {
     // decode-sized batches: weights as the M operand, a deep ring of packed weights in flight
     if (M <= 16) return launch_wo_decode<16, 4, 8>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);

@@ -144,6 +144,8 @@ def _run_wo_gemm(sq, Z16, codes, sw):
 
 WO_GEMM_SHAPES = [(1, 128, 64), (5, 136, 192), (64, 264, 256), (128, 128, 320), (130, 384, 1024), (200, 8, 4096),
                   (33, 5120, 512), (257, 16392, 128), (300, 16640, 448),
+                  # one or two tokens: the dot-product kernel (ragged row count, long rows)
+                  (2, 134, 4096), (1, 263 * 8, 14336), (2, 5, 32),
                   # shapes the tensor-core path does not take: the plain kernel
                   (7, 5, 72), (3, 12, 8), (20, 130, 200)]
 
@@ -164,7 +166,8 @@ def test_wo_gemm_is_bit_exact_on_small_integers(sq, M, N, K):
     assert np.array_equal(Yg.view(np.uint16), Yo.view(np.uint16))
 
 
-@pytest.mark.parametrize("M,N,K", [(70, 264, 4096), (16, 1024, 14336), (300, 512, 2048), (9, 130, 200)])
+@pytest.mark.parametrize("M,N,K", [(70, 264, 4096), (16, 1024, 14336), (300, 512, 2048), (9, 130, 200), (1, 520, 14336),
+                                   (2, 264, 4096)])
 def test_wo_gemm_real_values_within_the_fp32_accumulation_bound(sq, M, N, K):
     rng = np.random.default_rng(M + N + K)
     Z16 = (rng.standard_normal((M, K)) * rng.uniform(0.1, 10.0, size=(M, 1))).astype(np.float16)
