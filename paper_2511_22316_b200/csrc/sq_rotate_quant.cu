@@ -49,9 +49,11 @@ __device__ __forceinline__ void row_scale(float amax, __half& delta, float& inv,
   inv = (d > 0.0f) ? __fdiv_rn(1.0f, d) : 0.0f;
 }
 
-// `qmax` = 7 for INT4; qmax = 0 means rotation only: Xq then receives the rotated rows as fp16
-// [rows x n] and `scales` is not touched (weight-only variant).
-template <int MAXT, bool VEC>
+// `qmax` = 7 for INT4.  F16OUT: rotation only, Xq then receives the rotated rows as fp16 [rows x n]
+// and `scales` is not touched (weight-only variant); a separate instantiation, so that the quantising
+// kernel's code is what it was without it (as a run-time branch it cost that kernel half of its speed:
+// the compiler stopped software-pipelining its two product loops).
+template <int MAXT, bool VEC, bool F16OUT>
 __global__ void __launch_bounds__(512)
 rotate_quant_kernel(const float* __restrict__ R1, const float* __restrict__ R2, int n1, int n2,
                     const __half* __restrict__ X, long long rows, uint8_t* __restrict__ Xq,
@@ -154,7 +156,7 @@ rotate_quant_kernel(const float* __restrict__ R1, const float* __restrict__ R2, 
           for (int j = 0; j < TQ; ++j) amax = fmaxf(amax, fabsf(z[t][i][j]));   // padded entries are 0
       }
     }
-    if (qmax == 0) {
+    if constexpr (F16OUT) {
       // ---- rotation only: the row leaves as fp16 ---------------------------------------------------
       __half* zrow16 = reinterpret_cast<__half*>(Xq) + row * (long long)n;
 #pragma unroll
@@ -250,7 +252,7 @@ template <int MAXT, bool VEC>
 sq_status_t launch_generic(const float* dR1, const float* dR2, int n1, int n2, const void* X, int64_t rows,
                            void* Xq, void* scales, float* Zdbg, int threads, size_t smem, int sms,
                            cudaStream_t s, int qmax) {
-  auto kern = rotate_quant_kernel<MAXT, VEC>;
+  auto kern = qmax == 0 ? rotate_quant_kernel<MAXT, VEC, true> : rotate_quant_kernel<MAXT, VEC, false>;
   if (smem > 48 * 1024) {
     if (cudaFuncSetAttribute(kern, cudaFuncAttributeMaxDynamicSharedMemorySize, static_cast<int>(smem)) != cudaSuccess)
       return SQ_ERR_CUDA;
