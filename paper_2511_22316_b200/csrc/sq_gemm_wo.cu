@@ -306,8 +306,8 @@ wo_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_const
 // MMAs.  Two converter groups alternate stages (a third group and a third operand stage changed
 // nothing).  What bounds a stage now, at about 1300 cycles: not the MMAs (issuing half of them changes
 // nothing) and only a little the widening arithmetic (dropping it saves 15 %); what remains is moving
-// the 64 KB fp16 operand of a stage into tensor memory.  K is not split over CTAs: a layer with few
-// output channels (4096: 32 tiles) keeps only that many SMs busy.  The accumulator holds one channel
+// the 64 KB fp16 operand of a stage into tensor memory.  Where the tiles alone leave most SMs idle
+// (4096 channels: 32 tiles) K is split over a cluster of 2 or 4 CTAs.  The accumulator holds one channel
 // per thread and the tokens along its registers; a warp's stores of one token cover 32 consecutive
 // channels.
 constexpr int WOD_CONV_GROUPS = 2;
@@ -333,7 +333,7 @@ struct WoDecSmem {
 template <int NT, int ST, int SS>
 __global__ void __launch_bounds__(WOD_THREADS, 1)
 wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_constant__ CUtensorMap tmap_w,
-                      const __half* __restrict__ sw, int M, int N, int K, __half* __restrict__ Y) {
+                      const __half* __restrict__ sw, int M, int N, int K, __half* __restrict__ Y, int splits) {
   using L = WoDecSmem<NT, ST, SS>;
   griddep_launch_dependents();
   extern __shared__ unsigned char smem_dyn[];
@@ -354,6 +354,12 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
   const int num_sb = (num_kb + 3) / 4;        // stages per tile (the last may hold fewer than four k-blocks)
   const int num_tiles = (N + 127) / 128;
   const uint32_t limit = wait_limit();
+  // K split over a cluster of `splits` CTAs (1, 2 or 4) where the tiles alone leave most SMs idle: the
+  // cluster's CTAs work on the same tile, CTA r of it on the stages [sb0, sb1); the launcher then gives
+  // every cluster exactly one tile, and the partial tiles meet in CTA 0 at the end (see the epilogue).
+  const uint32_t crank = splits > 1 ? cluster_ctarank() : 0u;
+  const int cid = static_cast<int>(blockIdx.x) / splits, ncl = static_cast<int>(gridDim.x) / splits;
+  const int sb0 = static_cast<int>(crank) * num_sb / splits, sb1 = (static_cast<int>(crank) + 1) * num_sb / splits;
 
   // The weights do not depend on the kernel before this one: the first ring-full of them is requested
   // before anything else is set up and before that kernel's completion is awaited.
@@ -363,14 +369,14 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
     for (int s = 0; s < SS; ++s) mbar_init(&st_full[s], 1);
     mbar_fence_init();
     {
-      int t = blockIdx.x, sb = 0;
-      while (pre < SS && t < num_tiles) {
+      int t = cid, sb = sb0;
+      while (pre < SS && t < num_tiles && sb < sb1) {
         mbar_arrive_expect_tx(&st_full[pre], L::W_ST);
         tma_load_2d(smem + L::OFF_W_ST + pre * L::W_ST, &tmap_w, &st_full[pre], sb * 128, t * 128);
         ++pre;
-        if (++sb >= num_sb) {
-          sb = 0;
-          t += gridDim.x;
+        if (++sb >= sb1) {
+          sb = sb0;
+          t += ncl;
         }
       }
     }
@@ -405,8 +411,8 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
     if (lane == 0) {
       uint32_t sit = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-        for (int sb = 0; sb < num_sb && ok; ++sb, ++sit) {
+      for (int tile = cid; tile < num_tiles && ok; tile += ncl) {
+        for (int sb = sb0; sb < sb1 && ok; ++sb, ++sit) {
           if (sit >= static_cast<uint32_t>(pre)) {          // the first `pre` blocks are on their way already
             const int ss = sit % SS;
             ok = mbar_wait(&st_empty[ss], ((sit / SS) & 1) ^ 1, WO_ST_EMPTY, limit);
@@ -433,13 +439,13 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
       const uint64_t t_desc0 = umma_desc_sw128(smem_u32(smem + L::OFF_T));
       uint32_t it = 0, tcount = 0;
       bool ok = true;
-      for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+      for (int tile = cid; tile < num_tiles && ok; tile += ncl, ++tcount) {
         const uint32_t b = tcount & 1;
         ok = mbar_wait(&tmem_empty[b], ((tcount >> 1) & 1) ^ 1, WO_TMEM_EMPTY, limit);
         if (!ok) break;
         tc_fence_after_sync();
         const uint32_t tmem_d = tmem_base + b * NT;
-        for (int sb = 0; sb < num_sb; ++sb, ++it) {
+        for (int sb = sb0; sb < sb1; ++sb, ++it) {
           const int st = it % ST, sa = it % WOD_A_STAGES;
           const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
           ok = mbar_wait(&t_full[st], (it / ST) & 1, WO_A_FULL, limit) &&
@@ -454,7 +460,7 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
 #pragma unroll
               for (int k = 0; k < 4; ++k)         // K = 16 fp16: eight 32-bit columns of A, 32 bytes of a token row
                 umma_f16_ts(tmem_d, a_tmem + 32 * h + 8 * k, td + ((h * L::T_KB + k * 32) >> 4), idesc,
-                            (sb | h | k) != 0 ? 1u : 0u);
+                            ((sb - sb0) | h | k) != 0 ? 1u : 0u);
             }
           }
           umma_commit(&t_empty[st]);
@@ -471,8 +477,8 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
     const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
     uint32_t it = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x) {
-      for (int sb = 0; sb < num_sb && ok; ++sb, ++it) {
+    for (int tile = cid; tile < num_tiles && ok; tile += ncl) {
+      for (int sb = sb0; sb < sb1 && ok; ++sb, ++it) {
         if ((it % WOD_CONV_GROUPS) != static_cast<uint32_t>(grp)) continue;
         const int ss = it % SS, sa = it % WOD_A_STAGES;
         const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
@@ -519,7 +525,7 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
     const int quarter = warp & 3;
     uint32_t tcount = 0;
     bool ok = true;
-    for (int tile = blockIdx.x; tile < num_tiles && ok; tile += gridDim.x, ++tcount) {
+    for (int tile = cid; tile < num_tiles && ok; tile += ncl, ++tcount) {
       const uint32_t b = tcount & 1;
       const int ch = tile * 128 + quarter * 32 + lane;
       const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;
@@ -527,6 +533,24 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
       if (!ok) break;
       tc_fence_after_sync();
       const uint32_t tmem_d = tmem_base + b * NT + (static_cast<uint32_t>(quarter * 32) << 16);
+      if (splits > 1) {
+        // K split over the cluster (one tile per cluster): CTAs other than the first leave their partial
+        // tile in their own shared memory, [token][channel] fp32 over the token ring (every load into it
+        // has been consumed once the accumulator is complete); the first CTA adds them after the cluster
+        // barrier below.  Nothing is stored here.
+        if (crank != 0) {
+          float* part = reinterpret_cast<float*>(smem + L::OFF_T);
+#pragma unroll
+          for (int c = 0; c < NT / 16; ++c) {
+            uint32_t r[16];
+            tmem_ld_32x32b_x16(tmem_d + c * 16, r);
+            tmem_wait_ld();
+#pragma unroll
+            for (int e = 0; e < 16; ++e) part[(c * 16 + e) * 128 + quarter * 32 + lane] = __uint_as_float(r[e]);
+          }
+        }
+        continue;
+      }
 #pragma unroll
       for (int c = 0; c < NT / 16; ++c) {
         uint32_t r[16];
@@ -548,6 +572,46 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
 
   tc_fence_before_sync();
   __syncthreads();
+  if (splits > 1) {
+    // Every thread of every CTA of the cluster comes through here, whatever happened above: the two
+    // barriers are hardware barriers, not polled waits.
+    cluster_sync_all();                                 // the partial tiles are in place
+    if (crank == 0 && warp >= 2 + WOD_CONV_WARPS && cid < num_tiles) {
+      tc_fence_after_sync();
+      const int quarter = warp & 3;
+      const int ch = cid * 128 + quarter * 32 + lane;
+      const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;
+      const uint32_t tmem_d = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);     // accumulator 0: one tile
+      const float* part = reinterpret_cast<const float*>(smem + L::OFF_T);
+#pragma unroll
+      for (int c = 0; c < NT / 16; ++c) {
+        uint32_t r[16];
+        tmem_ld_32x32b_x16(tmem_d + c * 16, r);
+        tmem_wait_ld();
+        // all of a chunk's remote reads are issued before the first is used (each is a round trip to
+        // another SM); the sums are taken in a fixed order: deterministic
+        float a[16];
+#pragma unroll
+        for (int e = 0; e < 16; ++e) a[e] = __uint_as_float(r[e]);
+        for (int pr = 1; pr < splits; ++pr) {
+          const uint32_t base = cluster_map(part + (c * 16) * 128 + quarter * 32 + lane, static_cast<uint32_t>(pr));
+          float v[16];
+#pragma unroll
+          for (int e = 0; e < 16; ++e)
+            asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v[e]) : "r"(base + e * 512) : "memory");
+#pragma unroll
+          for (int e = 0; e < 16; ++e) a[e] += v[e];
+        }
+#pragma unroll
+        for (int e = 0; e < 16; ++e) {
+          const int tok = c * 16 + e;
+          if (ch < N && tok < M) Y[static_cast<size_t>(tok) * N + ch] = __float2half_rn(a[e] * swv);
+        }
+      }
+      tc_fence_before_sync();
+    }
+    cluster_sync_all();                                 // the others' shared memory has been read
+  }
   if (warp == 1) {
     tc_fence_after_sync();
     tmem_dealloc(tmem_base, 512);
@@ -758,9 +822,15 @@ sq_status_t launch_wo_decode(const void* Z16, const void* Wq, const void* sw, in
   const int sms = sm_count();
   if (sms <= 0) return SQ_ERR_CUDA;
   const int tiles = (N + 127) / 128;
-  const int grid = tiles < sms ? tiles : sms;
-  const cudaError_t err = launch_maybe_pdl(kern, dim3(grid), dim3(WOD_THREADS), L::DYN_BYTES, s, mz, mw,
-                                           static_cast<const __half*>(sw), M, N, K, static_cast<__half*>(Y));
+  // K over clusters of 2 or 4 CTAs where the tiles alone would leave more than half of the SMs idle and
+  // every CTA still gets at least four 256-channel stages; each cluster then has exactly one tile.
+  const int num_sb = (K / 64 + 3) / 4;
+  int splits = 1;
+  while (splits < 4 && tiles * splits * 2 <= sms && num_sb / (splits * 2) >= 4) splits *= 2;
+  const int grid = splits > 1 ? tiles * splits : (tiles < sms ? tiles : sms);
+  const cudaError_t err = launch_cluster_maybe_pdl(kern, dim3(grid), dim3(WOD_THREADS), L::DYN_BYTES, s,
+                                                   static_cast<unsigned>(splits), mz, mw, static_cast<const __half*>(sw),
+                                                   M, N, K, static_cast<__half*>(Y), splits);
   count_launch();
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
 }
