@@ -305,8 +305,10 @@ wo_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_const
 // whose hand-overs cost 920 cycles each).  A stage is a whole staging block: 256 channels, sixteen
 // MMAs.  Two converter groups alternate stages (a third group and a third operand stage changed
 // nothing).  What bounds a stage now, at about 1300 cycles: two things of about the same size -- the
-// sixteen MMAs of a stage take about 76 cycles each behind one issuing thread (with the converters
-// idle a stage still takes 1220 cycles), and a converter group needs about as long to widen and move
+// sixteen MMAs of a stage take about 76 cycles each (with the converters idle a stage still takes 1220
+// cycles; a second issuing thread with an accumulator of its own, with or without a third converter
+// group, changed nothing, so it is the tensor pipe reading its 4 KB A operand out of tensor memory per
+// MMA, not the issue), and a converter group needs about as long to widen and move
 // the 64 KB fp16 operand of a stage into tensor memory.  Where the tiles alone leave most SMs idle
 // (4096 channels: 32 tiles) K is split over a cluster of 2 or 4 CTAs.  The accumulator holds one channel
 // per thread and the tokens along its registers; a warp's stores of one token cover 32 consecutive
