@@ -168,6 +168,31 @@ def test_wo_gemm_is_bit_exact_on_small_integers(sq, M, N, K):
     assert np.array_equal(Yg.view(np.uint16), Yo.view(np.uint16))
 
 
+def test_wo_gemm_random_shapes_bit_exact(sq):
+    """Forty seeded random shapes over every kernel of the product (dot products, decode form with and
+    without the K split, prefill form with both tile widths, the plain kernel), small integers so that
+    the result must equal the oracle's bit for bit."""
+    rng = np.random.default_rng(20240607)
+    for trial in range(40):
+        kind = trial % 5
+        if kind == 0:
+            M, N, K = int(rng.integers(1, 3)), int(rng.integers(1, 400)), 32 * int(rng.integers(1, 200))
+        elif kind == 1:
+            M, N, K = int(rng.integers(3, 65)), 8 * int(rng.integers(16, 300)), 64 * int(rng.integers(1, 100))
+        elif kind == 2:
+            M, N, K = int(rng.integers(3, 65)), 8 * int(rng.integers(16, 40)), 64 * int(rng.integers(64, 200))
+        elif kind == 3:
+            M, N, K = int(rng.integers(65, 400)), 8 * int(rng.integers(1, 200)), 64 * int(rng.integers(1, 40))
+        else:
+            M, N, K = int(rng.integers(1, 40)), int(rng.integers(1, 150)), 8 * int(rng.integers(1, 60))
+        Z16 = rng.integers(-8, 9, size=(M, K)).astype(np.float16)
+        codes = rng.integers(-8, 8, size=(N, K), dtype=np.int8)
+        sw = (2.0 ** rng.integers(-12, -6, size=N)).astype(np.float16)
+        Yg = _run_wo_gemm(sq, Z16, codes, sw)
+        Yo = ora.gemm_w4a16(Z16, codes, sw)
+        assert np.array_equal(Yg.view(np.uint16), Yo.view(np.uint16)), (trial, M, N, K)
+
+
 @pytest.mark.parametrize("M,N,K", [(70, 264, 4096), (16, 1024, 14336), (300, 512, 2048), (9, 130, 200), (1, 520, 14336),
                                    (2, 264, 4096)])
 def test_wo_gemm_real_values_within_the_fp32_accumulation_bound(sq, M, N, K):
