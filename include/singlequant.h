@@ -145,7 +145,12 @@ sq_status_t sq_pack_weight(const sq_rotation_t* rot_or_null, const void* W, int6
  * exchanged through cluster shared memory).
  * Supported: K even, K <= 65536 (so that the 256x-scaled int32 accumulator cannot overflow).
  * The tensor-core path needs K % 128 == 0 and N % 8 == 0; other shapes run a plain integer
- * kernel with the same results. */
+ * kernel with the same results.
+ * Ordering: the kernel is queued as a programmatic dependent of the kernel before it in `stream`: it
+ * may request its first blocks of Wq while that kernel still runs, and waits for it before it reads Xq
+ * or sx or writes Y.  Weights packed by sq_pack_weight / sq_pack_weight_wo on the same stream are
+ * complete by then (those calls end with an ordinary kernel).  A caller that produces Wq with a
+ * kernel of its own which lets dependents start early must not let it do so before Wq is written. */
 sq_status_t sq_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw,
                          int64_t M, int64_t N, int64_t K, void* Y, void* accdbg_or_null,
                          void* stream);

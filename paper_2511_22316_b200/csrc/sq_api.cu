@@ -10,7 +10,7 @@
 
 namespace sq {
 std::atomic<uint64_t> g_launches{0};
-thread_local bool g_pdl_next = false;
+thread_local bool g_pdl_next = true;
 
 bool ensure_dyn_smem(const void* kern, int bytes) {
   struct Entry { int dev; const void* kern; int bytes; };
@@ -62,6 +62,13 @@ sq_status_t read_and_clear_device_status(cudaStream_t s) {
 extern "C" void sq_rotation_destroy(sq_rotation_t* rot);
 
 namespace sq {
+// Ends sq_pack_weight: an ordinary launch that never lets dependents start early.  The GEMM kernels are
+// launched as programmatic dependents and request their first weight blocks before they wait for their
+// predecessor; the rotate kernels that wrote those weights allow dependents while they are still
+// writing, this kernel does not, so a GEMM queued right behind sq_pack_weight starts after the weights
+// are complete.
+__global__ void weights_complete_kernel() {}
+
 // One thread, one barrier that nobody arrives at, the library's own bounded wait: it gives up after
 // `polls` polls, records its site in the status word and returns.  No copy, MMA or TMEM allocation
 // is in flight when it does.
@@ -261,10 +268,14 @@ sq_status_t sq_pack_weight(const sq_rotation_t* rot_or_null, const void* W, int6
   sq_status_t st = check_rows_args(W, Wq, sw, nullptr, N, K);
   if (st != SQ_OK || N == 0) return st;
   if (rot_or_null && (st = check_handle_device(rot_or_null)) != SQ_OK) return st;
-  if (rot_or_null)
-    return sq::rotate_quant_dispatch(rot_or_null, W, N, Wq, sw, nullptr, static_cast<cudaStream_t>(stream));
-  return sq::launch_rotate_quant(nullptr, nullptr, 1, static_cast<int>(K), W, N, Wq, sw, nullptr,
-                                 static_cast<cudaStream_t>(stream));
+  if (!rot_or_null)
+    return sq::launch_rotate_quant(nullptr, nullptr, 1, static_cast<int>(K), W, N, Wq, sw, nullptr,
+                                   static_cast<cudaStream_t>(stream));
+  st = sq::rotate_quant_dispatch(rot_or_null, W, N, Wq, sw, nullptr, static_cast<cudaStream_t>(stream));
+  if (st != SQ_OK) return st;
+  sq::weights_complete_kernel<<<1, 32, 0, static_cast<cudaStream_t>(stream)>>>();
+  sq::count_launch();
+  return cudaGetLastError() == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
 }
 
 sq_status_t sq_w4a4_gemm(const void* Xq, const void* sx, const void* Wq, const void* sw, int64_t M, int64_t N,
@@ -309,10 +320,7 @@ sq_status_t sq_linear(const sq_rotation_t* rot, const void* X, int64_t M, const 
   if (st != SQ_OK) return st;
   // Every tensor-core GEMM kernel and the dot-product kernel start their set-up (and their weight
   // loads) while the rotate kernel drains; they wait for it before they read Xq or sx.
-  sq::g_pdl_next = true;
-  st = sq::launch_w4a4_gemm(Xq, sx, Wq, sw, M, N, K, Y, nullptr, s);
-  sq::g_pdl_next = false;
-  return st;
+  return sq::launch_w4a4_gemm(Xq, sx, Wq, sw, M, N, K, Y, nullptr, s);
 }
 
 // Workspace layout of sq_linear_host: [X: 2*M*K][Y: 2*M*N][sq_linear workspace].
@@ -518,10 +526,7 @@ sq_status_t sq_linear_wo(const sq_rotation_t* rot, const void* X, int64_t M, con
   cudaStream_t s = static_cast<cudaStream_t>(stream);
   st = sq::rotate_f16_dispatch(rot, X, M, Z16, s);
   if (st != SQ_OK) return st;
-  sq::g_pdl_next = true;                  // the product may set itself up while the rotation drains
-  st = sq::launch_wo_gemm(Z16, Wq, sw, M, N, K, Y, s);
-  sq::g_pdl_next = false;
-  return st;
+  return sq::launch_wo_gemm(Z16, Wq, sw, M, N, K, Y, s);     // sets itself up while the rotation drains
 }
 
 sq_status_t sq_linear_grouped(const sq_rotation_t* const* rots, int32_t E, const int64_t* offsets, const void* X,

@@ -49,8 +49,12 @@ inline void count_launch(uint64_t k = 1) { g_launches.fetch_add(k, std::memory_o
 // Multiprocessor count of the current device (cached per device; <= 0 on failure).
 int sm_count();
 
-// Set by sq_linear around its GEMM launch: the GEMM may then start while the rotate+quant kernel
-// before it in the stream is still running (it waits on the device before reading Xq and sx).
+// True except around the launch of the one-launch decode layer: every GEMM kernel is launched as a
+// programmatic dependent of the kernel before it in the stream.  It may then set itself up and request
+// its first weight blocks while that kernel is still running (a rotate kernel, or another GEMM in a run
+// of projections); it waits on the device before it reads activations, steps or writes anything.  Weights
+// written by this library are complete by then: sq_pack_weight and sq_pack_weight_wo end with an ordinary
+// kernel, which never lets dependents start early.
 extern thread_local bool g_pdl_next;
 
 // Launches `kern` with thread-block clusters of `cluster` CTAs along x (1: no clusters), and as a
