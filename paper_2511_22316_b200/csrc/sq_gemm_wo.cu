@@ -633,7 +633,9 @@ template <int MT>
 __global__ void __launch_bounds__(512)
 wo_gemv_kernel(const __half* __restrict__ Z16, const uint8_t* __restrict__ Wq, const __half* __restrict__ sw, int M,
                int N, int K, __half* __restrict__ Y) {
-  griddep_launch_dependents();
+  // No early start for whatever follows: its CTAs would sit on the SMs beside this kernel's (a second
+  // large shared-memory allocation per SM) and slow the streaming down (36 us instead of 18 on
+  // 1 x 4096 x 14336 in back-to-back launches).
   griddep_wait();                                        // Z16 may come from the kernel launched before this one
   // Tokens as fp32, laid out [token][word of a piece g][half h][piece c][4]: the lanes of a warp work on
   // consecutive pieces c, so their 16-byte reads for one (g, h) are contiguous (no bank conflicts).
