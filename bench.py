@@ -53,8 +53,7 @@ NCU_TRAFFIC = {
     ("rotate_quant", "llama2_7b_down_prefill"): 45412608,   # rotate_quant_pair_kernel
     ("rotate_quant", "llama2_70b_gateup_prefill"): 69889536,   # rotate_quant_tc_kernel, n2 = 128
     ("rotate_quant", "llama2_70b_down_prefill"): 275649024,    # rotate_quant_pair_kernel, n2 = 128
-    ("wo_gemm", "llama3_8b_up_decode_m16"): 29557248,       # wo_gemm_decode_kernel (W4A16)
-    ("wo_gemm", "llama2_7b_qkvo_prefill"): 25196544,        # wo_gemm_tc_kernel (W4A16; Y stayed in L2)
+    ("wo_gemm", "llama3_8b_up_decode_m16"): 29557248,       # wo_gemm_tmem_kernel (W4A16)
 }
 
 
@@ -546,13 +545,14 @@ def weight_only_entry(sq, torch, w, bits, pk, l2, quick=False):
     rot_bytes = 4.0 * M * K
     if M <= 64:
         gbs = gemm_bytes_wo / (gemm_ms * 1e-3) / 1e9
-        roof = {"kernel": "wo_gemv_kernel" if M <= 2 else "wo_gemm_decode_kernel", "bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
+        roof = {"kernel": "wo_gemv_kernel" if M <= 2 else "wo_gemm_tmem_kernel", "bound": "hbm", "achieved": gbs, "peak": pk["hbm_gbs"], "unit": "GB/s",
                 "frac": gbs / pk["hbm_gbs"], "traffic": NCU_TRAFFIC.get(("wo_gemm", w.name)) if bits == 4 else None,
                 "ms_per_launch": gemm_ms,
                 "algorithmic_bytes": gemm_bytes_wo}
     else:
         tf = flops / (gemm_ms * 1e-3) / 1e12
-        roof = {"kernel": "wo_gemm_tc_kernel", "bound": "tensor", "achieved": tf, "peak": pk["bf16_tflops"],
+        roof = {"kernel": "wo_gemm_tmem_kernel" if (N >= 128 and K % 64 == 0 and N % 8 == 0) else "wo_gemm_tc_kernel",
+                "bound": "tensor", "achieved": tf, "peak": pk["bf16_tflops"],
                 "unit": "TFLOP/s", "frac": tf / pk["bf16_tflops"],
                 "traffic": NCU_TRAFFIC.get(("wo_gemm", w.name)) if bits == 4 else None, "ms_per_launch": gemm_ms,
                 "peak_source": f"{pk['source']} bf16 burst (fp16 runs at the same rate)", "algorithmic_flops": flops}

@@ -294,8 +294,10 @@ wo_gemm_tc_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_const
   }
 }
 
-// Decode-sized batches (M <= 64): the product is bound by reading the packed weights once, so the
-// operands swap roles.  A tile is 128 OUTPUT CHANNELS (the MMA's M and the accumulator's lanes), the
+// The main kernel.  Its design comes from decode-sized batches (M <= 64), where the product is bound by
+// reading the packed weights once; with 128-token tiles it also takes the larger batches (see the
+// dispatch at the end of the file), because the weights as a tensor-memory operand cost no
+// shared-memory traffic.  The operands swap roles.  A tile is 128 OUTPUT CHANNELS (the MMA's M and the accumulator's lanes), the
 // tokens are the MMA's N (16, 32 or 64): the token tiles are a few KB straight from TMA, and an MMA
 // with a narrow N takes a third of the time.  The widened weights never touch shared memory: each
 // thread of a converter group reads the 128 packed bytes of "its" channel from the staging ring,
@@ -317,7 +319,7 @@ constexpr int WOD_CONV_GROUPS = 2;
 constexpr int WOD_CONV_WARPS = 4 * WOD_CONV_GROUPS;
 constexpr int WOD_THREADS = (2 + WOD_CONV_WARPS + WO_EPI_WARPS) * 32;
 constexpr int WOD_A_STAGES = 2;           // tensor-memory operand stages of 128 columns (256 fp16 channels)
-constexpr int WOD_A_COL0 = 128;           // accumulators: columns [0, 2 NT); operand ring: [128, 384)
+// accumulators: columns [0, 2 NT); operand ring: two stages of 128 columns from column max(128, 2 NT) on
 
 template <int NT, int ST, int SS>
 struct WoDecSmem {
@@ -335,9 +337,10 @@ struct WoDecSmem {
 
 template <int NT, int ST, int SS>
 __global__ void __launch_bounds__(WOD_THREADS, 1)
-wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_constant__ CUtensorMap tmap_w,
+wo_gemm_tmem_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_constant__ CUtensorMap tmap_w,
                       const __half* __restrict__ sw, int M, int N, int K, __half* __restrict__ Y, int splits) {
   using L = WoDecSmem<NT, ST, SS>;
+  constexpr int WOD_A_COL0 = 2 * NT > 128 ? 2 * NT : 128;
   griddep_launch_dependents();
   extern __shared__ unsigned char smem_dyn[];
   unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
@@ -355,7 +358,10 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = K / 64;
   const int num_sb = (num_kb + 3) / 4;        // stages per tile (the last may hold fewer than four k-blocks)
-  const int num_tiles = (N + 127) / 128;
+  // A tile is 128 channels x NT tokens; the channel tiles run fastest, so that the CTAs at work at one
+  // time share a few token tiles (which stay in L2) and stream different weights.
+  const int tiles_n = (N + 127) / 128;
+  const int num_tiles = tiles_n * ((M + NT - 1) / NT);
   const uint32_t limit = wait_limit();
   // K split over a cluster of `splits` CTAs (1, 2 or 4) where the tiles alone leave most SMs idle: the
   // cluster's CTAs work on the same tile, CTA r of it on the stages [sb0, sb1); the launcher then gives
@@ -375,7 +381,7 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
       int t = cid, sb = sb0;
       while (pre < SS && t < num_tiles && sb < sb1) {
         mbar_arrive_expect_tx(&st_full[pre], L::W_ST);
-        tma_load_2d(smem + L::OFF_W_ST + pre * L::W_ST, &tmap_w, &st_full[pre], sb * 128, t * 128);
+        tma_load_2d(smem + L::OFF_W_ST + pre * L::W_ST, &tmap_w, &st_full[pre], sb * 128, (t % tiles_n) * 128);
         ++pre;
         if (++sb >= sb1) {
           sb = sb0;
@@ -421,7 +427,7 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
             ok = mbar_wait(&st_empty[ss], ((sit / SS) & 1) ^ 1, WO_ST_EMPTY, limit);
             if (!ok) break;
             mbar_arrive_expect_tx(&st_full[ss], L::W_ST);
-            tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, &tmap_w, &st_full[ss], sb * 128, tile * 128);
+            tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, &tmap_w, &st_full[ss], sb * 128, (tile % tiles_n) * 128);
           }
           const int st = sit % ST;
           const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
@@ -429,7 +435,8 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
           if (!ok) break;
           mbar_arrive_expect_tx(&t_full[st], static_cast<uint32_t>(nk * L::T_KB));
           for (int h = 0; h < nk; ++h)
-            tma_load_2d(smem + L::OFF_T + st * L::T_TILE + h * L::T_KB, &tmap_z, &t_full[st], (4 * sb + h) * 64, 0);
+            tma_load_2d(smem + L::OFF_T + st * L::T_TILE + h * L::T_KB, &tmap_z, &t_full[st], (4 * sb + h) * 64,
+                        (tile / tiles_n) * NT);
         }
       }
     }
@@ -530,7 +537,8 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
     bool ok = true;
     for (int tile = cid; tile < num_tiles && ok; tile += ncl, ++tcount) {
       const uint32_t b = tcount & 1;
-      const int ch = tile * 128 + quarter * 32 + lane;
+      const int ch = (tile % tiles_n) * 128 + quarter * 32 + lane;
+      const int tok0 = (tile / tiles_n) * NT;
       const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;
       ok = mbar_wait(&tmem_full[b], (tcount >> 1) & 1, WO_TMEM_FULL, limit);
       if (!ok) break;
@@ -562,7 +570,7 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
         if (ch < N) {
 #pragma unroll
           for (int e = 0; e < 16; ++e) {
-            const int tok = c * 16 + e;
+            const int tok = tok0 + c * 16 + e;
             if (tok < M) Y[static_cast<size_t>(tok) * N + ch] = __float2half_rn(__uint_as_float(r[e]) * swv);
           }
         }
@@ -582,7 +590,8 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
     if (crank == 0 && warp >= 2 + WOD_CONV_WARPS && cid < num_tiles) {
       tc_fence_after_sync();
       const int quarter = warp & 3;
-      const int ch = cid * 128 + quarter * 32 + lane;
+      const int ch = (cid % tiles_n) * 128 + quarter * 32 + lane;
+      const int tok0 = (cid / tiles_n) * NT;
       const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;
       const uint32_t tmem_d = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);     // accumulator 0: one tile
       const float* part = reinterpret_cast<const float*>(smem + L::OFF_T);
@@ -607,7 +616,7 @@ wo_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_c
         }
 #pragma unroll
         for (int e = 0; e < 16; ++e) {
-          const int tok = c * 16 + e;
+          const int tok = tok0 + c * 16 + e;
           if (ch < N && tok < M) Y[static_cast<size_t>(tok) * N + ch] = __float2half_rn(a[e] * swv);
         }
       }
@@ -822,11 +831,11 @@ sq_status_t launch_wo_decode(const void* Z16, const void* Wq, const void* sw, in
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return SQ_ERR_CUDA;
   if (!make_packed_map(&mw, Wq, N, K / 2, 128)) return SQ_ERR_CUDA;
-  auto kern = wo_gemm_decode_kernel<NT, ST, SS>;
+  auto kern = wo_gemm_tmem_kernel<NT, ST, SS>;
   if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), L::DYN_BYTES)) return SQ_ERR_CUDA;
   const int sms = sm_count();
   if (sms <= 0) return SQ_ERR_CUDA;
-  const int tiles = (N + 127) / 128;
+  const int tiles = ((N + 127) / 128) * ((M + NT - 1) / NT);
   // K over clusters of 2 or 4 CTAs where the tiles alone would leave more than half of the SMs idle and
   // every CTA still gets at least four 256-channel stages; each cluster then has exactly one tile.
   const int num_sb = (K / 64 + 3) / 4;
@@ -873,6 +882,12 @@ sq_status_t launch_wo_gemm(const void* Z16, const void* Wq, const void* sw, int6
     if (M <= 16) return launch_wo_decode<16, 4, 8>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
     if (M <= 32) return launch_wo_decode<32, 4, 8>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
     return launch_wo_decode<64, 3, 6>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
+  }
+  if (tc_ok && N >= 128) {
+    // Larger batches through the same kernel with 128-token tiles: the weights as the tensor-memory
+    // operand cost no shared-memory traffic at all, which is what bounds the kernel below (2048 x 4096 x
+    // 4096: 76 us there).
+    return launch_wo_decode<128, 2, 4>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
   }
   if (tc_ok) {
     // 256-channel tiles wherever there are enough token rows and channels: the kernel is bound by shared
