@@ -53,7 +53,8 @@ NCU_TRAFFIC = {
     ("rotate_quant", "llama2_7b_down_prefill"): 45412608,   # rotate_quant_pair_kernel
     ("rotate_quant", "llama2_70b_gateup_prefill"): 69889536,   # rotate_quant_tc_kernel, n2 = 128
     ("rotate_quant", "llama2_70b_down_prefill"): 275649024,    # rotate_quant_pair_kernel, n2 = 128
-    ("wo_gemm", "llama3_8b_up_decode_m16"): 29557248,       # wo_gemm_tmem_kernel (W4A16)
+    ("wo_gemm", "llama3_8b_up_decode_m16"): 29558016,       # wo_gemm_tmem_kernel<16, 4, 8> (W4A16)
+    ("wo_gemm", "llama2_7b_qkvo_prefill"): 25266944,        # wo_gemm_tmem_kernel<128, 2, 4> (W4A16; Y stayed in L2)
 }
 
 
