@@ -335,11 +335,18 @@ struct WoDecSmem {
   static constexpr int DYN_BYTES = TOTAL + 1024;
 };
 
-template <int NT, int ST, int SS>
+template <int NT, int ST, int SS, int CT>
 __global__ void __launch_bounds__(WOD_THREADS, 1)
 wo_gemm_tmem_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_constant__ CUtensorMap tmap_w,
                       const __half* __restrict__ sw, int M, int N, int K, __half* __restrict__ Y, int splits) {
   using L = WoDecSmem<NT, ST, SS>;
+  // CT = channel tiles of 128 that share a token tile (1 or 2).  With one, two accumulators alternate
+  // between tiles (the epilogue of a tile runs under the next tile's MMAs); with two, both accumulators
+  // belong to the same tile -- channels [0, 128) and [128, 256) of it -- and every token block that
+  // reaches shared memory feeds two MMAs instead of one.
+  static_assert(CT == 1 || CT == 2, "one or two channel tiles per token tile");
+  static_assert(2 * NT + 128 * WOD_A_STAGES <= 512, "tensor-memory plan does not fit");
+  constexpr int NBUF = 2 / CT;                           // accumulator sets that alternate between tiles
   constexpr int WOD_A_COL0 = 2 * NT > 128 ? 2 * NT : 128;
   griddep_launch_dependents();
   extern __shared__ unsigned char smem_dyn[];
@@ -360,7 +367,7 @@ wo_gemm_tmem_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_con
   const int num_sb = (num_kb + 3) / 4;        // stages per tile (the last may hold fewer than four k-blocks)
   // A tile is 128 channels x NT tokens; the channel tiles run fastest, so that the CTAs at work at one
   // time share a few token tiles (which stay in L2) and stream different weights.
-  const int tiles_n = (N + 127) / 128;
+  const int tiles_n = (N + 128 * CT - 1) / (128 * CT);
   const int num_tiles = tiles_n * ((M + NT - 1) / NT);
   const uint32_t limit = wait_limit();
   // K split over a cluster of `splits` CTAs (1, 2 or 4) where the tiles alone leave most SMs idle: the
@@ -378,11 +385,14 @@ wo_gemm_tmem_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_con
     for (int s = 0; s < SS; ++s) mbar_init(&st_full[s], 1);
     mbar_fence_init();
     {
-      int t = cid, sb = sb0;
+      int t = cid, sb = sb0, half = 0;
       while (pre < SS && t < num_tiles && sb < sb1) {
         mbar_arrive_expect_tx(&st_full[pre], L::W_ST);
-        tma_load_2d(smem + L::OFF_W_ST + pre * L::W_ST, &tmap_w, &st_full[pre], sb * 128, (t % tiles_n) * 128);
+        tma_load_2d(smem + L::OFF_W_ST + pre * L::W_ST, &tmap_w, &st_full[pre], sb * 128,
+                    ((t % tiles_n) * CT + half) * 128);
         ++pre;
+        if (++half < CT) continue;
+        half = 0;
         if (++sb >= sb1) {
           sb = sb0;
           t += ncl;
@@ -421,22 +431,27 @@ wo_gemm_tmem_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_con
       uint32_t sit = 0;
       bool ok = true;
       for (int tile = cid; tile < num_tiles && ok; tile += ncl) {
-        for (int sb = sb0; sb < sb1 && ok; ++sb, ++sit) {
-          if (sit >= static_cast<uint32_t>(pre)) {          // the first `pre` blocks are on their way already
-            const int ss = sit % SS;
-            ok = mbar_wait(&st_empty[ss], ((sit / SS) & 1) ^ 1, WO_ST_EMPTY, limit);
+        for (int sb = sb0; sb < sb1 && ok; ++sb) {
+          for (int half = 0; half < CT && ok; ++half, ++sit) {
+            if (sit >= static_cast<uint32_t>(pre)) {        // the first `pre` blocks are on their way already
+              const int ss = sit % SS;
+              ok = mbar_wait(&st_empty[ss], ((sit / SS) & 1) ^ 1, WO_ST_EMPTY, limit);
+              if (!ok) break;
+              mbar_arrive_expect_tx(&st_full[ss], L::W_ST);
+              tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, &tmap_w, &st_full[ss], sb * 128,
+                          ((tile % tiles_n) * CT + half) * 128);
+            }
+            if (half != 0) continue;                        // the token block serves both channel tiles
+            const uint32_t tit = sit / CT;
+            const int st = tit % ST;
+            const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
+            ok = mbar_wait(&t_empty[st], ((tit / ST) & 1) ^ 1, WO_A_EMPTY, limit);
             if (!ok) break;
-            mbar_arrive_expect_tx(&st_full[ss], L::W_ST);
-            tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, &tmap_w, &st_full[ss], sb * 128, (tile % tiles_n) * 128);
+            mbar_arrive_expect_tx(&t_full[st], static_cast<uint32_t>(nk * L::T_KB));
+            for (int h = 0; h < nk; ++h)
+              tma_load_2d(smem + L::OFF_T + st * L::T_TILE + h * L::T_KB, &tmap_z, &t_full[st], (4 * sb + h) * 64,
+                          (tile / tiles_n) * NT);
           }
-          const int st = sit % ST;
-          const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
-          ok = mbar_wait(&t_empty[st], ((sit / ST) & 1) ^ 1, WO_A_EMPTY, limit);
-          if (!ok) break;
-          mbar_arrive_expect_tx(&t_full[st], static_cast<uint32_t>(nk * L::T_KB));
-          for (int h = 0; h < nk; ++h)
-            tma_load_2d(smem + L::OFF_T + st * L::T_TILE + h * L::T_KB, &tmap_z, &t_full[st], (4 * sb + h) * 64,
-                        (tile / tiles_n) * NT);
         }
       }
     }
@@ -450,32 +465,37 @@ wo_gemm_tmem_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_con
       uint32_t it = 0, tcount = 0;
       bool ok = true;
       for (int tile = cid; tile < num_tiles && ok; tile += ncl, ++tcount) {
-        const uint32_t b = tcount & 1;
-        ok = mbar_wait(&tmem_empty[b], ((tcount >> 1) & 1) ^ 1, WO_TMEM_EMPTY, limit);
+        const uint32_t b = tcount % NBUF;
+        ok = mbar_wait(&tmem_empty[b], ((tcount / NBUF) & 1) ^ 1, WO_TMEM_EMPTY, limit);
         if (!ok) break;
         tc_fence_after_sync();
-        const uint32_t tmem_d = tmem_base + b * NT;
-        for (int sb = sb0; sb < sb1; ++sb, ++it) {
-          const int st = it % ST, sa = it % WOD_A_STAGES;
-          const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
-          ok = mbar_wait(&t_full[st], (it / ST) & 1, WO_A_FULL, limit) &&
-               mbar_wait(&a_full[sa], (it / WOD_A_STAGES) & 1, WO_B_FULL, limit);
-          if (!ok) break;
-          tc_fence_after_sync();
-          const uint32_t a_tmem = tmem_base + WOD_A_COL0 + sa * 128;
-          const uint64_t td = t_desc0 + static_cast<uint64_t>((st * L::T_TILE) >> 4);
+        for (int sb = sb0; sb < sb1 && ok; ++sb) {
 #pragma unroll
-          for (int h = 0; h < 4; ++h) {
-            if (h < nk) {
+          for (int half = 0; half < CT; ++half, ++it) {
+            const uint32_t tit = it / CT;
+            const int st = tit % ST, sa = it % WOD_A_STAGES;
+            const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
+            if (half == 0) ok = mbar_wait(&t_full[st], (tit / ST) & 1, WO_A_FULL, limit);
+            ok = ok && mbar_wait(&a_full[sa], (it / WOD_A_STAGES) & 1, WO_B_FULL, limit);
+            if (!ok) break;
+            tc_fence_after_sync();
+            const uint32_t tmem_d = tmem_base + (b * CT + half) * NT;
+            const uint32_t a_tmem = tmem_base + WOD_A_COL0 + sa * 128;
+            const uint64_t td = t_desc0 + static_cast<uint64_t>((st * L::T_TILE) >> 4);
 #pragma unroll
-              for (int k = 0; k < 4; ++k)         // K = 16 fp16: eight 32-bit columns of A, 32 bytes of a token row
-                umma_f16_ts(tmem_d, a_tmem + 32 * h + 8 * k, td + ((h * L::T_KB + k * 32) >> 4), idesc,
-                            ((sb - sb0) | h | k) != 0 ? 1u : 0u);
+            for (int h = 0; h < 4; ++h) {
+              if (h < nk) {
+#pragma unroll
+                for (int k = 0; k < 4; ++k)       // K = 16 fp16: eight 32-bit columns of A, 32 bytes of a token row
+                  umma_f16_ts(tmem_d, a_tmem + 32 * h + 8 * k, td + ((h * L::T_KB + k * 32) >> 4), idesc,
+                              ((sb - sb0) | h | k) != 0 ? 1u : 0u);
+              }
             }
+            if (half == CT - 1) umma_commit(&t_empty[st]);
+            umma_commit(&a_empty[sa]);
           }
-          umma_commit(&t_empty[st]);
-          umma_commit(&a_empty[sa]);
         }
+        if (!ok) break;
         umma_commit(&tmem_full[b]);
       }
     }
@@ -488,8 +508,9 @@ wo_gemm_tmem_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_con
     uint32_t it = 0;
     bool ok = true;
     for (int tile = cid; tile < num_tiles && ok; tile += ncl) {
-      for (int sb = sb0; sb < sb1 && ok; ++sb, ++it) {
+      for (int sbh = sb0 * CT; sbh < sb1 * CT && ok; ++sbh, ++it) {
         if ((it % WOD_CONV_GROUPS) != static_cast<uint32_t>(grp)) continue;
+        const int sb = sbh / CT;
         const int ss = it % SS, sa = it % WOD_A_STAGES;
         const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
         ok = mbar_wait(&st_full[ss], (it / SS) & 1, WO_ST_FULL, limit);
@@ -536,15 +557,17 @@ wo_gemm_tmem_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_con
     uint32_t tcount = 0;
     bool ok = true;
     for (int tile = cid; tile < num_tiles && ok; tile += ncl, ++tcount) {
-      const uint32_t b = tcount & 1;
-      const int ch = (tile % tiles_n) * 128 + quarter * 32 + lane;
+      const uint32_t b = tcount % NBUF;
+      const int ch0 = (tile % tiles_n) * (128 * CT) + quarter * 32 + lane;
       const int tok0 = (tile / tiles_n) * NT;
-      const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;
-      ok = mbar_wait(&tmem_full[b], (tcount >> 1) & 1, WO_TMEM_FULL, limit);
+      float swh[CT];
+#pragma unroll
+      for (int half = 0; half < CT; ++half) swh[half] = (ch0 + 128 * half < N) ? __half2float(sw[ch0 + 128 * half]) : 0.0f;
+      ok = mbar_wait(&tmem_full[b], (tcount / NBUF) & 1, WO_TMEM_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
-      const uint32_t tmem_d = tmem_base + b * NT + (static_cast<uint32_t>(quarter * 32) << 16);
-      if (splits > 1) {
+      const uint32_t tmem_d = tmem_base + b * CT * NT + (static_cast<uint32_t>(quarter * 32) << 16);
+      if (splits > 1) {                                   // (launched with CT = 1 only)
         // K split over the cluster (one tile per cluster): CTAs other than the first leave their partial
         // tile in their own shared memory, [token][channel] fp32 over the token ring (every load into it
         // has been consumed once the accumulator is complete); the first CTA adds them after the cluster
@@ -563,15 +586,20 @@ wo_gemm_tmem_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_con
         continue;
       }
 #pragma unroll
-      for (int c = 0; c < NT / 16; ++c) {
-        uint32_t r[16];
-        tmem_ld_32x32b_x16(tmem_d + c * 16, r);
-        tmem_wait_ld();
-        if (ch < N) {
+      for (int half = 0; half < CT; ++half) {
+        const int ch = ch0 + 128 * half;
+        const float swv = swh[half];
 #pragma unroll
-          for (int e = 0; e < 16; ++e) {
-            const int tok = tok0 + c * 16 + e;
-            if (tok < M) Y[static_cast<size_t>(tok) * N + ch] = __float2half_rn(__uint_as_float(r[e]) * swv);
+        for (int c = 0; c < NT / 16; ++c) {
+          uint32_t r[16];
+          tmem_ld_32x32b_x16(tmem_d + half * NT + c * 16, r);
+          tmem_wait_ld();
+          if (ch < N) {
+#pragma unroll
+            for (int e = 0; e < 16; ++e) {
+              const int tok = tok0 + c * 16 + e;
+              if (tok < M) Y[static_cast<size_t>(tok) * N + ch] = __float2half_rn(__uint_as_float(r[e]) * swv);
+            }
           }
         }
       }
@@ -590,7 +618,7 @@ wo_gemm_tmem_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_con
     if (crank == 0 && warp >= 2 + WOD_CONV_WARPS && cid < num_tiles) {
       tc_fence_after_sync();
       const int quarter = warp & 3;
-      const int ch = (cid % tiles_n) * 128 + quarter * 32 + lane;
+      const int ch = (cid % tiles_n) * 128 + quarter * 32 + lane;                          // CT = 1 here
       const int tok0 = (cid / tiles_n) * NT;
       const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;
       const uint32_t tmem_d = tmem_base + (static_cast<uint32_t>(quarter * 32) << 16);     // accumulator 0: one tile
@@ -814,7 +842,7 @@ sq_status_t launch_wo_tc(const void* Z16, const void* Wq, const void* sw, int M,
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
 }
 
-template <int NT, int ST, int SS>
+template <int NT, int ST, int SS, int CT = 1>
 sq_status_t launch_wo_decode(const void* Z16, const void* Wq, const void* sw, int M, int N, int K, void* Y,
                              cudaStream_t s) {
   using L = WoDecSmem<NT, ST, SS>;
@@ -831,16 +859,16 @@ sq_status_t launch_wo_decode(const void* Z16, const void* Wq, const void* sw, in
           CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
     return SQ_ERR_CUDA;
   if (!make_packed_map(&mw, Wq, N, K / 2, 128)) return SQ_ERR_CUDA;
-  auto kern = wo_gemm_tmem_kernel<NT, ST, SS>;
+  auto kern = wo_gemm_tmem_kernel<NT, ST, SS, CT>;
   if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), L::DYN_BYTES)) return SQ_ERR_CUDA;
   const int sms = sm_count();
   if (sms <= 0) return SQ_ERR_CUDA;
-  const int tiles = ((N + 127) / 128) * ((M + NT - 1) / NT);
+  const int tiles = ((N + 128 * CT - 1) / (128 * CT)) * ((M + NT - 1) / NT);
   // K over clusters of 2 or 4 CTAs where the tiles alone would leave more than half of the SMs idle and
   // every CTA still gets at least four 256-channel stages; each cluster then has exactly one tile.
   const int num_sb = (K / 64 + 3) / 4;
   int splits = 1;
-  while (splits < 4 && tiles * splits * 2 <= sms && num_sb / (splits * 2) >= 4) splits *= 2;
+  while (CT == 1 && splits < 4 && tiles * splits * 2 <= sms && num_sb / (splits * 2) >= 4) splits *= 2;
   const int grid = splits > 1 ? tiles * splits : (tiles < sms ? tiles : sms);
   const cudaError_t err = launch_cluster_maybe_pdl(kern, dim3(grid), dim3(WOD_THREADS), L::DYN_BYTES, s,
                                                    static_cast<unsigned>(splits), mz, mw, static_cast<const __half*>(sw),
@@ -886,7 +914,9 @@ sq_status_t launch_wo_gemm(const void* Z16, const void* Wq, const void* sw, int6
   if (tc_ok && N >= 128) {
     // Larger batches through the same kernel with 128-token tiles: the weights as the tensor-memory
     // operand cost no shared-memory traffic at all, which is what bounds the kernel below (2048 x 4096 x
-    // 4096: 76 us there).
+    // 4096: 76 us there).  From 256 channels on, two channel tiles share every token block (half the
+    // token traffic out of L2 per flop: 65 -> 61 us on that shape, 1.85 -> 1.65 ms on 4096 x 28672 x 8192).
+    if (N >= 256) return launch_wo_decode<128, 2, 4, 2>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
     return launch_wo_decode<128, 2, 4>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
   }
   if (tc_ok) {

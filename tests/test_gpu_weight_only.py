@@ -144,6 +144,9 @@ def _run_wo_gemm(sq, Z16, codes, sw):
 
 WO_GEMM_SHAPES = [(1, 128, 64), (5, 136, 192), (64, 264, 256), (128, 128, 320), (130, 384, 1024), (200, 8, 4096),
                   (33, 5120, 512), (257, 16392, 128), (300, 16640, 448),
+                  # two channel tiles per token tile: one tile pair; more tile pairs than SMs (a CTA's single
+                  # accumulator set is handed back and reused), the last pair half empty
+                  (129, 256, 64), (1300, 3592, 192),
                   # decode batches with few output channels: K split over clusters of 4 and of 2
                   (16, 264, 8192), (40, 1024, 4096), (64, 136, 2048),
                   # one or two tokens: the dot-product kernel (ragged row count, long rows)
