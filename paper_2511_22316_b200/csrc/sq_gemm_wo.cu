@@ -658,6 +658,275 @@ wo_gemm_tmem_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_con
   }
 }
 
+// The CTA-pair form of the kernel above for batches above 128 tokens (tcgen05 cta_group::2, M = 256,
+// N = 256).  In the single-CTA form an MMA of M = 128, N = 128 with its A operand in tensor memory
+// takes about 96 cycles instead of 64 (reading the 4 KB of A costs as much as the arithmetic), and every
+// 128 x 128 tile pulls its 128 tokens out of L2 again.  Here two CTAs share a tile of 256 channels x 256
+// tokens: CTA r widens channels [128 r, 128 r + 128) of the tile into its own tensor memory (its half of
+// the M operand, its accumulator lanes) and loads tokens [128 r, 128 r + 128) of the tile (its half of
+// the N operand).  An MMA then does 128 cycles of arithmetic per 4 KB of A, and a CTA reads 128 tokens per
+// 256 tokens' worth of work.  The accumulator (128 lanes x 256 columns per CTA) is single-buffered: the
+// operand ring needs the other 256 columns; eight epilogue warps (two per lane quarter, 128 columns
+// each) hand it back after their last read.
+//   warp 0        TMA: packed weights of this CTA's channels (staging ring), this CTA's tokens (ring
+//                 stage s = four 64-channel k-blocks)
+//   warps 2..9    two converter groups, alternating stages: staging -> registers -> tensor-memory ring
+//                 stage s; a warp reports the stage to the leader once its part is stored AND this
+//                 CTA's tokens of the stage have landed
+//   warp 1        (leader CTA) sixteen MMAs per stage; the commit frees stage s in both CTAs
+//   warps 10..17  epilogue: tensor memory -> scale -> fp16 stores
+constexpr int WP_EPI_WARPS = 8;
+constexpr int WP_THREADS = (2 + WOD_CONV_WARPS + WP_EPI_WARPS) * 32;
+constexpr int WP_S = 2;                  // ring stages: 256 channels of K (tokens in shared, weights in tensor memory)
+constexpr int WP_A_COL0 = 256;           // first column of the operand ring (0..255: accumulator)
+static_assert(WP_S == WOD_CONV_GROUPS, "a converter group owns one ring stage");
+
+enum WoPairSite : uint32_t {
+  WP_ST_EMPTY = 96, WP_ST_FULL, WP_T_FULL, WP_EMPTY_T, WP_EMPTY_A, WP_FULL, WP_TMEM_FULL, WP_TMEM_EMPTY
+};
+
+template <int SS>
+struct WoPairSmem {
+  static constexpr int T_KB = 128 * 128;              // 128 tokens x 64 channels fp16 (one k-block)
+  static constexpr int T_TILE = 4 * T_KB;             // a stage: four k-blocks
+  static constexpr int W_ST = 128 * 128;              // 128 channels x 256 packed codes
+  static constexpr int OFF_T = 0;
+  static constexpr int OFF_W_ST = OFF_T + WP_S * T_TILE;
+  static constexpr int OFF_BAR = OFF_W_ST + SS * W_ST;
+  static constexpr int NUM_BARS = 2 * SS + 3 * WP_S + 2;
+  static constexpr int OFF_TMEM = OFF_BAR + NUM_BARS * 8;
+  static constexpr int TOTAL = OFF_TMEM + 16;
+  static constexpr int DYN_BYTES = TOTAL + 1024;
+};
+
+template <int SS>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(WP_THREADS, 1)
+wo_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_z, const __grid_constant__ CUtensorMap tmap_w,
+                    const __half* __restrict__ sw, int M, int N, int K, __half* __restrict__ Y) {
+  using L = WoPairSmem<SS>;
+  griddep_launch_dependents();
+  extern __shared__ unsigned char smem_dyn[];
+  unsigned char* smem = reinterpret_cast<unsigned char*>((reinterpret_cast<uintptr_t>(smem_dyn) + 1023) & ~uintptr_t(1023));
+  uint64_t* bars = reinterpret_cast<uint64_t*>(smem + L::OFF_BAR);
+  uint64_t* st_full = bars;                           // [SS]    packed weights landed (local)
+  uint64_t* st_empty = st_full + SS;                  // [SS]    a converter group has read them (local)
+  uint64_t* t_full = st_empty + SS;                   // [WP_S]  tokens landed (local)
+  uint64_t* full = t_full + WP_S;                     // [WP_S]  stage complete in both CTAs (the leader's copy is used)
+  uint64_t* empty = full + WP_S;                      // [WP_S]  the stage's MMAs have retired (each CTA's own copy)
+  uint64_t* tmem_full = empty + WP_S;                 // accumulator complete (each CTA's own copy)
+  uint64_t* tmem_empty = tmem_full + 1;               // epilogue warps of the pair (the leader's copy is used)
+  uint32_t* tmem_slot = reinterpret_cast<uint32_t*>(smem + L::OFF_TMEM);
+
+  const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+  const uint32_t rank = cluster_ctarank();            // 0 = leader (issues the MMAs)
+  const int pair = blockIdx.x >> 1, npairs = gridDim.x >> 1;
+  const int num_kb = K / 64;
+  const int num_sb = (num_kb + 3) / 4;                // stages per tile (the last may hold fewer than four k-blocks)
+  // channel tiles run fastest: the pairs at work at one time share a few token tiles, which stay in L2
+  const int tiles_n = (N + 255) / 256;
+  const int num_tiles = tiles_n * ((M + 255) / 256);
+  const uint32_t limit = wait_limit();
+
+  // The weights do not depend on the kernel before this one: the first ring-full of them is requested
+  // (local barriers only) before anything else is set up and before that kernel's completion is awaited.
+  int pre = 0;
+  if (threadIdx.x == 0) {
+    tma_prefetch_desc(&tmap_w);
+    for (int s = 0; s < SS; ++s) mbar_init(&st_full[s], 1);
+    mbar_fence_init();
+    {
+      int t = pair, sb = 0;
+      while (pre < SS && t < num_tiles) {
+        mbar_arrive_expect_tx(&st_full[pre], L::W_ST);
+        tma_load_2d(smem + L::OFF_W_ST + pre * L::W_ST, &tmap_w, &st_full[pre], sb * 128,
+                    (t % tiles_n) * 256 + static_cast<int>(rank) * 128);
+        ++pre;
+        if (++sb >= num_sb) {
+          sb = 0;
+          t += npairs;
+        }
+      }
+    }
+    tma_prefetch_desc(&tmap_z);
+    for (int s = 0; s < SS; ++s) mbar_init(&st_empty[s], 4);          // the four warps of one converter group
+    for (int s = 0; s < WP_S; ++s) {
+      mbar_init(&t_full[s], 1);
+      mbar_init(&full[s], 2 * 4);                                      // one converter group in each CTA
+      mbar_init(&empty[s], 1);
+    }
+    mbar_init(tmem_full, 1);
+    mbar_init(tmem_empty, 2 * WP_EPI_WARPS);
+    mbar_fence_init();
+  }
+  if (warp == 1) {
+    tmem_alloc_pair(tmem_slot, 512);
+    tmem_relinquish_pair();
+  }
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();                                 // both CTAs' barriers exist before any remote arrival
+  tc_fence_after_sync();
+  const uint32_t tmem_base = *tmem_slot;
+  griddep_wait();                                     // Z16 may come from the kernel launched before this one
+
+  if (warp == 0) {
+    // ------------------------------ TMA producer ------------------------------------------
+    if (lane == 0) {                                  // thread 0: it knows how many blocks are on their way
+      uint32_t it = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+        const int ch0 = (tile % tiles_n) * 256 + static_cast<int>(rank) * 128;
+        const int tok0 = (tile / tiles_n) * 256 + static_cast<int>(rank) * 128;
+        for (int sb = 0; sb < num_sb && ok; ++sb, ++it) {
+          if (it >= static_cast<uint32_t>(pre)) {
+            const int ss = it % SS;
+            ok = mbar_wait(&st_empty[ss], ((it / SS) & 1) ^ 1, WP_ST_EMPTY, limit);
+            if (!ok) break;
+            mbar_arrive_expect_tx(&st_full[ss], L::W_ST);
+            tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, &tmap_w, &st_full[ss], sb * 128, ch0);
+          }
+          const int s = it % WP_S;
+          const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
+          ok = mbar_wait(&empty[s], ((it / WP_S) & 1) ^ 1, WP_EMPTY_T, limit);
+          if (!ok) break;
+          mbar_arrive_expect_tx(&t_full[s], static_cast<uint32_t>(nk * L::T_KB));
+          for (int h = 0; h < nk; ++h)
+            tma_load_2d(smem + L::OFF_T + s * L::T_TILE + h * L::T_KB, &tmap_z, &t_full[s], (4 * sb + h) * 64, tok0);
+        }
+      }
+    }
+  } else if (warp == 1) {
+    // ------------------------------ MMA issuer (leader CTA) -------------------------------
+    if (rank == 0 && elect_one()) {
+      constexpr uint32_t idesc = umma_idesc(/*c=f32*/ 1, /*a=f16*/ 0, /*b=f16*/ 0, 256, 256);
+      const uint64_t t_desc0 = umma_desc_sw128(smem_u32(smem + L::OFF_T));
+      uint32_t it = 0, tcount = 0;
+      bool ok = true;
+      for (int tile = pair; tile < num_tiles && ok; tile += npairs, ++tcount) {
+        ok = mbar_wait(tmem_empty, (tcount & 1) ^ 1, WP_TMEM_EMPTY, limit);
+        if (!ok) break;
+        tc_fence_after_sync();
+        for (int sb = 0; sb < num_sb; ++sb, ++it) {
+          const int s = it % WP_S;
+          const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
+          ok = mbar_wait(&full[s], (it / WP_S) & 1, WP_FULL, limit);
+          if (!ok) break;
+          tc_fence_after_sync();
+          const uint32_t a_tmem = tmem_base + WP_A_COL0 + s * 128;
+          const uint64_t td = t_desc0 + static_cast<uint64_t>((s * L::T_TILE) >> 4);
+#pragma unroll
+          for (int h = 0; h < 4; ++h) {
+            if (h < nk) {
+#pragma unroll
+              for (int k = 0; k < 4; ++k)         // K = 16 fp16: eight 32-bit columns of A, 32 bytes of a token row
+                umma_f16_ts_pair(tmem_base, a_tmem + 32 * h + 8 * k, td + ((h * L::T_KB + k * 32) >> 4), idesc,
+                                 (sb | h | k) != 0 ? 1u : 0u);
+            }
+          }
+          umma_commit_pair_mc(&empty[s], 3);          // frees ring stage s in both CTAs
+        }
+        umma_commit_pair_mc(tmem_full, 3);            // accumulator complete (or abandoned)
+      }
+    }
+  } else if (warp < 2 + WOD_CONV_WARPS) {
+    // ------------------------------ weight converters: staging -> registers -> tensor memory ------
+    const int q = warp & 3;
+    const int grp = (warp - 2) >> 2;                    // this group's ring stage
+    const int r = q * 32 + lane;                        // channel of the CTA's 128 = TMEM lane
+    const uint32_t lane_addr = static_cast<uint32_t>(q * 32) << 16;
+    uint32_t it = 0;
+    bool ok = true;
+    for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
+      for (int sb = 0; sb < num_sb && ok; ++sb, ++it) {
+        if ((it % WP_S) != static_cast<uint32_t>(grp)) continue;
+        const int ss = it % SS, s = grp;
+        const int nk = (num_kb - 4 * sb) < 4 ? (num_kb - 4 * sb) : 4;
+        ok = mbar_wait(&st_full[ss], (it / SS) & 1, WP_ST_FULL, limit);
+        if (!ok) break;
+        const unsigned char* row = smem + L::OFF_W_ST + ss * L::W_ST + r * 128;
+        uint4 w[8];
+#pragma unroll
+        for (int c = 0; c < 8; ++c) w[c] = *reinterpret_cast<const uint4*>(row + ((c ^ (r & 7)) << 4));
+        ok = mbar_wait(&empty[s], ((it / WP_S) & 1) ^ 1, WP_EMPTY_A, limit);
+        if (!ok) break;
+        tc_fence_after_sync();
+#pragma unroll
+        for (int h = 0; h < 4; ++h) {                   // k-block h: chunks 2h, 2h+1 -> 32 columns
+          if (h < nk) {
+            uint32_t v[32];
+#pragma unroll
+            for (int j = 0; j < 2; ++j) {
+              const uint4 x = w[2 * h + j];
+              const uint32_t xs[4] = {x.x, x.y, x.z, x.w};
+#pragma unroll
+              for (int g = 0; g < 4; ++g) {
+                const uint4 f = widen_word(xs[g]);
+                v[16 * j + 4 * g + 0] = f.x;
+                v[16 * j + 4 * g + 1] = f.y;
+                v[16 * j + 4 * g + 2] = f.z;
+                v[16 * j + 4 * g + 3] = f.w;
+              }
+            }
+            tmem_st_32x32b_x32(tmem_base + lane_addr + WP_A_COL0 + s * 128 + h * 32, v);
+          }
+        }
+        tmem_wait_st();
+        tc_fence_before_sync();
+        // the stage also needs this CTA's tokens: the leader learns of both with one arrival
+        ok = mbar_wait(&t_full[s], (it / WP_S) & 1, WP_T_FULL, limit);
+        if (!ok) break;
+        __syncwarp();
+        if (lane == 0) {
+          mbar_arrive_cluster(&full[s], 0);
+          mbar_arrive(&st_empty[ss]);
+        }
+      }
+    }
+  } else {
+    // ------------------------------ epilogue warps ------------------------------------------
+    const int q = warp & 3;                             // TMEM lane quarter this warp may read
+    const int half = (warp - (2 + WOD_CONV_WARPS)) >> 2;  // its 128 of the 256 token columns
+    uint32_t tcount = 0;
+    bool ok = true;
+    for (int tile = pair; tile < num_tiles && ok; tile += npairs, ++tcount) {
+      const int ch = (tile % tiles_n) * 256 + static_cast<int>(rank) * 128 + q * 32 + lane;
+      const int tok0 = (tile / tiles_n) * 256 + half * 128;
+      const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;
+      ok = mbar_wait(tmem_full, tcount & 1, WP_TMEM_FULL, limit);
+      if (!ok) break;
+      tc_fence_after_sync();
+      const uint32_t tmem_d = tmem_base + (static_cast<uint32_t>(q * 32) << 16) + half * 128;
+#pragma unroll
+      for (int c = 0; c < 8; ++c) {
+        uint32_t r[16];
+        tmem_ld_32x32b_x16(tmem_d + c * 16, r);
+        tmem_wait_ld();
+        if (c == 7) {                                   // last read of this warp: hand the accumulator back
+          tc_fence_before_sync();
+          __syncwarp();
+          if (lane == 0) mbar_arrive_cluster(tmem_empty, 0);
+        }
+        if (ch < N) {
+#pragma unroll
+          for (int e = 0; e < 16; ++e) {
+            const int tok = tok0 + c * 16 + e;
+            if (tok < M) Y[static_cast<size_t>(tok) * N + ch] = __float2half_rn(__uint_as_float(r[e]) * swv);
+          }
+        }
+      }
+    }
+  }
+
+  // Neither CTA may leave while its partner can still reach its shared memory, barriers or TMEM.
+  tc_fence_before_sync();
+  __syncthreads();
+  cluster_sync_all();
+  if (warp == 1) {
+    tc_fence_after_sync();
+    tmem_dealloc_pair(tmem_base, 512);
+  }
+}
+
 // One or two tokens: dot products on the CUDA cores.  The product is pure streaming then (29 MB of
 // packed weights against a few MFLOP), and the tensor-core forms pay more in hand-overs than the read
 // costs.  Each warp takes four weight rows at a time; every lane reads 16-byte pieces of them straight
@@ -877,6 +1146,34 @@ sq_status_t launch_wo_decode(const void* Z16, const void* Wq, const void* sw, in
   return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
 }
 
+template <int SS>
+sq_status_t launch_wo_pair(const void* Z16, const void* Wq, const void* sw, int M, int N, int K, void* Y, cudaStream_t s) {
+  using L = WoPairSmem<SS>;
+  static_assert(L::DYN_BYTES <= 227 * 1024, "shared-memory plan does not fit");
+  EncodeTiledFn enc = get_encode_fn();
+  if (!enc) return SQ_ERR_CUDA;
+  CUtensorMap mz, mw;
+  const cuuint64_t dims[2] = {static_cast<cuuint64_t>(K), static_cast<cuuint64_t>(M)};
+  const cuuint64_t strides[1] = {static_cast<cuuint64_t>(K) * 2};
+  const cuuint32_t box[2] = {64, 128};
+  const cuuint32_t estr[2] = {1, 1};
+  if (enc(&mz, CU_TENSOR_MAP_DATA_TYPE_FLOAT16, 2, const_cast<void*>(Z16), dims, strides, box, estr,
+          CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+          CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
+    return SQ_ERR_CUDA;
+  if (!make_packed_map(&mw, Wq, N, K / 2, 128)) return SQ_ERR_CUDA;
+  auto kern = wo_gemm_pair_kernel<SS>;
+  if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), L::DYN_BYTES)) return SQ_ERR_CUDA;
+  const int sms = sm_count();
+  if (sms <= 0) return SQ_ERR_CUDA;
+  const int tiles = ((N + 255) / 256) * ((M + 255) / 256);
+  const int pairs = tiles < sms / 2 ? tiles : sms / 2;
+  const cudaError_t err = launch_maybe_pdl(kern, dim3(2 * pairs), dim3(WP_THREADS), L::DYN_BYTES, s, mz, mw,
+                                           static_cast<const __half*>(sw), M, N, K, static_cast<__half*>(Y));
+  count_launch();
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
+}
+
 template <int MT>
 sq_status_t launch_wo_gemv(const void* Z16, const void* Wq, const void* sw, int M, int N, int K, void* Y, cudaStream_t s) {
   const int sms = sm_count();
@@ -916,6 +1213,8 @@ sq_status_t launch_wo_gemm(const void* Z16, const void* Wq, const void* sw, int6
     // operand cost no shared-memory traffic at all, which is what bounds the kernel below (2048 x 4096 x
     // 4096: 76 us there).  From 256 channels on, two channel tiles share every token block (half the
     // token traffic out of L2 per flop: 65 -> 61 us on that shape, 1.85 -> 1.65 ms on 4096 x 28672 x 8192).
+    // Above 128 tokens: CTA pairs on 256 x 256 tiles (an MMA's 4 KB of A then feed twice the arithmetic).
+    if (M > 128 && N >= 256) return launch_wo_pair<4>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
     if (N >= 256) return launch_wo_decode<128, 2, 4, 2>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
     return launch_wo_decode<128, 2, 4>(Z16, Wq, sw, (int)M, (int)N, (int)K, Y, s);
   }
