@@ -54,7 +54,7 @@ NCU_TRAFFIC = {
     ("rotate_quant", "llama2_70b_gateup_prefill"): 69889536,   # rotate_quant_tc_kernel, n2 = 128
     ("rotate_quant", "llama2_70b_down_prefill"): 275649024,    # rotate_quant_pair_kernel, n2 = 128
     ("wo_gemm", "llama3_8b_up_decode_m16"): 29558016,       # wo_gemm_tmem_kernel<16, 4, 8> (W4A16)
-    ("wo_gemm", "llama2_7b_qkvo_prefill"): 25266944,        # wo_gemm_tmem_kernel<128, 2, 4> (W4A16; Y stayed in L2)
+    ("wo_gemm", "llama2_7b_qkvo_prefill"): 25311744,        # wo_gemm_pair_kernel (W4A16; Y stayed in L2)
 }
 
 
@@ -552,7 +552,8 @@ def weight_only_entry(sq, torch, w, bits, pk, l2, quick=False):
                 "algorithmic_bytes": gemm_bytes_wo}
     else:
         tf = flops / (gemm_ms * 1e-3) / 1e12
-        roof = {"kernel": "wo_gemm_tmem_kernel" if (N >= 128 and K % 64 == 0 and N % 8 == 0) else "wo_gemm_tc_kernel",
+        tc_ok = N >= 128 and K % 64 == 0 and N % 8 == 0
+        roof = {"kernel": ("wo_gemm_pair_kernel" if (M > 128 and N >= 256) else "wo_gemm_tmem_kernel") if tc_ok else "wo_gemm_tc_kernel",
                 "bound": "tensor", "achieved": tf, "peak": pk["bf16_tflops"],
                 "unit": "TFLOP/s", "frac": tf / pk["bf16_tflops"],
                 "traffic": NCU_TRAFFIC.get(("wo_gemm", w.name)) if bits == 4 else None, "ms_per_launch": gemm_ms,
