@@ -171,6 +171,22 @@ def test_wo_gemm_is_bit_exact_on_small_integers(sq, M, N, K):
     assert np.array_equal(Yg.view(np.uint16), Yo.view(np.uint16))
 
 
+@pytest.mark.parametrize("M,N,K", [(2048, 4096, 4096), (2048, 4096, 11008), (4096, 28672, 8192)])
+def test_wo_gemm_full_size_bit_exact_on_sampled_rows(sq, M, N, K):
+    """The benchmark's prefill shapes (up to 24 tiles per CTA pair, 43 stages per tile, weights beyond
+    L2): same integer construction as above (|partial sums| <= 64 K < 2^24), every channel of sampled
+    token rows against the oracle, bit for bit."""
+    rng = np.random.default_rng(M + N + K)
+    Z16 = rng.integers(-8, 9, size=(M, K), dtype=np.int8).astype(np.float16)
+    codes = rng.integers(-8, 8, size=(N, K), dtype=np.int8)
+    sw = (2.0 ** rng.integers(-12, -6, size=N)).astype(np.float16)
+    Yg = _run_wo_gemm(sq, Z16, codes, sw)
+    rows = np.unique(np.concatenate([[0, 127, 128, 255, 256, M - 1], rng.integers(0, M, size=26)]))
+    for c0 in range(0, N, 4096):                      # the oracle widens the codes to float64: in blocks of channels
+        Yo = ora.gemm_w4a16(Z16[rows], codes[c0:c0 + 4096], sw[c0:c0 + 4096])
+        assert np.array_equal(Yg[rows, c0:c0 + 4096].view(np.uint16), Yo.view(np.uint16))
+
+
 def test_wo_gemm_random_shapes_bit_exact(sq):
     """Forty seeded random shapes over every kernel of the product (dot products, decode form with and
     without the K split, prefill form with both tile widths, the plain kernel), small integers so that
