@@ -188,12 +188,12 @@ def test_wo_gemm_full_size_bit_exact_on_sampled_rows(sq, M, N, K):
 
 
 def test_wo_gemm_random_shapes_bit_exact(sq):
-    """Forty seeded random shapes over every kernel of the product (dot products, decode form with and
-    without the K split, prefill form with both tile widths, the plain kernel), small integers so that
-    the result must equal the oracle's bit for bit."""
+    """Forty-eight seeded random shapes over every kernel of the product (dot products, the single-CTA
+    form with and without the K split and with one or two channel tiles, the CTA-pair form, the plain
+    kernel), small integers so that the result must equal the oracle's bit for bit."""
     rng = np.random.default_rng(20240607)
-    for trial in range(40):
-        kind = trial % 5
+    for trial in range(48):
+        kind = trial % 6
         if kind == 0:
             M, N, K = int(rng.integers(1, 3)), int(rng.integers(1, 400)), 32 * int(rng.integers(1, 200))
         elif kind == 1:
@@ -202,6 +202,8 @@ def test_wo_gemm_random_shapes_bit_exact(sq):
             M, N, K = int(rng.integers(3, 65)), 8 * int(rng.integers(16, 40)), 64 * int(rng.integers(64, 200))
         elif kind == 3:
             M, N, K = int(rng.integers(65, 400)), 8 * int(rng.integers(1, 200)), 64 * int(rng.integers(1, 40))
+        elif kind == 5:
+            M, N, K = int(rng.integers(129, 1200)), 8 * int(rng.integers(32, 500)), 64 * int(rng.integers(1, 24))
         else:
             M, N, K = int(rng.integers(1, 40)), int(rng.integers(1, 150)), 8 * int(rng.integers(1, 60))
         Z16 = rng.integers(-8, 9, size=(M, K)).astype(np.float16)
