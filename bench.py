@@ -682,15 +682,18 @@ def run_ours(args, w):
             dist.barrier()
             torch.cuda.synchronize()
 
-    warm = max(args.warmup, 3)
-    for i in range(warm):
-        layer.step(i)
-    sync_all()
-
+    # the clock sampler is up before the warm-up, so that nothing but the barrier and the synchronize
+    # stands between the last warm-up step and the timed region (an idle GPU drops its clocks)
     sampler = ClockSampler(ClockSampler.resolve(torch, local_rank))
     if rank == 0:
         sampler.start()
         time.sleep(0.3)
+    sync_all()
+
+    warm = max(args.warmup, 3)
+    for i in range(warm):
+        layer.step(i)
+    sync_all()
 
     # ---- timed region: exactly K steps of sq_linear ------------------------------------------
     launches0 = sq.sq_kernel_launch_count()
