@@ -299,8 +299,12 @@ def test_linear_wo_full_size_sampled_rows(sq, w):
 
 
 # ------------------------------------------------------------------ the grouped W4A4 layer
+@pytest.mark.parametrize("shared", [False, True], ids=["own_handles", "one_handle"])
 @pytest.mark.parametrize("counts", [[5, 0, 3, 1], [64, 7, 130, 0, 0, 9, 1, 40], [0, 0, 12], [300]])
-def test_linear_grouped_matches_oracle_and_the_per_expert_calls(sq, counts):
+def test_linear_grouped_matches_oracle_and_the_per_expert_calls(sq, counts, shared):
+    """Each expert with a handle of its own, and all experts on one handle (then steps 1 and 2 run once
+    over all rows and only step 3 per expert): against the oracle, and bit for bit against sq_linear on
+    each expert's rows."""
     torch = torch_mod()
     n1, n2, N = 64, 64, 264
     K = n1 * n2
@@ -313,9 +317,13 @@ def test_linear_grouped_matches_oracle_and_the_per_expert_calls(sq, counts):
     Ws = [(0.02 * rng.standard_normal((N, K))).astype(np.float16) for _ in range(E)]
     rots_o = []
     for e in range(E):
-        cal = wl.make_activations(wl.small("grpc", 64, n1, n2, N, seed=70 + e)).astype(np.float32)
-        rots_o.append(ora.build_rotation(cal, n1, n2, O=ora.haar_orthogonal(n1 - 2, np.random.default_rng(e))))
-    rots = [sq.sq_rotation_from_factors(R1, R2) for R1, R2 in rots_o]
+        cal = wl.make_activations(wl.small("grpc", 64, n1, n2, N, seed=70 + (0 if shared else e))).astype(np.float32)
+        rots_o.append(ora.build_rotation(cal, n1, n2, O=ora.haar_orthogonal(n1 - 2, np.random.default_rng(0 if shared else e))))
+    if shared:
+        one = sq.sq_rotation_from_factors(*rots_o[0])
+        rots = [one] * E
+    else:
+        rots = [sq.sq_rotation_from_factors(R1, R2) for R1, R2 in rots_o]
     wqs, sws = [], []
     for e in range(E):
         q, s = Guarded(N * K // 2), Guarded(N * 2)
@@ -331,7 +339,8 @@ def test_linear_grouped_matches_oracle_and_the_per_expert_calls(sq, counts):
     launched = sq.sq_kernel_launch_count() - before
     _sync_ok(sq)
     y.check()
-    assert launched == 2 * sum(1 for c in counts if c > 0)          # experts without tokens cost nothing
+    with_rows = sum(1 for c in counts if c > 0)                     # experts without tokens cost nothing
+    assert launched == (1 + with_rows if shared and with_rows >= 2 else 2 * with_rows)
     Yg = y.numpy(np.float16, (M, N))
     Yo = ora.linear_grouped(X, offsets, Ws, rots_o).astype(np.float64)
     for e in range(E):
@@ -343,7 +352,7 @@ def test_linear_grouped_matches_oracle_and_the_per_expert_calls(sq, counts):
             sq.sq_linear(rots[e], dX[a:b], b - a, wqs[e], sws[e], N, K, wsp, nbytes, y1)
             _sync_ok(sq)
             assert np.array_equal(y1.numpy(np.float16, (b - a, N)).view(np.uint16), Yg[a:b].view(np.uint16))
-    for r in rots:
+    for r in ([rots[0]] if shared else rots):
         r.close()
 
 
