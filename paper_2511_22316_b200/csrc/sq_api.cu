@@ -599,6 +599,33 @@ sq_status_t sq_linear_grouped(const sq_rotation_t* const* rots, int32_t E, const
     unsigned char* sx = ws + align_up(static_cast<size_t>(M) * (K / 2), 256);
     sq_status_t st = sq::rotate_quant_dispatch(shared, X, M, Xq, sx, nullptr, s);
     if (st != SQ_OK) return st;
+    // Decode-sized expert batches (at most 64 rows each): step 3 for up to sixteen experts per launch, a
+    // tile being (expert, 128 channels) -- one start-up and one stream of weights instead of one per expert.
+    bool small = true;
+    for (int32_t e = 0; e < E && small; ++e) {
+      const int64_t r = offsets[e + 1] - offsets[e];
+      if (r > 0 && !sq::gemm_decode_supported(r, N, K)) small = false;
+    }
+    if (small) {
+      const int cap = sq::gemm_decode_max_groups();
+      std::vector<const void*> gw, gs;
+      std::vector<int64_t> g0, gr;
+      auto flush = [&]() -> sq_status_t {
+        if (gw.empty()) return SQ_OK;
+        const sq_status_t fs = sq::launch_w4a4_gemm_decode_grouped(Xq, sx, M, static_cast<int>(gw.size()), gw.data(),
+                                                                   gs.data(), g0.data(), gr.data(), static_cast<int>(N),
+                                                                   static_cast<int>(K), Y, s);
+        gw.clear(); gs.clear(); g0.clear(); gr.clear();
+        return fs;
+      };
+      for (int32_t e = 0; e < E; ++e) {
+        const int64_t r0 = offsets[e], r = offsets[e + 1] - r0;
+        if (r == 0) continue;
+        gw.push_back(Wq[e]); gs.push_back(sw[e]); g0.push_back(r0); gr.push_back(r);
+        if (static_cast<int>(gw.size()) == cap && (st = flush()) != SQ_OK) return st;
+      }
+      return flush();
+    }
     for (int32_t e = 0; e < E; ++e) {
       const int64_t r0 = offsets[e], r = offsets[e + 1] - r0;
       if (r == 0) continue;

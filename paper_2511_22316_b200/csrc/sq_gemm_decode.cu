@@ -114,16 +114,30 @@ __device__ __forceinline__ void unpack_rows(const unsigned char* __restrict__ st
   }
 }
 
+// The grouped form (one launch for the experts of a mixture-of-experts layer): expert g has its own
+// packed weights and channel steps and owns `rows[g]` <= NT consecutive token rows from `r0[g]` on, of a
+// common Xq, sx and Y.  A tile is (expert, 128 channels); nothing else changes.
+constexpr int D_MAX_GROUPS = 16;
+struct alignas(64) DecGroups {
+  CUtensorMap wmap[D_MAX_GROUPS];
+  const __half* sw[D_MAX_GROUPS];
+  int r0[D_MAX_GROUPS];
+  int rows[D_MAX_GROUPS];
+  int count;
+};
+
 // The kernel's body for CTA `cta` of `ncta` (a multiple of the cluster size `splits`).  `tokens_ready`:
 // nullptr when the tokens come from the kernel before this one in the stream (programmatic dependent
 // launch); else a counter that the token-producing CTAs of the SAME launch bump to `tokens_target`
 // (the fused kernel of sq_linear_fused.cu).
-template <int NT>
+// GROUPED: the tiles run over the experts of `G` (splits == 1, no token counter); M, sw and tmap_w are unused.
+template <int NT, bool GROUPED = false>
 __device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w, const CUtensorMap& tmap_x,
                                                       const __half* __restrict__ sx, const __half* __restrict__ sw,
                                                       int M, int N, int K, int splits, __half* __restrict__ Y,
                                                       int32_t* __restrict__ accdbg, int cta, int ncta,
-                                                      const uint32_t* tokens_ready, uint32_t tokens_target) {
+                                                      const uint32_t* tokens_ready, uint32_t tokens_target,
+                                                      const DecGroups* G = nullptr) {
   using L = DecSmem<NT>;
   constexpr int S_ST = L::S_ST;
   griddep_launch_dependents();          // a rotate kernel launched behind this one may set itself up on the idle SMs
@@ -145,7 +159,8 @@ __device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w,
   const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
   const int num_kb = K / 128;
   const int num_sb = (num_kb + 1) / 2;                 // blocks of 256 channels (the last may be half)
-  const int tiles = (N + 127) / 128;
+  const int tiles_pe = (N + 127) / 128;                // channel tiles (per expert)
+  const int tiles = GROUPED ? tiles_pe * G->count : tiles_pe;
   const uint32_t limit = wait_limit();
 
   // The cluster (a single CTA when splits == 1) takes the tiles cid, cid + ncl, ...; CTA `crank`
@@ -160,7 +175,7 @@ __device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w,
   // "empty" barriers may not exist yet).  The weights do not depend on the kernel before this
   // one, the tokens do: with `defer_x` only the weights are requested and the blocks are noted.
   int p_tile = cid, p_sb = b0, pre_n = 0;
-  int pre_sb[S_ST];
+  int pre_sb[S_ST], pre_row[S_ST];
   uint32_t p_it = 0;
   auto produce = [&](uint32_t budget, bool defer_x) -> bool {
     while (budget > 0 && p_tile < tiles) {
@@ -168,9 +183,16 @@ __device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w,
       if (p_it >= static_cast<uint32_t>(S_ST) &&
           !mbar_wait(&st_empty[ss], ((p_it / S_ST) & 1) ^ 1, DSITE_ST_EMPTY, limit)) return false;
       mbar_arrive_expect_tx(&st_full[ss], L::W_ST + L::X_ST);
-      tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, &tmap_w, &st_full[ss], p_sb * 128, p_tile * 128);
-      if (defer_x) pre_sb[pre_n++] = p_sb;
-      else tma_load_2d(smem + L::OFF_X_ST + ss * L::X_ST, &tmap_x, &st_full[ss], p_sb * 128, 0);
+      const int pg = GROUPED ? p_tile / tiles_pe : 0;                  // expert of the tile
+      const int xrow = GROUPED ? G->r0[pg] : 0;                        // its first token row
+      tma_load_2d(smem + L::OFF_W_ST + ss * L::W_ST, GROUPED ? &G->wmap[pg] : &tmap_w, &st_full[ss], p_sb * 128,
+                  (GROUPED ? p_tile % tiles_pe : p_tile) * 128);
+      if (defer_x) {
+        pre_sb[pre_n] = p_sb;
+        pre_row[pre_n++] = xrow;
+      } else {
+        tma_load_2d(smem + L::OFF_X_ST + ss * L::X_ST, &tmap_x, &st_full[ss], p_sb * 128, xrow);
+      }
       ++p_it;
       --budget;
       if (++p_sb >= b1) {
@@ -226,7 +248,7 @@ __device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w,
     if (lane == 0 && (tokens_ready == nullptr || wait_counter(tokens_ready, tokens_target, DSITE_TOKENS, limit))) {
       if (tokens_ready != nullptr) mbar_arrive(tok_seen);
       for (int i = 0; i < pre_n; ++i)
-        tma_load_2d(smem + L::OFF_X_ST + i * L::X_ST, &tmap_x, &st_full[i], pre_sb[i] * 128, 0);
+        tma_load_2d(smem + L::OFF_X_ST + i * L::X_ST, &tmap_x, &st_full[i], pre_sb[i] * 128, pre_row[i]);
       produce(0xFFFFFFFFu, false);
     }
   } else if (warp == 1) {
@@ -369,7 +391,7 @@ __device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w,
     const bool piece_mine = static_cast<uint32_t>((q * 32 + piece * 8) / rows_per) == crank;
     const uint32_t pick = (prow & 1) ? 0x7632u : 0x5410u;            // the odd or the even token of a pair
     // The tokens' scales as floats (zero beyond M): read once, before any accumulator is ready.
-    if (et < NT) {
+    if (!GROUPED && et < NT) {
       const bool there = tokens_ready == nullptr || mbar_wait(tok_seen, 0, DSITE_TOKENS, limit);
       // written during this launch by another CTA in the fused form: read past the L1 / read-only path
       const __half v = (et < M && there)
@@ -385,8 +407,13 @@ __device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w,
     for (int tile = cid; tile < tiles && ok; tile += ncl, ++icount) {
       const uint32_t acc = icount % D_ACCS;
       const uint32_t par = 0u, g = icount;                            // reduce buffer and its use count
-      const int ch = tile * 128 + rowl;                    // output channel of this thread
-      const float swv = (ch < N) ? __half2float(sw[ch]) : 0.0f;      // in flight while the accumulator is awaited
+      const int tg = GROUPED ? tile / tiles_pe : 0;        // expert of the tile
+      const int ct = GROUPED ? tile % tiles_pe : tile;     // channel tile
+      const int Mt = GROUPED ? G->rows[tg] : M;            // token rows of the tile
+      const int trow0 = GROUPED ? G->r0[tg] : 0;           // the first of them in Xq, sx and Y
+      const __half* swp = GROUPED ? G->sw[tg] : sw;
+      const int ch = ct * 128 + rowl;                      // output channel of this thread
+      const float swv = (ch < N) ? __half2float(swp[ch]) : 0.0f;     // in flight while the accumulator is awaited
       if (splits > 1 && eg == 0 && mine && rloc == 0) mbar_arrive_expect_tx(&red_full[par], red_bytes);
       ok = mbar_wait(&tmem_full[acc], (icount / D_ACCS) & 1, DSITE_TMEM_FULL, limit);
       if (!ok) break;
@@ -462,7 +489,16 @@ __device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w,
               }
             }
             const int e0 = t0 + 4 * c;
-            const float4 s4 = *reinterpret_cast<const float4*>(sxs + e0);
+            float4 s4;
+            if constexpr (GROUPED) {                     // the experts' token steps straight from global memory
+              const __half* sxg = sx + trow0;
+              s4.x = (e0 + 0 < Mt) ? __half2float(sxg[e0 + 0]) : 0.0f;
+              s4.y = (e0 + 1 < Mt) ? __half2float(sxg[e0 + 1]) : 0.0f;
+              s4.z = (e0 + 2 < Mt) ? __half2float(sxg[e0 + 2]) : 0.0f;
+              s4.w = (e0 + 3 < Mt) ? __half2float(sxg[e0 + 3]) : 0.0f;
+            } else {
+              s4 = *reinterpret_cast<const float4*>(sxs + e0);
+            }
             const __half2 h01 = __floats2half2_rn((__int_as_float(0x4B400000 + a.x) - 12582912.0f) * (s4.x * swv),
                                                   (__int_as_float(0x4B400000 + a.y) - 12582912.0f) * (s4.y * swv));
             const __half2 h23 = __floats2half2_rn((__int_as_float(0x4B400000 + a.z) - 12582912.0f) * (s4.z * swv),
@@ -473,13 +509,13 @@ __device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w,
               const int32_t av[4] = {a.x, a.y, a.z, a.w};
 #pragma unroll
               for (int x = 0; x < 4; ++x)
-                if (e0 + x < M) accdbg[static_cast<size_t>(e0 + x) * N + ch] = av[x];
+                if (e0 + x < Mt) accdbg[static_cast<size_t>(trow0 + e0 + x) * N + ch] = av[x];
             }
           }
         }
         __syncwarp();
         {
-          const int ch0 = tile * 128 + q * 32 + piece * 8;
+          const int ch0 = ct * 128 + q * 32 + piece * 8;
 #pragma unroll
           for (int pass = 0; pass < CH / 8; ++pass) {
             const int e = t0 + 8 * pass + prow;
@@ -490,7 +526,8 @@ __device__ __forceinline__ void w4a4_gemm_decode_body(const CUtensorMap& tmap_w,
             v.y = __byte_perm(w0.z, w0.w, pick);
             v.z = __byte_perm(w1.x, w1.y, pick);
             v.w = __byte_perm(w1.z, w1.w, pick);
-            if (piece_mine && e < M && ch0 < N) *reinterpret_cast<uint4*>(Y + static_cast<size_t>(e) * N + ch0) = v;
+            if (piece_mine && e < Mt && ch0 < N)
+              *reinterpret_cast<uint4*>(Y + static_cast<size_t>(trow0 + e) * N + ch0) = v;
           }
         }
       }
@@ -524,6 +561,14 @@ w4a4_gemm_decode_kernel(const __grid_constant__ CUtensorMap tmap_w, const __grid
                         int splits, __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
   w4a4_gemm_decode_body<NT>(tmap_w, tmap_x, sx, sw, M, N, K, splits, Y, accdbg, static_cast<int>(blockIdx.x),
                             static_cast<int>(gridDim.x), nullptr, 0u);
+}
+
+template <int NT>
+__global__ void __launch_bounds__(D_THREADS, 1)
+w4a4_gemm_decode_grouped_kernel(const __grid_constant__ DecGroups G, const __grid_constant__ CUtensorMap tmap_x,
+                                const __half* __restrict__ sx, int N, int K, __half* __restrict__ Y) {
+  w4a4_gemm_decode_body<NT, true>(G.wmap[0], tmap_x, sx, nullptr, 0, N, K, 1, Y, nullptr, static_cast<int>(blockIdx.x),
+                                  static_cast<int>(gridDim.x), nullptr, 0u, &G);
 }
 
 // Largest number of clusters of `s` CTAs of this kernel that the device holds at once.
@@ -604,7 +649,52 @@ sq_status_t launch_decode(const void* Xq, const void* sx, const void* Wq, const 
   return err == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
 }
 
+template <int NT>
+sq_status_t launch_decode_grouped(const void* Xq, const void* sx, int64_t M_total, int count, const void* const* Wq,
+                                  const void* const* sw, const int64_t* r0, const int64_t* rows, int N, int K, void* Y,
+                                  cudaStream_t s) {
+  using L = DecSmem<NT>;
+  const int sms = sm_count();
+  if (sms <= 0) return SQ_ERR_CUDA;
+  auto kern = w4a4_gemm_decode_grouped_kernel<NT>;
+  if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), L::DYN_BYTES)) return SQ_ERR_CUDA;
+  DecGroups G;
+  CUtensorMap mx;
+  if (!make_packed_map(&mx, Xq, static_cast<uint64_t>(M_total), K / 2, NT)) return SQ_ERR_CUDA;
+  for (int g = 0; g < D_MAX_GROUPS; ++g) {
+    const int src = g < count ? g : 0;                   // unused entries repeat the first (never read)
+    if (!make_packed_map(&G.wmap[g], Wq[src], N, K / 2, 128)) return SQ_ERR_CUDA;
+    G.sw[g] = static_cast<const __half*>(sw[src]);
+    G.r0[g] = static_cast<int>(r0[src]);
+    G.rows[g] = static_cast<int>(rows[src]);
+  }
+  G.count = count;
+  const int tiles = ((N + 127) / 128) * count;
+  const int grid = tiles < sms ? tiles : sms;
+  const cudaError_t err = launch_maybe_pdl(kern, dim3(static_cast<unsigned>(grid)), dim3(D_THREADS),
+                                           static_cast<size_t>(L::DYN_BYTES), s, G, mx, static_cast<const __half*>(sx), N,
+                                           K, static_cast<__half*>(Y));
+  count_launch();
+  return err == cudaSuccess ? SQ_OK : SQ_ERR_CUDA;
+}
+
 }  // namespace
+
+int gemm_decode_max_groups() { return D_MAX_GROUPS; }
+
+// Step 3 for up to D_MAX_GROUPS experts in one launch: expert g owns rows[g] (1..64) token rows from r0[g]
+// on of Xq [M_total x K/2], sx and Y, and has its own Wq[g], sw[g].  Shapes as gemm_decode_supported.
+sq_status_t launch_w4a4_gemm_decode_grouped(const void* Xq, const void* sx, int64_t M_total, int count,
+                                            const void* const* Wq, const void* const* sw, const int64_t* r0,
+                                            const int64_t* rows, int N, int K, void* Y, cudaStream_t s) {
+  if (count < 1 || count > D_MAX_GROUPS) return SQ_ERR_INVALID_ARG;
+  int64_t most = 0;
+  for (int g = 0; g < count; ++g) most = rows[g] > most ? rows[g] : most;
+  if (most < 1 || most > 64) return SQ_ERR_INVALID_ARG;
+  if (most <= 16) return launch_decode_grouped<16>(Xq, sx, M_total, count, Wq, sw, r0, rows, N, K, Y, s);
+  if (most <= 32) return launch_decode_grouped<32>(Xq, sx, M_total, count, Wq, sw, r0, rows, N, K, Y, s);
+  return launch_decode_grouped<64>(Xq, sx, M_total, count, Wq, sw, r0, rows, N, K, Y, s);
+}
 
 bool gemm_decode_supported(int64_t M, int64_t N, int64_t K) {
   return M >= 1 && M <= 64 && N >= 128 && (K % 128 == 0) && K >= 256 && (N % 8 == 0);
