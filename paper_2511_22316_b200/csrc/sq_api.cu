@@ -606,15 +606,20 @@ sq_status_t sq_linear_grouped(const sq_rotation_t* const* rots, int32_t E, const
       const int64_t r = offsets[e + 1] - offsets[e];
       if (r > 0 && !sq::gemm_decode_supported(r, N, K)) small = false;
     }
-    if (small) {
-      const int cap = sq::gemm_decode_max_groups();
+    // Larger expert batches: the CTA-pair kernel over up to sixteen experts per launch (one tile list: the
+    // last wave of one expert's tiles no longer leaves SMs idle, and there is one start-up instead of E).
+    const bool pairs = !small && sq::gemm_pair_supported(129, N, K);
+    if (small || pairs) {
+      const int cap = small ? sq::gemm_decode_max_groups() : sq::gemm_pair_max_groups();
       std::vector<const void*> gw, gs;
       std::vector<int64_t> g0, gr;
       auto flush = [&]() -> sq_status_t {
         if (gw.empty()) return SQ_OK;
-        const sq_status_t fs = sq::launch_w4a4_gemm_decode_grouped(Xq, sx, M, static_cast<int>(gw.size()), gw.data(),
-                                                                   gs.data(), g0.data(), gr.data(), static_cast<int>(N),
-                                                                   static_cast<int>(K), Y, s);
+        const sq_status_t fs =
+            small ? sq::launch_w4a4_gemm_decode_grouped(Xq, sx, M, static_cast<int>(gw.size()), gw.data(), gs.data(),
+                                                        g0.data(), gr.data(), static_cast<int>(N), static_cast<int>(K), Y, s)
+                  : sq::launch_w4a4_gemm_pair_grouped(Xq, sx, M, static_cast<int>(gw.size()), gw.data(), gs.data(),
+                                                      g0.data(), gr.data(), static_cast<int>(N), static_cast<int>(K), Y, s);
         gw.clear(); gs.clear(); g0.clear(); gr.clear();
         return fs;
       };

@@ -74,11 +74,27 @@ bool make_out_map(CUtensorMap* map, void* Y, uint64_t M, uint64_t N) {
              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
-template <int S_OP, int S_ST>
-__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1)
-w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
-                      const __grid_constant__ CUtensorMap tmap_y, const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
-                      __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
+// The grouped form (one launch for the experts of a mixture-of-experts layer): expert g has its own packed
+// weights, channel steps and output map (Y restricted to its rows, so that the TMA store clips there) and
+// owns rows[g] consecutive token rows from r0[g] on of a common Xq and sx.  Its tiles are tile0[g] ..
+// tile0[g + 1] - 1 of the launch, token tiles innermost as in the plain form.
+constexpr int P_MAX_GROUPS = 16;
+struct alignas(64) PairGroups {
+  CUtensorMap wmap[P_MAX_GROUPS];
+  CUtensorMap ymap[P_MAX_GROUPS];
+  const __half* sw[P_MAX_GROUPS];
+  int r0[P_MAX_GROUPS];
+  int rows[P_MAX_GROUPS];
+  int tile0[P_MAX_GROUPS + 1];
+  int count;
+};
+
+// GROUPED: the tiles run over the experts of `G`; tmap_w, tmap_y, sw and M are unused.
+template <int S_OP, int S_ST, bool GROUPED>
+__device__ __forceinline__ void w4a4_gemm_pair_body(const CUtensorMap& tmap_x, const CUtensorMap& tmap_w,
+                                                    const CUtensorMap& tmap_y, const __half* __restrict__ sx,
+                                                    const __half* __restrict__ sw, int M, int N, int K,
+                                                    int32_t* __restrict__ accdbg, const PairGroups* G) {
   using L = PairSmem<S_OP, S_ST>;
   griddep_launch_dependents();          // a rotate kernel launched behind this one may set itself up on SMs that fall idle
   extern __shared__ unsigned char smem_dyn[];
@@ -98,7 +114,21 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   const int num_kb = K / 128;
   const int num_sb = (num_kb + 1) / 2;
   const int tiles_n = (N + P_TILE_N - 1) / P_TILE_N, tiles_m = (M + P_TILE_M - 1) / P_TILE_M;
-  const int num_tiles = tiles_n * tiles_m;
+  const int num_tiles = GROUPED ? G->tile0[G->count] : tiles_n * tiles_m;
+  // tile -> expert g, first token row of the tile within the expert, first channel of the tile
+  auto locate = [&](int tile, int& g, int& mrow, int& ncol) {
+    if constexpr (GROUPED) {
+      g = 0;
+      while (g + 1 < G->count && tile >= G->tile0[g + 1]) ++g;
+      const int local = tile - G->tile0[g], tm = (G->rows[g] + P_TILE_M - 1) / P_TILE_M;
+      mrow = (local % tm) * P_TILE_M;
+      ncol = (local / tm) * P_TILE_N;
+    } else {
+      g = 0;
+      mrow = (tile % tiles_m) * P_TILE_M;
+      ncol = (tile / tiles_m) * P_TILE_N;
+    }
+  };
   const uint32_t limit = wait_limit();
   const int pre_sb = num_sb < S_ST ? num_sb : S_ST;    // blocks whose weights are requested during set-up
 
@@ -120,10 +150,12 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     // The weights of the first tile's first blocks do not depend on the kernel launched before this
     // one: they are requested now (local barriers only), the activations after the wait below.
     if (pair < num_tiles) {
-      const int n0 = (pair / tiles_m) * P_TILE_N + static_cast<int>(rank) * 128;
+      int g, mrow, ncol;
+      locate(pair, g, mrow, ncol);
+      const int n0 = ncol + static_cast<int>(rank) * 128;
       for (int sb = 0; sb < pre_sb; ++sb) {
         mbar_arrive_expect_tx(&st_full[sb], L::A_ST + L::B_ST);
-        tma_load_2d(smem + L::OFF_B_ST + sb * L::B_ST, &tmap_w, &st_full[sb], sb * 128, n0);
+        tma_load_2d(smem + L::OFF_B_ST + sb * L::B_ST, GROUPED ? &G->wmap[g] : &tmap_w, &st_full[sb], sb * 128, n0);
       }
     }
   }
@@ -147,8 +179,11 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
       // tiles and all of X, which stays in L2; with the channel tiles innermost every token tile
       // streamed the whole weight matrix from HBM again once it no longer fitted L2.
       for (int tile = pair; tile < num_tiles && ok; tile += npairs) {
-        const int m0 = (tile % tiles_m) * P_TILE_M + static_cast<int>(rank) * 128;
-        const int n0 = (tile / tiles_m) * P_TILE_N + static_cast<int>(rank) * 128;
+        int g, mrow, ncol;
+        locate(tile, g, mrow, ncol);
+        const int m0 = (GROUPED ? G->r0[g] : 0) + mrow + static_cast<int>(rank) * 128;    // row of Xq
+        const int n0 = ncol + static_cast<int>(rank) * 128;
+        const CUtensorMap* wm = GROUPED ? &G->wmap[g] : &tmap_w;
         for (int sb = 0; sb < num_sb; ++sb, ++it) {
           const int ss = it % S_ST;
           if (it < static_cast<uint32_t>(pre_sb)) {     // armed and half loaded during set-up
@@ -159,7 +194,7 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
           if (!ok) break;
           mbar_arrive_expect_tx(&st_full[ss], L::A_ST + L::B_ST);
           tma_load_2d(smem + L::OFF_A_ST + ss * L::A_ST, &tmap_x, &st_full[ss], sb * 128, m0);
-          tma_load_2d(smem + L::OFF_B_ST + ss * L::B_ST, &tmap_w, &st_full[ss], sb * 128, n0);
+          tma_load_2d(smem + L::OFF_B_ST + ss * L::B_ST, wm, &st_full[ss], sb * 128, n0);
         }
       }
     }
@@ -298,14 +333,18 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
     uint32_t tcount = 0, nstore = 0;
     bool ok = true;
     for (int tile = pair; tile < num_tiles && ok; tile += npairs, ++tcount) {
-      const int m0 = (tile % tiles_m) * P_TILE_M + static_cast<int>(rank) * 128;
-      const int n0 = (tile / tiles_m) * P_TILE_N;
+      int tg, mrow, n0;
+      locate(tile, tg, mrow, n0);
+      const int Mt = GROUPED ? G->rows[tg] : M;            // token rows of the tile's expert
+      const int trow0 = GROUPED ? G->r0[tg] : 0;           // the first of them in Xq and sx
+      const int m0 = mrow + static_cast<int>(rank) * 128;
       // Fetched while the MMAs still run: this row's token step, and the channel steps of the warp's
       // 128 columns, four per lane (handed round by shuffles when a chunk needs them).
-      const int row0 = m0 + q * 32, row = row0 + lane;
-      const float sxv = (row < M) ? __half2float(sx[row]) : 0.0f;
+      const int row0 = m0 + q * 32, row = row0 + lane;     // rows within the expert (= rows of its Y map)
+      const float sxv = (row < Mt) ? __half2float(sx[trow0 + row]) : 0.0f;
       const int swcol = n0 + c_first * 32 + 4 * lane;
-      const uint2 swp = (swcol < N) ? __ldg(reinterpret_cast<const uint2*>(sw + swcol)) : make_uint2(0u, 0u);
+      const uint2 swp = (swcol < N) ? __ldg(reinterpret_cast<const uint2*>((GROUPED ? G->sw[tg] : sw) + swcol))
+                                    : make_uint2(0u, 0u);
       ok = mbar_wait(tmem_full, tcount & 1, PSITE_TMEM_FULL, limit);
       if (!ok) break;
       tc_fence_after_sync();
@@ -336,8 +375,8 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
           swraw.w = __shfl_sync(0xffffffffu, swp.y, 8 * j + 2 * g + 1);
           int32_t a[8];
           *reinterpret_cast<uint4*>(buf + lane * 64 + ((g ^ ((lane >> 1) & 3)) << 4)) = dequant8(&r[g * 8], sxv, swraw, a);
-          if (accdbg != nullptr && row < M && col0 + g * 8 < N) {
-            int32_t* arow = accdbg + static_cast<size_t>(row) * N + col0 + g * 8;
+          if (accdbg != nullptr && row < Mt && col0 + g * 8 < N) {
+            int32_t* arow = accdbg + static_cast<size_t>(trow0 + row) * N + col0 + g * 8;
             *reinterpret_cast<int4*>(arow) = make_int4(a[0], a[1], a[2], a[3]);
             *reinterpret_cast<int4*>(arow + 4) = make_int4(a[4], a[5], a[6], a[7]);
           }
@@ -345,7 +384,7 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
         fence_proxy_async_smem();                       // the tile in `buf` -> visible to the TMA store
         __syncwarp();
         if (lane == 0) {
-          if (row0 < M && col0 < N) tma_store_2d(&tmap_y, buf, col0, row0);
+          if (row0 < Mt && col0 < N) tma_store_2d(GROUPED ? &G->ymap[tg] : &tmap_y, buf, col0, row0);
           tma_store_commit();
         }
       }
@@ -363,7 +402,67 @@ w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_c
   }
 }
 
+template <int S_OP, int S_ST>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1)
+w4a4_gemm_pair_kernel(const __grid_constant__ CUtensorMap tmap_x, const __grid_constant__ CUtensorMap tmap_w,
+                      const __grid_constant__ CUtensorMap tmap_y, const __half* __restrict__ sx, const __half* __restrict__ sw, int M, int N, int K,
+                      __half* __restrict__ Y, int32_t* __restrict__ accdbg) {
+  (void)Y;                                              // the output goes through tmap_y
+  w4a4_gemm_pair_body<S_OP, S_ST, false>(tmap_x, tmap_w, tmap_y, sx, sw, M, N, K, accdbg, nullptr);
+}
+
+template <int S_OP, int S_ST>
+__global__ void __cluster_dims__(2, 1, 1) __launch_bounds__(P_THREADS, 1)
+w4a4_gemm_pair_grouped_kernel(const __grid_constant__ PairGroups G, const __grid_constant__ CUtensorMap tmap_x,
+                              const __half* __restrict__ sx, int N, int K) {
+  w4a4_gemm_pair_body<S_OP, S_ST, true>(tmap_x, G.wmap[0], G.ymap[0], sx, nullptr, 0, N, K, nullptr, &G);
+}
+
 }  // namespace
+
+int gemm_pair_max_groups() { return P_MAX_GROUPS; }
+
+// Step 3 for up to P_MAX_GROUPS experts in one launch: expert g owns rows[g] >= 1 token rows from r0[g] on of
+// Xq [M_total x K/2], sx and Y, and has its own Wq[g], sw[g].  Shapes as gemm_pair_supported (whatever rows[g]).
+sq_status_t launch_w4a4_gemm_pair_grouped(const void* Xq, const void* sx, int64_t M_total, int count,
+                                          const void* const* Wq, const void* const* sw, const int64_t* r0,
+                                          const int64_t* rows, int N, int K, void* Y, cudaStream_t s) {
+  constexpr int S_OP = 3, S_ST = 3;
+  using L = PairSmem<S_OP, S_ST>;
+  if (count < 1 || count > P_MAX_GROUPS) return SQ_ERR_INVALID_ARG;
+  PairGroups G;
+  CUtensorMap mx;
+  if (!make_packed_map(&mx, Xq, static_cast<uint64_t>(M_total), K / 2, 128)) return SQ_ERR_CUDA;
+  const int tiles_n = (N + P_TILE_N - 1) / P_TILE_N;
+  long long total = 0;
+  for (int g = 0; g < P_MAX_GROUPS; ++g) {
+    const int src = g < count ? g : 0;                   // unused entries repeat the first (never read)
+    if (rows[src] < 1) return SQ_ERR_INVALID_ARG;
+    void* Yg = static_cast<unsigned char*>(Y) + static_cast<size_t>(r0[src]) * N * 2;
+    if (!make_packed_map(&G.wmap[g], Wq[src], N, K / 2, 128) ||
+        !make_out_map(&G.ymap[g], Yg, static_cast<uint64_t>(rows[src]), N))
+      return SQ_ERR_CUDA;
+    G.sw[g] = static_cast<const __half*>(sw[src]);
+    G.r0[g] = static_cast<int>(r0[src]);
+    G.rows[g] = static_cast<int>(rows[src]);
+    if (g < count) {
+      G.tile0[g] = static_cast<int>(total);
+      total += static_cast<long long>(tiles_n) * ((rows[src] + P_TILE_M - 1) / P_TILE_M);
+    }
+  }
+  if (total > 0x7fffffffll) return SQ_ERR_UNSUPPORTED;
+  for (int g = count; g <= P_MAX_GROUPS; ++g) G.tile0[g] = static_cast<int>(total);
+  G.count = count;
+  auto kern = w4a4_gemm_pair_grouped_kernel<S_OP, S_ST>;
+  if (!ensure_dyn_smem(reinterpret_cast<const void*>(kern), L::DYN_BYTES)) return SQ_ERR_CUDA;
+  const int sms = sm_count();
+  if (sms <= 0) return SQ_ERR_CUDA;
+  const int pairs = total < sms / 2 ? static_cast<int>(total) : sms / 2;
+  const cudaError_t err = launch_maybe_pdl(kern, dim3(2 * pairs), dim3(P_THREADS), L::DYN_BYTES, s, G, mx,
+                                           static_cast<const __half*>(sx), N, K);
+  count_launch();
+  return (err == cudaSuccess && cudaGetLastError() == cudaSuccess) ? SQ_OK : SQ_ERR_CUDA;
+}
 
 bool gemm_pair_supported(int64_t M, int64_t N, int64_t K) {
   return M > 128 && N >= 128 && (K % 128 == 0) && K >= 128 && (N % 8 == 0);

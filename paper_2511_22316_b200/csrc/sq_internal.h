@@ -167,7 +167,12 @@ sq_status_t launch_w4a4_gemm_pair(const void* Xq, const void* sx, const void* Wq
 // Step 3 for decode-sized problems (sq_gemm_decode.cu): weights as the A operand, K split over a
 // thread-block cluster with the partial tiles exchanged on chip (no scratch in global memory).
 bool gemm_decode_supported(int64_t M, int64_t N, int64_t K);
-// The same kernel over the experts of a grouped layer in one launch (a tile = expert x 128 channels).
+// The CTA-pair kernel over the experts of a grouped layer in one launch (any number of rows per expert).
+int gemm_pair_max_groups();
+sq_status_t launch_w4a4_gemm_pair_grouped(const void* Xq, const void* sx, int64_t M_total, int count,
+                                          const void* const* Wq, const void* const* sw, const int64_t* r0,
+                                          const int64_t* rows, int N, int K, void* Y, cudaStream_t s);
+// The decode kernel over the experts of a grouped layer in one launch (a tile = expert x 128 channels).
 int gemm_decode_max_groups();
 sq_status_t launch_w4a4_gemm_decode_grouped(const void* Xq, const void* sx, int64_t M_total, int count,
                                             const void* const* Wq, const void* const* sw, const int64_t* r0,

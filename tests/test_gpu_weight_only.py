@@ -301,7 +301,8 @@ def test_linear_wo_full_size_sampled_rows(sq, w):
 # ------------------------------------------------------------------ the grouped W4A4 layer
 @pytest.mark.parametrize("shared", [False, True], ids=["own_handles", "one_handle"])
 @pytest.mark.parametrize("counts", [[5, 0, 3, 1], [64, 7, 130, 0, 0, 9, 1, 40], [0, 0, 12], [300],
-                                    [64, 33, 17, 16, 1, 2, 0, 48], [3, 1, 4, 1, 5, 9, 2, 6, 5, 3, 5, 8, 9, 7, 9, 3, 2, 3]])
+                                    [64, 33, 17, 16, 1, 2, 0, 48], [3, 1, 4, 1, 5, 9, 2, 6, 5, 3, 5, 8, 9, 7, 9, 3, 2, 3],
+                                    [300, 5, 0, 257, 64, 513, 129]])
 def test_linear_grouped_matches_oracle_and_the_per_expert_calls(sq, counts, shared):
     """Each expert with a handle of its own, and all experts on one handle (then steps 1 and 2 run once
     over all rows and only step 3 per expert): against the oracle, and bit for bit against sq_linear on
@@ -342,8 +343,9 @@ def test_linear_grouped_matches_oracle_and_the_per_expert_calls(sq, counts, shar
     y.check()
     with_rows = sum(1 for c in counts if c > 0)                     # experts without tokens cost nothing
     if shared and with_rows >= 2:
-        # steps 1+2 once; step 3 per expert, or -- every expert within 64 rows -- for sixteen experts per launch
-        assert launched == 1 + ((with_rows + 15) // 16 if max(counts) <= 64 else with_rows)
+        # steps 1+2 once; step 3 for sixteen experts per launch (the decode kernel's grouped form when every
+        # expert has at most 64 rows, else the CTA-pair kernel's)
+        assert launched == 1 + (with_rows + 15) // 16
     else:
         assert launched == 2 * with_rows
     Yg = y.numpy(np.float16, (M, N))
