@@ -252,9 +252,10 @@ sq_status_t sq_linear_wo(const sq_rotation_t* rot, const void* X, int64_t M, con
  * offsets[e] .. offsets[e+1]-1 of X and of Y and has its own packed weights and its own rotation
  * handle (experts that share an input distribution may share a handle).  Each expert's rows go
  * through the same kernels as sq_linear, queued back to back on `stream`; experts without tokens
- * cost nothing.  When every expert with tokens has the SAME handle (and K % 32 == 0), steps 1 and 2
- * run once over all M rows and step 3 runs over up to sixteen experts per launch (one list of tiles
- * over the experts); the outputs are the same bits either way.
+ * cost nothing.  With K % 32 == 0, steps 1 and 2 run once over all M rows when every expert with
+ * tokens has the SAME handle (else once per expert), and step 3 runs over up to sixteen experts per
+ * launch (one list of tiles over the experts); the outputs are the same bits as those of sq_linear
+ * on each expert's rows.
  *   rots          HOST array of E handles (all with n1*n2 == K)
  *   offsets       HOST array of E+1 non-decreasing row offsets, offsets[0] == 0, offsets[E] == M
  *   X             DEVICE fp16 [M x K]

@@ -579,11 +579,12 @@ sq_status_t sq_linear_grouped(const sq_rotation_t* const* rots, int32_t E, const
     if (st == SQ_OK) st = check_handle_device(rot);
     if (st != SQ_OK) return st;
   }
-  // Experts that share one handle (one rotation for the block's common input): steps 1 and 2 run once over
-  // all rows -- one launch that fills the SMs instead of one small launch per expert -- and step 3 once per
-  // expert on its rows of Xq and sx.  A token's codes do not depend on which rows are rotated with it, so
-  // the result is that of the per-expert calls.  (Row slices of Xq start on 16-byte boundaries when
-  // K % 32 == 0; the kernels read the token steps one by one, so a slice of sx may start anywhere.)
+  // All rows share one Xq and one sx in the workspace (row slices of Xq start on 16-byte boundaries when
+  // K % 32 == 0; the kernels read and write the token steps one by one, so a slice of sx may start
+  // anywhere).  Experts that share one handle (one rotation for the block's common input): steps 1 and 2 run
+  // once over all rows -- one launch that fills the SMs instead of one small launch per expert; experts with
+  // handles of their own: one launch each, into their rows.  A token's codes do not depend on which rows
+  // are rotated with it, so the result is that of the per-expert calls.  Step 3 then runs over the experts.
   const sq_rotation_t* shared = nullptr;
   int with_rows = 0;
   bool same = true;
@@ -593,11 +594,21 @@ sq_status_t sq_linear_grouped(const sq_rotation_t* const* rots, int32_t E, const
     if (!shared) shared = rots[e];
     else if (rots[e] != shared) same = false;
   }
-  if (same && with_rows >= 2 && K % 32 == 0) {
+  if (with_rows >= 2 && K % 32 == 0) {
     cudaStream_t s = static_cast<cudaStream_t>(stream);
     unsigned char* Xq = ws;
     unsigned char* sx = ws + align_up(static_cast<size_t>(M) * (K / 2), 256);
-    sq_status_t st = sq::rotate_quant_dispatch(shared, X, M, Xq, sx, nullptr, s);
+    sq_status_t st = SQ_OK;
+    if (same) {
+      st = sq::rotate_quant_dispatch(shared, X, M, Xq, sx, nullptr, s);
+    } else {
+      for (int32_t e = 0; e < E && st == SQ_OK; ++e) {
+        const int64_t r0 = offsets[e], r = offsets[e + 1] - r0;
+        if (r > 0)
+          st = sq::rotate_quant_dispatch(rots[e], Xb + static_cast<size_t>(r0) * K * 2, r,
+                                         Xq + static_cast<size_t>(r0) * (K / 2), sx + static_cast<size_t>(r0) * 2, nullptr, s);
+      }
+    }
     if (st != SQ_OK) return st;
     // Decode-sized expert batches (at most 64 rows each): step 3 for up to sixteen experts per launch, a
     // tile being (expert, 128 channels) -- one start-up and one stream of weights instead of one per expert.

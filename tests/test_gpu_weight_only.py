@@ -342,10 +342,10 @@ def test_linear_grouped_matches_oracle_and_the_per_expert_calls(sq, counts, shar
     _sync_ok(sq)
     y.check()
     with_rows = sum(1 for c in counts if c > 0)                     # experts without tokens cost nothing
-    if shared and with_rows >= 2:
-        # steps 1+2 once; step 3 for sixteen experts per launch (the decode kernel's grouped form when every
-        # expert has at most 64 rows, else the CTA-pair kernel's)
-        assert launched == 1 + (with_rows + 15) // 16
+    if with_rows >= 2:
+        # steps 1+2 once (one handle) or once per expert; step 3 for sixteen experts per launch (the decode
+        # kernel's grouped form when every expert has at most 64 rows, else the CTA-pair kernel's)
+        assert launched == (1 if shared else with_rows) + (with_rows + 15) // 16
     else:
         assert launched == 2 * with_rows
     Yg = y.numpy(np.float16, (M, N))
