@@ -6,7 +6,7 @@ the named workload.  Prints ONE JSON line.
 
   python bench.py [--gpus N] [--steps K] [--warmup W] [--workload NAME] [--impl ours|reference]
                   [--structured-r2] [--fuse-decode] [--no-sweep] [--no-cpu-baseline] [--quick]
-                  [--variants-only]
+                  [--variants-only [--grouped-tokens T]]
 
 After the headline workload the default run also times every other benchmark workload briefly and
 reports them under "per_workload" of the same line, and the weight-only variant (W4A16 / W3A16) and the
@@ -645,6 +645,10 @@ def run_variants_only(args, w):
     sqbuild.build()
     sq.load()
     l2 = torch.cuda.get_device_properties(0).L2_cache_size
+    if args.grouped_tokens:
+        entry = grouped_entry(sq, torch, l2, T=args.grouped_tokens)
+        print(json.dumps({"variants": {"grouped": entry}, "n_gpus": 1, "data": "synthetic"}))
+        return 0
     entry = weight_only_entry(sq, torch, w, 4, peaks(), l2, quick=args.quick)
     print(json.dumps({"variants": {"weight_only": {f"{w.name}_w4a16": entry}}, "n_gpus": 1, "data": "synthetic"}))
     return 0
@@ -896,6 +900,9 @@ def main():
     ap.add_argument("--variants-only", action="store_true",
                     help="time only the weight-only variant of the named workload (W4A16) and print it under "
                          "\"variants\" (for profiler runs of those kernels)")
+    ap.add_argument("--grouped-tokens", type=int, default=0,
+                    help="with --variants-only: time the grouped (mixture-of-experts) layer on this many tokens "
+                         "instead of the weight-only variant")
     args = ap.parse_args()
     if args.quick:
         args.no_sweep = args.no_cpu_baseline = True
