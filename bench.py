@@ -44,13 +44,13 @@ INT8_OVER_BF16 = 2.0      # nominal dense ratio (4.5 POPS int8 : 2.25 PFLOP/s bf
 # dram__bytes_read.sum + dram__bytes_write.sum per launch from the ncu captures summarised under
 # profiles/ (bytes; None until a capture exists for that kernel and workload).
 NCU_TRAFFIC = {
-    ("gemm", "llama2_7b_qkvo_prefill"): 12632832,           # w4a4_gemm_pair_kernel: reads (Y stays in L2)
-    ("rotate_quant", "llama2_7b_qkvo_prefill"): 16888576,   # rotate_quant_tc_kernel
+    ("gemm", "llama2_7b_qkvo_prefill"): 12632576,           # w4a4_gemm_pair_kernel: reads (Y stays in L2)
+    ("rotate_quant", "llama2_7b_qkvo_prefill"): 16888320,   # rotate_quant_tc_kernel
     ("rotate_quant_st", "llama2_7b_qkvo_prefill"): 16873472,  # rotate_quant_st_kernel (--structured-r2)
-    ("gemm", "llama3_8b_up_decode_m16"): 29457152,          # w4a4_gemm_decode_kernel, K not split
-    ("gemm", "llama3_8b_down_decode_m16"): 29519616,        # w4a4_gemm_decode_kernel, K over clusters of 4
-    ("gemm", "llama3_8b_up_decode_m1"): 29409024,           # w4a4_gemv_kernel
-    ("rotate_quant", "llama2_7b_down_prefill"): 45412608,   # rotate_quant_pair_kernel
+    ("gemm", "llama3_8b_up_decode_m16"): 29457408,          # w4a4_gemm_decode_kernel, K not split
+    ("gemm", "llama3_8b_down_decode_m16"): 29518592,        # w4a4_gemm_decode_kernel, K over clusters of 4
+    ("gemm", "llama3_8b_up_decode_m1"): 29408768,           # w4a4_gemv_kernel
+    ("rotate_quant", "llama2_7b_down_prefill"): 45464320,   # rotate_quant_pair_kernel
     ("rotate_quant", "llama2_70b_gateup_prefill"): 69889536,   # rotate_quant_tc_kernel, n2 = 128
     ("rotate_quant", "llama2_70b_down_prefill"): 275649024,    # rotate_quant_pair_kernel, n2 = 128
     ("wo_gemm", "llama3_8b_up_decode_m16"): 29558016,       # wo_gemm_tmem_kernel<16, 4, 8> (W4A16)
