@@ -344,6 +344,8 @@ GEMM_SHAPES = [
     # tiles per pair and more k-blocks than the operand ring holds
     (129, 128, 128), (256, 256, 128), (200, 136, 384), (384, 520, 1664), (1000, 1288, 896),
     (513, 2304, 2176),
+    # more CTA-pair shapes: N a multiple of 64 only, several bands with a ragged last one
+    (300, 1024, 256), (520, 832, 384), (2048, 4096, 128), (1100, 1792, 640),
     # 65..128 tokens: the pair kernel with a half-empty tile (many channel tiles or short K) or the
     # decode kernel twice (few channels, long K), with one and with 63 rows in the second launch
     (100, 9608, 512), (96, 520, 8192), (65, 256, 6144), (127, 264, 4096),
